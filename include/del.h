@@ -1,0 +1,198 @@
+/*
+ * libdel — the hot path of one greedy self-speculative decode round with dynamic exit-layer
+ * selection (DEL) on a Llama-style decoder, as hand-written CUDA kernels for sm_100a.
+ *
+ * The calls follow the paper's statement of the method:
+ *   Sec. 2 ("Early-exit self-speculative decoding"): draft gamma tokens with the first E layers plus the
+ *          LM head, verify them with the full model, reusing the KV cache written while drafting;
+ *   Sec. 2 ("Speculative decoding", greedy case): keep the longest prefix of drafts whose tokens equal
+ *          the target model's top-1 tokens, plus the target's next token (1..gamma+1 tokens per round);
+ *   Sec. 4.2: run the LM head over every layer's cached hidden states of the round ("shadow tokens"),
+ *          count matches with the target's tokens inside the valid context, keep decayed sums;
+ *   Sec. 4.1 (Eq. 1) and Sec. 4.3: pick the next (E, gamma) maximising expected tokens per loaded layer;
+ *   Algorithm 1: the loop (without its confidence-threshold early break).
+ *
+ * Conventions
+ *   - Plain C ABI.  Every pointer is either HOST or DEVICE memory as stated per field/argument.
+ *   - Return value 0 on success, a negative DEL_E* code otherwise; nothing throws or aborts.
+ *   - The library never allocates device memory: weights, KV pages, page table and the workspace are
+ *     allocated by the caller, stay owned by the caller and must outlive the context.  Weights are
+ *     never written.  KV pages, the page table and the workspace are written only by work enqueued on
+ *     the stream given to del_init.  The context itself (host bookkeeping, pinned staging buffers,
+ *     events) is owned by the library and freed by del_destroy.
+ *   - All device work is enqueued on that one stream.  Calls documented "async" return without
+ *     synchronising; the others synchronise the stream before returning.
+ *   - One context serves max_batch independent sequences (0 <= seq < max_batch), each with its own
+ *     committed length, acceptance statistics and (E, gamma).
+ *   - Layers are 1-based (layer 0 = embedding output); gamma = 0 is a legal speculation length and
+ *     makes a round one plain auto-regressive step.
+ */
+#ifndef DEL_H
+#define DEL_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DEL_MAX_GAMMA 31          /* largest g_max accepted by del_init */
+#define DEL_MAX_ROWS 64           /* most rows (over all sequences) one layer pass may carry */
+
+enum {
+    DEL_OK = 0,
+    DEL_EINVAL = -1,              /* bad shape, bad argument, E or gamma out of range */
+    DEL_ENOSPC = -2,              /* KV pages or max_seq exhausted, workspace too small */
+    DEL_ESTATE = -3,              /* call order wrong (e.g. verify before draft, round before prefill) */
+    DEL_ETIMEOUT = -4,            /* a bounded device-side wait expired (kernel reported it) */
+    DEL_ECUDA = -5                /* a CUDA call failed; see del_last_cuda_error */
+};
+
+typedef struct del_ctx del_ctx;   /* opaque, owned by the library */
+
+/* Model shape, cache geometry and DEL hyper-parameters.
+ * Requirements checked by del_init: head_dim in {64, 128}; n_heads % n_kv_heads == 0;
+ * d_model % 32 == 0; vocab % 32 == 0; d_ffn % 16 == 0; page_size == 16; max_seq % page_size == 0;
+ * 1 <= e_min <= e_max < n_layers; 0 <= g_min <= g_max <= DEL_MAX_GAMMA;
+ * max_batch * (g_max + 1) <= DEL_MAX_ROWS; 1 <= init_window <= 32. */
+typedef struct {
+    int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+    float rms_eps, rope_theta;    /* rope_theta is informational: the tables below are what is used */
+    int32_t max_batch, max_seq, page_size, n_pages;
+    int32_t e_min, e_max, g_min, g_max;   /* search ranges of the selection (Sec. 4.3) */
+    int32_t init_window;          /* prompt positions that seed the statistics (App. B.2: 32) */
+    double omega;                 /* decay of the acceptance statistics (App. B.2: 0.95) */
+} del_shape;
+
+/* All tensors bf16 in DEVICE memory, matrices row-major [out_features, in_features].  The per-layer
+ * members are HOST arrays of n_layers DEVICE pointers (index l-1 for layer l); the arrays themselves
+ * are read only during del_init. */
+typedef struct {
+    const void *tok_emb;          /* [vocab, d_model] */
+    const void *final_norm;       /* [d_model] gains of the final RMSNorm (shared by every exit) */
+    const void *lm_head;          /* [vocab, d_model] */
+    const void *const *attn_norm; /* [d_model] */
+    const void *const *wq;        /* [n_heads*head_dim, d_model] */
+    const void *const *wk;        /* [n_kv_heads*head_dim, d_model] */
+    const void *const *wv;        /* [n_kv_heads*head_dim, d_model] */
+    const void *const *wo;        /* [d_model, n_heads*head_dim] */
+    const void *const *ffn_norm;  /* [d_model] */
+    const void *const *w_gate;    /* [d_ffn, d_model] */
+    const void *const *w_up;      /* [d_ffn, d_model] */
+    const void *const *w_down;    /* [d_model, d_ffn] */
+    const float *rope_cos;        /* DEVICE fp32 [max_seq, head_dim/2]: cos(pos * theta^(-2j/head_dim)) */
+    const float *rope_sin;        /* DEVICE fp32 [max_seq, head_dim/2]; pairing is (j, j + head_dim/2) */
+} del_weights;
+
+/* Paged KV cache in DEVICE memory.  The library assigns pages to sequences and writes page_table.
+ *   k_pages: bf16 [n_pages][n_layers][n_kv_heads][page_size][head_dim]   (keys after rotary embedding)
+ *   v_pages: bf16 [n_pages][n_layers][n_kv_heads][head_dim][page_size]   (values, transposed per page)
+ *   page_table: int32 [max_batch][max_seq / page_size] */
+typedef struct {
+    void *k_pages, *v_pages;
+    int32_t *page_table;
+} del_kv;
+
+/* Result of one round for one sequence (HOST memory). */
+typedef struct {
+    int32_t E, gamma;             /* the setting the round ran with */
+    int32_t g;                    /* drafts made: gamma clipped to the tokens still wanted minus one */
+    int32_t n_accept;             /* accepted drafts, 0..g */
+    int32_t n_emitted;            /* n_accept + 1; 0 if the sequence was not live */
+    int32_t tokens[DEL_MAX_GAMMA + 1];   /* the n_emitted tokens committed by the round */
+    int32_t next_E, next_gamma;   /* choice for the next round */
+    int32_t status;               /* 0, or a DEL_E* code reported by a kernel */
+} del_round_out;
+
+/* Bytes of DEVICE workspace del_init needs for this shape (256-byte aligned base expected). */
+size_t del_workspace_bytes(const del_shape *shape);
+
+/* Creates a context.  shape, weights, kv: HOST structs (copied).  workspace: DEVICE, ws_bytes >=
+ * del_workspace_bytes(shape); its contents are clobbered.  cuda_stream: a cudaStream_t (0 = default
+ * stream).  Errors: DEL_EINVAL (shape requirements, null pointers), DEL_ENOSPC (workspace too small,
+ * n_pages cannot hold even one sequence), DEL_ECUDA. */
+int del_init(del_ctx **ctx, const del_shape *shape, const del_weights *weights, const del_kv *kv,
+             void *workspace, size_t ws_bytes, void *cuda_stream);
+
+/* Prefill (Algorithm 1, "Require"; Sec. 4.3 last sentence; App. B.2): runs all layers over the prompt
+ * (HOST int32 [n_prompt], 1 <= n_prompt, n_prompt + max_new_tokens + g_max + 1 <= max_seq), fills the KV
+ * cache, computes every layer's shadow tokens over the last min(init_window, n_prompt) positions,
+ * seeds the statistics with their agreement with the last layer, emits the first token and picks the
+ * first (E, gamma).  max_new_tokens (>= 1) counts that first token; later rounds clip gamma so that
+ * exactly max_new_tokens tokens are produced.  Any previous state of `seq` is released first.
+ * Synchronises.  first_out (HOST, may be NULL): n_emitted = 1, tokens[0], next_E, next_gamma. */
+int del_prefill(del_ctx *ctx, int seq, const int32_t *prompt, int n_prompt, int max_new_tokens,
+                del_round_out *first_out);
+
+/* Draft phase (Sec. 2 early-exit drafting; Algorithm 1 draft loop without the break): gamma tokens,
+ * each through embedding, layers 1..E, shared final RMSNorm, LM head, argmax.  gamma is clipped like
+ * in del_round.  Async.  Errors: DEL_EINVAL (E outside [1, n_layers-1], gamma outside [0, g_max]),
+ * DEL_ESTATE (no prefill, sequence finished, previous round not completed), DEL_ENOSPC. */
+int del_draft(del_ctx *ctx, int seq, int E, int gamma);
+
+/* Verify phase (Sec. 2; Algorithm 1 "Verify D by M_p"): the last input token through layers 1..E, then
+ * the g+1 positions through layers E+1..L starting from the exit layer's cached hidden states; KV
+ * written for all g+1 positions; every layer's hidden state of every position kept.  Async.
+ * DEL_ESTATE unless del_draft came before. */
+int del_verify(del_ctx *ctx, int seq);
+
+/* Shadow tokens, acceptance and statistics (Sec. 4.2, Algorithm 1 DEL_Update up to the alpha update):
+ * one LM-head pass over the stacked hidden states of all layers and positions with a fused argmax,
+ * longest-matching-prefix acceptance, per-layer match counts over the n_accept+1 valid positions,
+ * decayed sums.  Commits the accepted tokens.  Synchronises (the host learns n_accept).
+ * out (HOST, may be NULL) gets everything except next_E / next_gamma. */
+int del_layer_accept(del_ctx *ctx, int seq, del_round_out *out);
+
+/* Selection (Eq. 1 in its sum form, Sec. 4.3): argmax over E in [e_min, e_max], gamma in
+ * [g_min, g_max] of (sum_{k<=gamma} alpha_E^k) / (gamma*E + L), first maximum in E-major order.
+ * Synchronises; writes the choice to *E and *gamma (HOST, may be NULL) and keeps it for del_round. */
+int del_select(del_ctx *ctx, int seq, int32_t *E, int32_t *gamma);
+
+/* One whole round for every live sequence at once (each with its own E, gamma and state): draft,
+ * verify, layer_accept and select with layer passes shared by the sequences, one host
+ * synchronisation at the end.  out: HOST array [max_batch]; entries of sequences that are not live
+ * get n_emitted = 0.  Returns DEL_ESTATE if no sequence is live. */
+int del_round(del_ctx *ctx, del_round_out *out);
+
+/* Fix the policy of a sequence: del_round uses (E, gamma) as given instead of the selection
+ * (gamma = 0: plain auto-regressive decoding).  E <= 0 restores the dynamic choice. */
+int del_set_policy(del_ctx *ctx, int seq, int E, int gamma);
+
+/* Acceptance statistics, for resuming and for tests.  Sc: HOST double [n_layers], entry l-1 is the
+ * decayed match count of layer l; Sn: decayed number of valid positions.  Synchronise. */
+int del_get_stats(del_ctx *ctx, int seq, double *Sc, double *Sn, int32_t *E, int32_t *gamma);
+int del_set_stats(del_ctx *ctx, int seq, const double *Sc, double Sn, int32_t E, int32_t gamma);
+
+/* Introspection for tests; all synchronise and copy to HOST memory.
+ *   del_get_shadow: int32 [n_layers][g_max + 1] shadow tokens and int32 [n_layers] match counts of the
+ *                   last del_layer_accept of `seq` (either pointer may be NULL).
+ *   del_get_hidden: fp32 [d_model], hidden state of `layer` (0..n_layers) at row `row` of the last pass.
+ *   del_debug_logits: fp32 [vocab], logits of the exit head applied to that hidden state, computed by a
+ *                   separate unfused kernel.
+ *   del_get_kv:     fp32 [n_kv_heads*head_dim] key and value rows of `layer` (1-based) at position pos. */
+int del_get_shadow(del_ctx *ctx, int seq, int32_t *shadow, int32_t *counts);
+int del_get_hidden(del_ctx *ctx, int seq, int layer, int row, float *out);
+int del_debug_logits(del_ctx *ctx, int seq, int layer, int row, float *out);
+int del_get_kv(del_ctx *ctx, int seq, int layer, int pos, float *k_out, float *v_out);
+
+/* Committed length (prompt + emitted tokens) of a sequence, or a negative code. */
+int del_committed_len(del_ctx *ctx, int seq);
+/* Frees the sequence's KV pages and marks it empty. */
+int del_release(del_ctx *ctx, int seq);
+/* Kernel launches enqueued since del_init (for launch accounting). */
+int64_t del_launch_count(const del_ctx *ctx);
+/* Switches of the launch machinery (bit 0: programmatic dependent launch, bit 1: CUDA graphs for
+ * single-sequence rounds, bit 2: tcgen05 LM head instead of the streaming one).  Returns the
+ * previous flags. */
+int del_set_flags(del_ctx *ctx, int flags);
+
+const char *del_strerror(int code);
+/* Text of the last CUDA error seen by this context ("" if none). */
+const char *del_last_cuda_error(const del_ctx *ctx);
+void del_destroy(del_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,112 @@
+/*
+ * CPU oracle for the greedy self-speculative decode round with dynamic exit
+ * layer selection (DEL).  TEST INFRASTRUCTURE ONLY: it exists to check the
+ * CUDA library and to be timed as the CPU baseline; the product never calls it.
+ * It shares no code with the CUDA path.
+ *
+ * Precision: weights are bf16 bit patterns (expanded exactly to float);
+ * activations, the KV cache and logits are stored as float; every reduction
+ * (dot products, mean of squares, softmax sums, attention-weighted sums) is
+ * accumulated in double in a fixed order that does not depend on how many rows
+ * are processed together.  The acceptance statistics and the selection run in
+ * double with no fused multiply-add.
+ *
+ * Pinned by tests/test_oracle_*.py against: an independent non-cached forward
+ * pass, closed forms for RMSNorm / softmax / SiLU / RoPE, greedy speculative ==
+ * greedy auto-regressive for every (E, gamma), the paper's worked example of a
+ * round, brute-force shadow tokens from truncated models, the decayed-sum
+ * definition, and exhaustive evaluation of the tokens-per-layer formula.
+ * Parity unpinned: the absolute values of logits of the random model (no
+ * published activations exist) and any distribution-level behaviour that would
+ * need the paper's trained checkpoints.
+ */
+#ifndef DEL_ORACLE_H
+#define DEL_ORACLE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ORA_MAX_GAMMA 32
+
+typedef struct {
+    int32_t n_layers, d_model, n_heads, n_kv_heads, head_dim, d_ffn, vocab;
+    float rms_eps, rope_theta;
+    int32_t max_seq;
+    int32_t e_min, e_max, g_min, g_max, init_window;
+    double omega;
+} ora_shape;
+
+/* bf16 bit patterns, matrices [out, in] row-major; per-layer arrays have n_layers entries */
+typedef struct {
+    const uint16_t *tok_emb, *final_norm, *lm_head;
+    const uint16_t *const *attn_norm, *const *wq, *const *wk, *const *wv, *const *wo;
+    const uint16_t *const *ffn_norm, *const *w_gate, *const *w_up, *const *w_down;
+} ora_weights;
+
+typedef struct {
+    int32_t E, gamma;        /* the (E, gamma) this round ran with */
+    int32_t g;               /* drafts actually made (gamma clipped near the end of generation) */
+    int32_t n_accept;        /* accepted drafts, 0..g */
+    int32_t n_emitted;       /* n_accept + 1 */
+    int32_t drafts[ORA_MAX_GAMMA];
+    int32_t emitted[ORA_MAX_GAMMA + 1];
+    int32_t next_E, next_gamma;
+    int32_t loaded_layers;   /* g * E + L : the paper's cost of the round */
+    double Sn;               /* decayed number of valid positions after this round */
+} ora_round_info;
+
+typedef struct ora_seq ora_seq;
+
+ora_seq *ora_seq_create(const ora_shape *shape, const ora_weights *w);
+void ora_seq_destroy(ora_seq *s);
+
+/* Fix the policy: (E, gamma) stay as given (gamma = 0 is vanilla auto-regressive decoding).
+ * E <= 0 restores the dynamic selection. */
+void ora_set_policy(ora_seq *s, int32_t fixed_E, int32_t fixed_gamma);
+
+/* Prefill over the prompt, initial statistics from the last init_window positions, first token and
+ * first (E, gamma).  shadow/margin (may be NULL): [n_layers][init_window] row-major, layer 1 first,
+ * only the first W = min(init_window, n_prompt) columns are written.  Returns the first token. */
+int32_t ora_prefill(ora_seq *s, const int32_t *prompt, int32_t n_prompt, int32_t *shadow, float *margin,
+                    ora_round_info *info);
+
+/* One speculative round; remaining = tokens still to be generated (>= 1).
+ * shadow/margin/counts may be NULL; shadow and margin are [n_layers][g_max + 1], counts [n_layers]. */
+int ora_round(ora_seq *s, int32_t remaining, ora_round_info *info, int32_t *shadow, float *margin,
+              int32_t *counts);
+
+/* state access */
+int32_t ora_committed_len(const ora_seq *s);
+void ora_get_stats(const ora_seq *s, double *Sc /*[n_layers], index l-1*/, double *Sn, int32_t *E, int32_t *gamma);
+void ora_set_stats(ora_seq *s, const double *Sc, double Sn, int32_t E, int32_t gamma);
+/* hidden state h^l (l = 0 is the embedding) of row i of the last round / of window column i after prefill */
+const float *ora_hidden(const ora_seq *s, int32_t layer, int32_t row);
+/* cached key / value row of 1-based layer at a position, n_kv_heads * head_dim floats */
+const float *ora_k_row(const ora_seq *s, int32_t layer, int32_t pos);
+const float *ora_v_row(const ora_seq *s, int32_t layer, int32_t pos);
+
+/* building blocks, exposed so that tests can pin each of them */
+void ora_embed(const ora_seq *s, int32_t token, float *h);
+void ora_rmsnorm(const float *x, const uint16_t *gain_bf16, int32_t d, float eps, float *out);
+void ora_rope(float *x, int32_t n_heads, int32_t head_dim, int32_t pos, float theta);
+void ora_softmax(const float *x, int32_t n, double *p);
+float ora_silu(float x);
+/* rows at consecutive positions pos0..pos0+m-1 through 1-based layer; writes K,V at those positions */
+void ora_layer_rows(ora_seq *s, int32_t layer, const float *h_in, int32_t pos0, int32_t m, float *h_out);
+/* shared final RMSNorm + LM head + greedy choice (lowest id on ties); margin = top1 - top2 logit */
+void ora_exit_head(const ora_seq *s, const float *h, int32_t *token, float *margin, float *logits_or_null);
+
+int32_t ora_accept_len(const int32_t *drafts, const int32_t *verified, int32_t g);
+double ora_decay_step(double S, double omega, double a);
+double ora_tpl(double alpha, int32_t l, int32_t d, int32_t L);
+void ora_select(const double *Sc /*index l-1*/, double Sn, int32_t L, int32_t e_min, int32_t e_max, int32_t g_min,
+                int32_t g_max, int32_t *E, int32_t *gamma);
+int ora_num_threads(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

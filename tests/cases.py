@@ -1,0 +1,10 @@
+"""Small model variants shared by the test modules (inputs only; built from synth.Config)."""
+import synth
+
+TINY = synth.CONFIGS["tiny"]
+# grouped-query attention, non-unit norm gains, depth-decaying branches, 6 layers: has rejections
+TINY_GQA = synth.small_variant(TINY, name="tiny_gqa", n_layers=6, n_kv_heads=2, gain_spread=0.1,
+                               residual_scaling="decay", e_min=1, e_max=5, g_max=5, emb_scale=10.0,
+                               prompt_len=40, gen_len=48, seed=77)
+# ragged shapes: prompt shorter than the initialisation window, odd generation length
+TINY_SHORT = synth.small_variant(TINY, name="tiny_short", prompt_len=7, gen_len=21, emb_scale=10.0, seed=5)
