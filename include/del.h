@@ -172,6 +172,10 @@ int del_set_stats(del_ctx *ctx, int seq, const double *Sc, double Sn, int32_t E,
  *                   separate unfused kernel.
  *   del_get_kv:     fp32 [n_kv_heads*head_dim] key and value rows of `layer` (1-based) at position pos. */
 int del_get_shadow(del_ctx *ctx, int seq, int32_t *shadow, int32_t *counts);
+/* int32 [g_max]: the draft tokens of the sequence's last draft phase (first g entries are meaningful). */
+int del_get_drafts(del_ctx *ctx, int seq, int32_t *drafts);
+/* Overrides the token that the next round feeds first (used when resuming from a known stream). */
+int del_force_token(del_ctx *ctx, int seq, int32_t token);
 int del_get_hidden(del_ctx *ctx, int seq, int layer, int row, float *out);
 int del_debug_logits(del_ctx *ctx, int seq, int layer, int row, float *out);
 int del_get_kv(del_ctx *ctx, int seq, int layer, int pos, float *k_out, float *v_out);

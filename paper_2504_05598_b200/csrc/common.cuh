@@ -1,0 +1,134 @@
+// Shared device-side definitions of libdel: plan structures that describe the rows of a layer pass,
+// the device-resident model / workspace description, and small PTX wrappers (streaming 16-byte loads,
+// bf16 tensor-core MMA, programmatic-dependent-launch control).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#define DEL_ROWS_MAX 64        // rows of one layer pass
+#define DEL_SEQ_MAX 16         // sequences per context
+#define DEL_GEMM_THREADS 256
+#define DEL_GEMM_WARPS 8
+
+typedef __nv_bfloat16 bf16;
+
+// One row of a layer pass: which sequence, which slot of the hidden stack, which position of the
+// sequence, and where its input token sits in the token buffer (embedding passes only).
+struct RowDesc {
+    int32_t seq, slot, pos, tok;
+};
+
+// Rows of one sequence inside a pass: consecutive rows, consecutive slots, consecutive positions.
+struct Segment {
+    int32_t seq, row0, nrows, pos0;
+};
+
+struct PassPlan {
+    int32_t m, n_seg, pad0, pad1;
+    RowDesc rows[DEL_ROWS_MAX];
+    Segment seg[DEL_SEQ_MAX];
+};
+
+// Per-sequence state that lives on the device.
+struct SeqState {
+    double Sn;
+    int32_t E, gamma;            // choice for the next round
+    int32_t fixed_E, fixed_gamma;
+    int32_t pad[2];
+};
+
+// Device view of the model shape and of the workspace carve-up (passed by value to kernels).
+struct Dims {
+    int32_t L, d, nh, nkv, hd, F, V;
+    int32_t B, S;                // sequences, hidden-stack slots per sequence
+    int32_t max_seq, page_size, pages_per_seq;
+    int32_t n_sst;               // sum-of-squares partials per row (= d / 16)
+    float eps;
+};
+
+struct Buffers {
+    float *H;                    // [L+1][B][S][d]    hidden stack (layer 0 = embedding)
+    bf16 *XS;                    // [L+1][B][S][d]    h * gain of the next layer's attention norm
+    float *SS;                   // [L+1][B][S][n_sst] partial sums of squares of h
+    bf16 *XE;                    // [B][S][d]         h * gain of the final norm at the exit layer
+    bf16 *Q;                     // [ROWS][nh*hd]
+    bf16 *ATT;                   // [ROWS][nh*hd]
+    float *HM;                   // [ROWS][d]         residual after attention
+    bf16 *XM;                    // [ROWS][d]         HM * gain of the ffn norm
+    float *SSM;                  // [ROWS][n_sst]
+    bf16 *ACT;                   // [ROWS][F]
+    float *APO;                  // attention partial outputs [ROWS][nh][splits][hd]
+    float *APML;                 // attention partial (max, sum) [ROWS][nh][splits][2]
+    int32_t *ACNT;               // [DEL_SEQ_MAX][nkv] arrival counters of the split combine
+    float *LPV;                  // streaming LM head: arg-max partial values [ctas][ROWS]
+    int32_t *LPI;                // ... and indices
+    float *TPV;                  // tensor-core LM head: partial values [R_max][vocab tiles]
+    int32_t *TPI;
+    int32_t *PROMPT_ALL;         // [max_seq] prompt tokens of the sequence being prefilled
+    bf16 *XN;                    // [R_max][d] normalised rows for the batched LM head
+    int32_t *SHADOW;             // [B][L][S] shadow tokens
+    int32_t *COUNTS;             // [B][L]
+    int32_t *TOK;                // [B][S+1] token buffer: [0] next input, [1+i] draft i
+    double *SC;                  // [B][L] decayed match counts
+    SeqState *ST;                // [B]
+    int32_t *ERR;                // device error word
+    bf16 *KP, *VP;               // KV pages
+    int32_t *PT;                 // page table [B][pages_per_seq]
+    const float *rope_cos, *rope_sin;
+};
+
+__device__ __forceinline__ size_t stack_row(const Dims &D, int layer, int seq, int slot) {
+    return ((size_t)layer * D.B + seq) * D.S + slot;
+}
+
+// ---------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// 16-byte streaming load of immutable data (weights): read-only path, no L1 allocation.
+__device__ __forceinline__ uint4 ldg_stream16(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+// 16-byte load of activations written by an earlier kernel (coherent at L2).
+__device__ __forceinline__ uint4 ldg_act16(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint2 ldg_act8(const void *p) {
+    uint2 v;
+    asm volatile("ld.global.cg.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ float ldg_cg_f32(const float *p) {
+    float v;
+    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+
+// D += A(16x16, row) * B(16x8, col), bf16 inputs, fp32 accumulate.
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+__device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
+__device__ __forceinline__ float bf16_to_f(bf16 v) { return __bfloat162float(v); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}

@@ -1,0 +1,311 @@
+// Small kernels around the weight-streaming ones: token embedding, arg-max finalisation of the draft
+// head, row preparation and arg-max reduction of the stacked LM head, prefix acceptance with the
+// acceptance-statistics update, the (E, gamma) selection, and two test-only readers.
+#include "../../include/del.h"
+#include "kernels.h"
+
+namespace {
+
+constexpr int CTL_THREADS = 256;
+
+__device__ __forceinline__ void write_embedding(const CtlArgs &a, int token, int seq, int slot) {
+    // h^0 = embedding row; also the bf16 input of layer 1's attention norm and its partial sums of squares
+    const int d = a.D.d;
+    const bf16 *e = a.tok_emb + (size_t)token * d;
+    const size_t sr = stack_row(a.D, 0, seq, slot);
+    for (int o0 = 0; o0 < d; o0 += CTL_THREADS) {
+        const int o = o0 + threadIdx.x;
+        float h = 0.f;
+        if (o < d) {
+            h = bf16_to_f(e[o]);
+            a.B.H[sr * d + o] = h;
+            a.B.XS[sr * d + o] = __float2bfloat16_rn(h * bf16_to_f(a.gain0[o]));
+        }
+        float ss = h * h;
+        ss += __shfl_xor_sync(0xffffffffu, ss, 8);
+        ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+        ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+        ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+        if (o < d && (o & 15) == 0) a.B.SS[sr * a.D.n_sst + (o >> 4)] = ss;
+    }
+}
+
+__global__ void __launch_bounds__(CTL_THREADS) embed_kernel(const CtlArgs a) {
+    pdl_launch();
+    pdl_wait();
+    const RowDesc rd = a.plan->rows[blockIdx.x];
+    const int token = a.tok_src[rd.tok];
+    write_embedding(a, token, rd.seq, rd.slot);
+}
+
+// block-wide arg-max with ties to the lowest index; result valid in thread 0
+__device__ __forceinline__ void block_argmax(float &v, int &idx) {
+    __shared__ float sv[CTL_THREADS / 32];
+    __shared__ int si[CTL_THREADS / 32];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float v2 = __shfl_xor_sync(0xffffffffu, v, o);
+        const int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
+        if (v2 > v || (v2 == v && i2 < idx)) { v = v2; idx = i2; }
+    }
+    if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = v; si[threadIdx.x >> 5] = idx; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < CTL_THREADS / 32; ++w)
+            if (sv[w] > v || (sv[w] == v && si[w] < idx)) { v = sv[w]; idx = si[w]; }
+    }
+}
+
+// Draft head, last step: reduce the per-CTA arg-max partials of the streaming LM head into the draft
+// token, store it, and write the embedding of that token as the next row of the sequence.
+__global__ void __launch_bounds__(CTL_THREADS) draft_finalize_embed_kernel(const CtlArgs a, int embed_next) {
+    __shared__ int s_tok;
+    pdl_launch();
+    pdl_wait();
+    const int c = blockIdx.x;
+    const RowDesc rd = a.plan->rows[c];
+    float v = -INFINITY;
+    int idx = 0x7fffffff;
+    for (int p = threadIdx.x; p < a.n_part; p += CTL_THREADS) {
+        const float v2 = ldg_cg_f32(a.B.LPV + (size_t)p * DEL_ROWS_MAX + c);
+        const int i2 = a.B.LPI[(size_t)p * DEL_ROWS_MAX + c];
+        if (v2 > v || (v2 == v && i2 < idx)) { v = v2; idx = i2; }
+    }
+    block_argmax(v, idx);
+    if (threadIdx.x == 0) {
+        s_tok = idx;
+        a.B.TOK[rd.seq * (a.D.S + 1) + rd.slot + 1] = idx;
+    }
+    __syncthreads();
+    if (embed_next) write_embedding(a, s_tok, rd.seq, rd.slot + 1);
+}
+
+__device__ __forceinline__ bool locate_row(const UpdatePlan *up, int L, int mode, int rr, int &seq, int &layer, int &slot) {
+    for (int u = 0; u < up->n_seq; ++u) {
+        const int per = mode ? up->s[u].n_valid_init : up->s[u].g + 1;
+        const int r = rr - up->s[u].row0;
+        if (r >= 0 && r < per * L) {
+            seq = up->s[u].seq;
+            layer = r / per + 1;
+            slot = r - (layer - 1) * per;
+            return true;
+        }
+    }
+    return false;
+}
+
+// Stacked LM head input: row (seq, layer, slot) of the hidden stack times the final norm's gain, as
+// bf16.  The norm's 1/rms is a positive per-row scalar and cannot change the arg-max, so it is left out.
+__global__ void __launch_bounds__(CTL_THREADS) prep_rows_kernel(const CtlArgs a, const UpdatePlan *up) {
+    pdl_launch();
+    pdl_wait();
+    int seq, layer, slot;
+    if (!locate_row(up, a.D.L, a.mode, blockIdx.x, seq, layer, slot)) return;
+    const int d = a.D.d;
+    const float *h = a.B.H + stack_row(a.D, layer, seq, slot) * d;
+    bf16 *x = a.B.XN + (size_t)blockIdx.x * d;
+    for (int o = threadIdx.x; o < d; o += CTL_THREADS) x[o] = __float2bfloat16_rn(ldg_cg_f32(h + o) * bf16_to_f(a.final_gain[o]));
+}
+
+// Reduce the vocabulary-tile partials of one stacked row into its shadow token.
+__global__ void __launch_bounds__(CTL_THREADS) shadow_reduce_kernel(const CtlArgs a, const UpdatePlan *up, const float *pv,
+                                                                    const int32_t *pi, int n_part, int pstride, int cstride,
+                                                                    int row_base) {
+    pdl_launch();
+    pdl_wait();
+    const int c = blockIdx.x;
+    float v = -INFINITY;
+    int idx = 0x7fffffff;
+    for (int p = threadIdx.x; p < n_part; p += CTL_THREADS) {
+        const float v2 = ldg_cg_f32(pv + (size_t)p * pstride + (size_t)c * cstride);
+        const int i2 = pi[(size_t)p * pstride + (size_t)c * cstride];
+        if (v2 > v || (v2 == v && i2 < idx)) { v = v2; idx = i2; }
+    }
+    block_argmax(v, idx);
+    if (threadIdx.x == 0) {
+        int seq, layer, slot;
+        if (locate_row(up, a.D.L, a.mode, row_base + c, seq, layer, slot))
+            a.B.SHADOW[((size_t)seq * a.D.L + (layer - 1)) * a.D.S + slot] = idx;
+    }
+}
+
+// Prefix acceptance, per-layer match counts over the valid context and decayed statistics
+// (S <- omega * S + a, no fused multiply-add so that the host oracle's doubles are reproduced).
+__global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const UpdatePlan *up, del_round_out *out) {
+    __shared__ int s_n;
+    pdl_launch();
+    pdl_wait();
+    const int u = blockIdx.x;
+    const int seq = up->s[u].seq, g = up->s[u].g, L = a.D.L, S = a.D.S;
+    const int32_t *sh = a.B.SHADOW + (size_t)seq * L * S;
+    const int32_t *verified = sh + (size_t)(L - 1) * S;
+    int32_t *tok = a.B.TOK + seq * (S + 1);
+    del_round_out *o = out + seq;
+    if (a.mode == 1) {
+        const int W = up->s[u].n_valid_init;
+        for (int l = threadIdx.x; l < L; l += blockDim.x) {
+            int c = 0;
+            for (int j = 0; j < W; ++j) c += (sh[(size_t)l * S + j] == verified[j]);
+            a.B.COUNTS[seq * L + l] = c;
+            a.B.SC[seq * L + l] = (double)c;
+        }
+        if (threadIdx.x == 0) {
+            a.B.ST[seq].Sn = (double)W;
+            tok[0] = verified[W - 1];
+            o->n_accept = 0;
+            o->n_emitted = 1;
+            o->tokens[0] = verified[W - 1];
+        }
+        return;
+    }
+    if (threadIdx.x == 0) {
+        int n = 0;
+        while (n < g && tok[1 + n] == verified[n]) ++n;
+        s_n = n;
+        o->n_accept = n;
+        o->n_emitted = n + 1;
+        for (int i = 0; i <= n; ++i) o->tokens[i] = verified[i];
+        a.B.ST[seq].Sn = __dadd_rn(__dmul_rn(a.omega, a.B.ST[seq].Sn), (double)(n + 1));
+    }
+    __syncthreads();
+    const int n = s_n;
+    for (int l = threadIdx.x; l < L; l += blockDim.x) {
+        int c = 0;
+        for (int i = 0; i <= n; ++i) c += (sh[(size_t)l * S + i] == verified[i]);
+        a.B.COUNTS[seq * L + l] = c;
+        a.B.SC[seq * L + l] = __dadd_rn(__dmul_rn(a.omega, a.B.SC[seq * L + l]), (double)c);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) tok[0] = verified[n];      // next round's input token
+}
+
+// (E, gamma) = argmax of (sum_{k<=gamma} alpha_E^k) / (gamma*E + L), first maximum in E-major order.
+__global__ void __launch_bounds__(64) select_kernel(const CtlArgs a, const UpdatePlan *up, del_round_out *out) {
+    __shared__ double s_best[64];
+    __shared__ int s_g[64];
+    pdl_launch();
+    pdl_wait();
+    const int seq = up->s[blockIdx.x].seq, L = a.D.L;
+    SeqState *st = a.B.ST + seq;
+    int E = a.e_min, G = a.g_min;
+    if (st->fixed_E > 0) {
+        E = st->fixed_E;
+        G = st->fixed_gamma;
+    } else {
+        const double Sn = st->Sn;
+        double bestE = -1.0;
+        for (int l0 = a.e_min; l0 <= a.e_max; l0 += 64) {
+            const int l = l0 + threadIdx.x;
+            double best = -1.0;
+            int bg = a.g_min;
+            if (l <= a.e_max) {
+                const double alpha = __ddiv_rn(a.B.SC[seq * L + l - 1], Sn);
+                double term = 1.0, sum = 1.0;
+                for (int dd = 0; dd <= a.g_max; ++dd) {
+                    if (dd > 0) { term = __dmul_rn(term, alpha); sum = __dadd_rn(sum, term); }
+                    if (dd >= a.g_min) {
+                        const double tpl = __ddiv_rn(sum, (double)(dd * l + L));
+                        if (tpl > best) { best = tpl; bg = dd; }
+                    }
+                }
+            }
+            s_best[threadIdx.x] = best;
+            s_g[threadIdx.x] = bg;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                for (int j = 0; j < 64 && l0 + j <= a.e_max; ++j)
+                    if (s_best[j] > bestE) { bestE = s_best[j]; E = l0 + j; G = s_g[j]; }
+            }
+            __syncthreads();
+        }
+    }
+    if (threadIdx.x == 0) {
+        st->E = E;
+        st->gamma = G;
+        out[seq].next_E = E;
+        out[seq].next_gamma = G;
+    }
+}
+
+// Test-only: logits of the exit head on one hidden row, straightforward one-warp-per-vocab-row dots.
+__global__ void __launch_bounds__(CTL_THREADS) debug_logits_kernel(const CtlArgs a, int layer, int seq, int slot, float *out) {
+    __shared__ float s_red[CTL_THREADS / 32];
+    __shared__ float s_r;
+    const int d = a.D.d;
+    const float *h = a.B.H + stack_row(a.D, layer, seq, slot) * d;
+    float ss = 0.f;
+    for (int o = threadIdx.x; o < d; o += CTL_THREADS) ss += h[o] * h[o];
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int w = 0; w < CTL_THREADS / 32; ++w) t += s_red[w];
+        s_r = rsqrtf(t / (float)d + a.D.eps);
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int v = blockIdx.x * (CTL_THREADS / 32) + warp; v < a.D.V; v += gridDim.x * (CTL_THREADS / 32)) {
+        const bf16 *w = a.lm_head + (size_t)v * d;
+        float acc = 0.f;
+        for (int o = lane; o < d; o += 32) {
+            const float x = bf16_to_f(__float2bfloat16_rn(h[o] * bf16_to_f(a.final_gain[o])));
+            acc += bf16_to_f(w[o]) * x;
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) out[v] = acc * s_r;
+    }
+}
+
+__global__ void gather_kv_kernel(const CtlArgs a, int layer, int seq, int pos, float *k_out, float *v_out) {
+    const int hd = a.D.hd, n = a.D.nkv * hd;
+    const int pg = a.B.PT[seq * a.D.pages_per_seq + (pos >> 4)], sl = pos & 15;
+    for (int e = threadIdx.x; e < n; e += blockDim.x) {
+        const int kvh = e / hd, dim = e - kvh * hd;
+        const size_t base = (((size_t)pg * a.D.L + (layer - 1)) * a.D.nkv + kvh) * 16 * hd;
+        k_out[e] = bf16_to_f(a.B.KP[base + (size_t)sl * hd + dim]);
+        v_out[e] = bf16_to_f(a.B.VP[base + (size_t)dim * 16 + sl]);
+    }
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch(void (*kern)(KArgs...), int grid, int block, cudaStream_t st, bool pdl, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
+}  // namespace
+
+cudaError_t launch_embed(const CtlArgs &a, int m, cudaStream_t st, bool pdl) {
+    return launch(embed_kernel, m, CTL_THREADS, st, pdl, a);
+}
+cudaError_t launch_draft_finalize_embed(const CtlArgs &a, int m, bool embed_next, cudaStream_t st, bool pdl) {
+    return launch(draft_finalize_embed_kernel, m, CTL_THREADS, st, pdl, a, (int)embed_next);
+}
+cudaError_t launch_prep_rows(const CtlArgs &a, const UpdatePlan *up, int n_rows, cudaStream_t st, bool pdl) {
+    return launch(prep_rows_kernel, n_rows, CTL_THREADS, st, pdl, a, up);
+}
+cudaError_t launch_shadow_reduce(const CtlArgs &a, const UpdatePlan *up, const float *pv, const int32_t *pi, int n_part,
+                                 int pstride, int cstride, int row_base, int n_rows, cudaStream_t st, bool pdl) {
+    return launch(shadow_reduce_kernel, n_rows, CTL_THREADS, st, pdl, a, up, pv, pi, n_part, pstride, cstride, row_base);
+}
+cudaError_t launch_update(const CtlArgs &a, const UpdatePlan *up, void *out_dev, int n_seq, cudaStream_t st, bool pdl) {
+    return launch(update_kernel, n_seq, 128, st, pdl, a, up, (del_round_out *)out_dev);
+}
+cudaError_t launch_select(const CtlArgs &a, const UpdatePlan *up, void *out_dev, int n_seq, cudaStream_t st, bool pdl) {
+    return launch(select_kernel, n_seq, 64, st, pdl, a, up, (del_round_out *)out_dev);
+}
+cudaError_t launch_debug_logits(const CtlArgs &a, int layer, int seq, int slot, float *out_dev, cudaStream_t st) {
+    return launch(debug_logits_kernel, 296, CTL_THREADS, st, false, a, layer, seq, slot, out_dev);
+}
+cudaError_t launch_gather_kv(const CtlArgs &a, int layer, int seq, int pos, float *k_out, float *v_out, cudaStream_t st) {
+    return launch(gather_kv_kernel, 1, 256, st, false, a, layer, seq, pos, k_out, v_out);
+}

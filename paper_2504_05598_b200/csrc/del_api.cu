@@ -1,0 +1,861 @@
+// Host side of libdel: the C ABI of include/del.h, the round scheduler (which rows go through which
+// layers in which order), paged-KV bookkeeping and the launch sequence.  No device memory is allocated
+// here: every buffer is carved out of the caller's workspace.
+#include "../../include/del.h"
+#include "kernels.h"
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+namespace {
+
+constexpr int PLAN_RING = 192;
+constexpr int FLAG_PDL = 1, FLAG_GRAPH = 2, FLAG_TC = 4;
+
+struct SeqHost {
+    bool active = false;
+    int T = 0;               // committed positions
+    int remaining = 0;       // tokens still to emit
+    int E = 0, gamma = 0;    // choice for the next round
+    int fixed_E = 0, fixed_gamma = 0;
+    int phase = 0;           // 0 idle, 1 drafted, 2 verified
+    int cur_E = 0, cur_g = 0, cur_gamma = 0;
+    std::vector<int> pages;
+};
+
+struct Carve {
+    size_t off = 0;
+    template <typename T> T *take(void *base, size_t n) {
+        off = (off + 255) & ~(size_t)255;
+        T *p = base ? reinterpret_cast<T *>(reinterpret_cast<char *>(base) + off) : nullptr;
+        off += n * sizeof(T);
+        return p;
+    }
+};
+
+}  // namespace
+
+struct del_ctx {
+    del_shape sh;
+    Dims D;
+    Buffers B;
+    int R_max = 0, n_vtiles = 0;
+    const bf16 *tok_emb, *final_norm, *lm_head;
+    std::vector<const bf16 *> attn_norm, wq, wk, wv, wo, ffn_norm, w_gate, w_up, w_down;
+    cudaStream_t st = nullptr;
+    int n_sms = 148;
+    int flags = FLAG_PDL;
+    SeqHost seq[DEL_SEQ_MAX];
+    std::vector<int> free_pages;
+    std::vector<int32_t> pt_host;
+    // plans
+    PassPlan *plan_host = nullptr, *plan_dev = nullptr;
+    int plan_cur = 0;
+    UpdatePlan *up_host = nullptr, *up_dev = nullptr;      // [2]
+    del_round_out *out_host = nullptr, *out_dev = nullptr; // [B]
+    void *stage_host = nullptr;                            // small pinned scratch
+    float *dbg_dev = nullptr;                              // [V] debug logits / kv rows
+    int64_t launches = 0;
+    char err[256] = {0};
+    cudaError_t last = cudaSuccess;
+};
+
+namespace {
+
+size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max, int &n_vtiles, PassPlan **plan_dev,
+                 UpdatePlan **up_dev, del_round_out **out_dev, float **dbg_dev) {
+    D.L = s.n_layers; D.d = s.d_model; D.nh = s.n_heads; D.nkv = s.n_kv_heads; D.hd = s.head_dim; D.F = s.d_ffn; D.V = s.vocab;
+    D.B = s.max_batch;
+    D.S = std::max(s.g_max + 1, s.init_window);
+    D.max_seq = s.max_seq; D.page_size = s.page_size; D.pages_per_seq = s.max_seq / s.page_size;
+    D.n_sst = s.d_model / 16;
+    D.eps = s.rms_eps;
+    R_max = s.n_layers * std::max(D.S, std::min(s.max_batch * (s.g_max + 1), DEL_ROWS_MAX));
+    n_vtiles = (s.vocab + 127) / 128;
+    const size_t L1 = (size_t)D.L + 1, BS = (size_t)D.B * D.S, qd = (size_t)D.nh * D.hd;
+    Carve c;
+    B.H = c.take<float>(base, L1 * BS * D.d);
+    B.XS = c.take<bf16>(base, L1 * BS * D.d);
+    B.SS = c.take<float>(base, L1 * BS * D.n_sst);
+    B.XE = c.take<bf16>(base, BS * D.d);
+    B.Q = c.take<bf16>(base, DEL_ROWS_MAX * qd);
+    B.ATT = c.take<bf16>(base, DEL_ROWS_MAX * qd);
+    B.HM = c.take<float>(base, (size_t)DEL_ROWS_MAX * D.d);
+    B.XM = c.take<bf16>(base, (size_t)DEL_ROWS_MAX * D.d);
+    B.SSM = c.take<float>(base, (size_t)DEL_ROWS_MAX * D.n_sst);
+    B.ACT = c.take<bf16>(base, (size_t)DEL_ROWS_MAX * D.F);
+    B.APO = c.take<float>(base, (size_t)DEL_ROWS_MAX * D.nh * 16 * D.hd);
+    B.APML = c.take<float>(base, (size_t)DEL_ROWS_MAX * D.nh * 16 * 2);
+    B.ACNT = c.take<int32_t>(base, (size_t)DEL_SEQ_MAX * D.nkv);
+    B.LPV = c.take<float>(base, (size_t)1024 * DEL_ROWS_MAX);
+    B.LPI = c.take<int32_t>(base, (size_t)1024 * DEL_ROWS_MAX);
+    B.TPV = c.take<float>(base, (size_t)(R_max + 128) * n_vtiles);
+    B.TPI = c.take<int32_t>(base, (size_t)(R_max + 128) * n_vtiles);
+    B.PROMPT_ALL = c.take<int32_t>(base, (size_t)D.max_seq);
+    B.XN = c.take<bf16>(base, (size_t)(R_max + 128) * D.d);
+    B.SHADOW = c.take<int32_t>(base, (size_t)D.B * D.L * D.S);
+    B.COUNTS = c.take<int32_t>(base, (size_t)D.B * D.L);
+    B.TOK = c.take<int32_t>(base, (size_t)D.B * (D.S + 1));
+    B.SC = c.take<double>(base, (size_t)D.B * D.L);
+    B.ST = c.take<SeqState>(base, (size_t)D.B);
+    B.ERR = c.take<int32_t>(base, 64);
+    *plan_dev = c.take<PassPlan>(base, PLAN_RING);
+    *up_dev = c.take<UpdatePlan>(base, 2);
+    *out_dev = c.take<del_round_out>(base, (size_t)D.B);
+    *dbg_dev = c.take<float>(base, (size_t)std::max(D.V, 2 * D.nkv * D.hd));
+    return (c.off + 255) & ~(size_t)255;
+}
+
+int validate(const del_shape *s) {
+    if (!s) return DEL_EINVAL;
+    if (s->n_layers < 2 || s->n_layers > 512) return DEL_EINVAL;
+    if (s->head_dim != 64 && s->head_dim != 128) return DEL_EINVAL;
+    if (s->n_heads < 1 || s->n_kv_heads < 1 || s->n_heads % s->n_kv_heads) return DEL_EINVAL;
+    if (s->d_model < 256 || s->d_model % 32) return DEL_EINVAL;
+    if (s->n_heads * s->head_dim < 256) return DEL_EINVAL;
+    if (s->vocab < 32 || s->vocab % 32) return DEL_EINVAL;
+    if (s->d_ffn < 256 || s->d_ffn % 16) return DEL_EINVAL;
+    if (s->page_size != 16 || s->max_seq < 16 || s->max_seq % 16) return DEL_EINVAL;
+    if (s->max_batch < 1 || s->max_batch > DEL_SEQ_MAX) return DEL_EINVAL;
+    if (s->e_min < 1 || s->e_min > s->e_max || s->e_max >= s->n_layers) return DEL_EINVAL;
+    if (s->g_min < 0 || s->g_min > s->g_max || s->g_max > DEL_MAX_GAMMA) return DEL_EINVAL;
+    if (s->max_batch * (s->g_max + 1) > DEL_ROWS_MAX) return DEL_EINVAL;
+    if (s->init_window < 1 || s->init_window > 32) return DEL_EINVAL;
+    if (!(s->omega >= 0.0 && s->omega <= 1.0)) return DEL_EINVAL;
+    if (s->n_pages < 1) return DEL_EINVAL;
+    return DEL_OK;
+}
+
+int fail(del_ctx *c, cudaError_t e) {
+    c->last = e;
+    snprintf(c->err, sizeof(c->err), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+    return DEL_ECUDA;
+}
+#define CK(call)                                   \
+    do {                                           \
+        cudaError_t e__ = (call);                  \
+        if (e__ != cudaSuccess) return fail(c, e__); \
+    } while (0)
+#define LAUNCH(call)                               \
+    do {                                           \
+        cudaError_t e__ = (call);                  \
+        if (e__ != cudaSuccess) return fail(c, e__); \
+        ++c->launches;                             \
+    } while (0)
+
+bool pdl(const del_ctx *c) { return (c->flags & FLAG_PDL) != 0; }
+
+// ---- plan ring: plans are written into pinned host memory and copied to the device ring in one go
+struct PlanBatch {
+    del_ctx *c;
+    int first, count = 0;
+    explicit PlanBatch(del_ctx *ctx) : c(ctx), first(ctx->plan_cur) {}
+    PassPlan *add(int *index) {
+        *index = first + count;
+        return &c->plan_host[first + count++];
+    }
+};
+
+int plan_begin(del_ctx *c, int need) {
+    if (need > PLAN_RING) return DEL_EINVAL;
+    if (c->plan_cur + need > PLAN_RING) {
+        // wrap: earlier copies out of the pinned ring must have been consumed
+        CK(cudaStreamSynchronize(c->st));
+        c->plan_cur = 0;
+    }
+    return DEL_OK;
+}
+int plan_commit(del_ctx *c, const PlanBatch &b) {
+    if (b.count == 0) return DEL_OK;
+    CK(cudaMemcpyAsync(c->plan_dev + b.first, c->plan_host + b.first, sizeof(PassPlan) * b.count, cudaMemcpyHostToDevice, c->st));
+    c->plan_cur = b.first + b.count;
+    return DEL_OK;
+}
+
+// rows of one pass: for every listed sequence `nrows` consecutive slots starting at slot0
+struct RowSpec { int seq, slot0, nrows; };
+
+void fill_plan(const del_ctx *c, PassPlan *p, const std::vector<RowSpec> &specs, bool prompt_tokens) {
+    memset(p, 0, sizeof(*p));
+    int m = 0, ns = 0;
+    for (const RowSpec &r : specs) {
+        const SeqHost &s = c->seq[r.seq];
+        p->seg[ns++] = Segment{r.seq, m, r.nrows, s.T + r.slot0};
+        for (int i = 0; i < r.nrows; ++i) {
+            const int slot = r.slot0 + i, pos = s.T + slot;
+            p->rows[m++] = RowDesc{r.seq, slot, pos, prompt_tokens ? pos : r.seq * (c->D.S + 1) + slot};
+        }
+    }
+    p->m = m;
+    p->n_seg = ns;
+}
+
+int ensure_pages(del_ctx *c, int sq, int positions) {
+    SeqHost &s = c->seq[sq];
+    const int need = (positions + 15) / 16;
+    if (positions > c->D.max_seq) return DEL_ENOSPC;
+    if ((int)s.pages.size() >= need) return DEL_OK;
+    const int first_new = (int)s.pages.size();
+    if ((int)c->free_pages.size() < need - first_new) return DEL_ENOSPC;
+    while ((int)s.pages.size() < need) {
+        const int pg = c->free_pages.back();
+        c->free_pages.pop_back();
+        c->pt_host[(size_t)sq * c->D.pages_per_seq + s.pages.size()] = pg;
+        s.pages.push_back(pg);
+    }
+    // the source is pageable host memory: the copy is staged before the call returns
+    CK(cudaMemcpyAsync(c->B.PT + (size_t)sq * c->D.pages_per_seq + first_new,
+                       c->pt_host.data() + (size_t)sq * c->D.pages_per_seq + first_new,
+                       sizeof(int32_t) * (need - first_new), cudaMemcpyHostToDevice, c->st));
+    return DEL_OK;
+}
+
+void release_seq(del_ctx *c, int sq) {
+    SeqHost &s = c->seq[sq];
+    for (int pg : s.pages) c->free_pages.push_back(pg);
+    s = SeqHost();
+}
+
+GemmArgs gemm_base(const del_ctx *c, int plan_idx, int layer) {
+    GemmArgs a;
+    memset(&a, 0, sizeof(a));
+    a.D = c->D;
+    a.B = c->B;
+    a.plan = c->plan_dev + plan_idx;
+    a.layer = layer;
+    return a;
+}
+
+CtlArgs ctl_base(const del_ctx *c, int plan_idx) {
+    CtlArgs a;
+    memset(&a, 0, sizeof(a));
+    a.D = c->D;
+    a.B = c->B;
+    a.plan = plan_idx >= 0 ? c->plan_dev + plan_idx : nullptr;
+    a.tok_emb = c->tok_emb;
+    a.gain0 = c->attn_norm[0];
+    a.final_gain = c->final_norm;
+    a.lm_head = c->lm_head;
+    a.tok_src = c->B.TOK;
+    a.e_min = c->sh.e_min; a.e_max = c->sh.e_max; a.g_min = c->sh.g_min; a.g_max = c->sh.g_max;
+    a.omega = c->sh.omega;
+    a.n_vtiles = c->n_vtiles;
+    return a;
+}
+
+struct PassInfo {
+    int plan_idx, m, n_seg, max_rows, max_kv;
+};
+
+PassInfo pass_info(const del_ctx *c, int plan_idx) {
+    const PassPlan &p = c->plan_host[plan_idx];
+    PassInfo pi{plan_idx, p.m, p.n_seg, 0, 0};
+    for (int i = 0; i < p.n_seg; ++i) {
+        pi.max_rows = std::max(pi.max_rows, p.seg[i].nrows);
+        pi.max_kv = std::max(pi.max_kv, p.seg[i].pos0 + p.seg[i].nrows);
+    }
+    return pi;
+}
+
+// one decoder layer over the rows of a pass
+int run_layer(del_ctx *c, const PassInfo &pi, int l, bool write_exit) {
+    const Dims &D = c->D;
+    const bool P = pdl(c);
+    {
+        GemmArgs a = gemm_base(c, pi.plan_idx, l);
+        a.K = D.d;
+        a.n_items = (D.nh + 2 * D.nkv) * (D.hd / 32);
+        a.X = c->B.XS;
+        a.W0 = c->wq[l - 1]; a.W1 = c->wk[l - 1]; a.W2 = c->wv[l - 1];
+        LAUNCH(launch_rowgemm(EPI_QKV, a, pi.m, c->n_sms, c->st, P));
+    }
+    {
+        AttnArgs a;
+        memset(&a, 0, sizeof(a));
+        a.D = D; a.B = c->B; a.plan = c->plan_dev + pi.plan_idx; a.layer = l;
+        const int pages = (pi.max_kv + 15) / 16;
+        int ns = (2 * c->n_sms + pi.n_seg * D.nkv - 1) / (pi.n_seg * D.nkv);
+        ns = std::max(1, std::min(std::min(ns, 16), (pages + 1) / 2));
+        a.n_splits = ns;
+        a.max_rows = pi.max_rows;
+        LAUNCH(launch_attention(a, pi.n_seg, c->st, P));
+    }
+    {
+        GemmArgs a = gemm_base(c, pi.plan_idx, l);
+        a.K = D.nh * D.hd;
+        a.n_items = D.d / 16;
+        a.X = c->B.ATT;
+        a.W0 = c->wo[l - 1];
+        a.gain_a = c->ffn_norm[l - 1];
+        LAUNCH(launch_rowgemm(EPI_OPROJ, a, pi.m, c->n_sms, c->st, P));
+    }
+    {
+        GemmArgs a = gemm_base(c, pi.plan_idx, l);
+        a.K = D.d;
+        a.n_items = D.F / 16;
+        a.X = c->B.XM;
+        a.W0 = c->w_gate[l - 1]; a.W1 = c->w_up[l - 1];
+        LAUNCH(launch_rowgemm(EPI_GATEUP, a, pi.m, c->n_sms, c->st, P));
+    }
+    {
+        GemmArgs a = gemm_base(c, pi.plan_idx, l);
+        a.K = D.F;
+        a.n_items = D.d / 16;
+        a.X = c->B.ACT;
+        a.W0 = c->w_down[l - 1];
+        a.gain_a = l < D.L ? c->attn_norm[l] : nullptr;
+        a.gain_b = write_exit ? c->final_norm : nullptr;
+        LAUNCH(launch_rowgemm(EPI_DOWN, a, pi.m, c->n_sms, c->st, P));
+    }
+    return DEL_OK;
+}
+
+// sequences of a call with their round parameters
+struct Job { int seq, E, g; };
+
+// ---- draft (a1-a3): g tokens per sequence, layers 1..E, exit head, arg-max, next embedding
+int plans_needed_draft(const std::vector<Job> &jobs) {
+    int gmax = 0;
+    for (const Job &j : jobs) gmax = std::max(gmax, j.g);
+    return gmax * ((int)jobs.size() + 1);
+}
+
+int enqueue_draft(del_ctx *c, const std::vector<Job> &jobs) {
+    int gmax = 0;
+    for (const Job &j : jobs) gmax = std::max(gmax, j.g);
+    if (gmax == 0) return DEL_OK;
+    int rc = plan_begin(c, plans_needed_draft(jobs));
+    if (rc) return rc;
+    PlanBatch pb(c);
+    // distinct exit layers, ascending: the rows of a pass thin out as sequences reach their exit
+    std::vector<int> Es;
+    for (const Job &j : jobs) Es.push_back(j.E);
+    std::sort(Es.begin(), Es.end());
+    Es.erase(std::unique(Es.begin(), Es.end()), Es.end());
+    struct Step { int full_idx; std::vector<int> sub_idx; };
+    std::vector<Step> steps(gmax);
+    for (int i = 0; i < gmax; ++i) {
+        std::vector<RowSpec> full;
+        for (const Job &j : jobs)
+            if (i < j.g) full.push_back(RowSpec{j.seq, i, 1});
+        fill_plan(c, pb.add(&steps[i].full_idx), full, false);
+        for (size_t e = 0; e < Es.size(); ++e) {
+            if (e == 0) { steps[i].sub_idx.push_back(steps[i].full_idx); continue; }
+            std::vector<RowSpec> sub;
+            for (const Job &j : jobs)
+                if (i < j.g && j.E >= Es[e]) sub.push_back(RowSpec{j.seq, i, 1});
+            int idx = -1;
+            if (!sub.empty()) fill_plan(c, pb.add(&idx), sub, false);
+            steps[i].sub_idx.push_back(idx);
+        }
+    }
+    rc = plan_commit(c, pb);
+    if (rc) return rc;
+    const bool P = pdl(c);
+    for (int i = 0; i < gmax; ++i) {
+        const PassInfo full = pass_info(c, steps[i].full_idx);
+        if (i == 0) {
+            CtlArgs ca = ctl_base(c, full.plan_idx);
+            LAUNCH(launch_embed(ca, full.m, c->st, P));
+        }
+        int l = 1;
+        for (size_t e = 0; e < Es.size(); ++e) {
+            if (steps[i].sub_idx[e] < 0) break;
+            const PassInfo pi = pass_info(c, steps[i].sub_idx[e]);
+            for (; l <= Es[e]; ++l) {
+                rc = run_layer(c, pi, l, l == Es[e]);
+                if (rc) return rc;
+            }
+        }
+        // exit head of every drafting sequence in one pass over W_lm, then arg-max and next embedding
+        GemmArgs a = gemm_base(c, full.plan_idx, 0);
+        a.K = c->D.d;
+        a.n_items = c->D.V / 16;
+        a.X = c->B.XE;
+        a.W0 = c->lm_head;
+        LAUNCH(launch_rowgemm(EPI_LMHEAD, a, full.m, c->n_sms, c->st, P));
+        CtlArgs ca = ctl_base(c, full.plan_idx);
+        ca.n_part = rowgemm_lmhead_grid(a.n_items, full.m, c->n_sms);
+        LAUNCH(launch_draft_finalize_embed(ca, full.m, true, c->st, P));
+    }
+    return DEL_OK;
+}
+
+// ---- verify (a4-a5)
+int enqueue_verify(del_ctx *c, const std::vector<Job> &jobs) {
+    int rc = plan_begin(c, (int)jobs.size() + 2);
+    if (rc) return rc;
+    PlanBatch pb(c);
+    std::vector<int> Es;
+    for (const Job &j : jobs) Es.push_back(j.E);
+    std::sort(Es.begin(), Es.end());
+    Es.erase(std::unique(Es.begin(), Es.end()), Es.end());
+    // segment k covers layers (Es[k-1], Es[k]] ; the last one (Es.back(), L]
+    std::vector<int> idx(Es.size() + 1);
+    std::vector<int> embed_rows;
+    for (size_t k = 0; k <= Es.size(); ++k) {
+        const int l_first = k == 0 ? 1 : Es[k - 1] + 1;
+        std::vector<RowSpec> specs;
+        for (const Job &j : jobs) {
+            if (l_first <= j.E) specs.push_back(RowSpec{j.seq, j.g, 1});
+            else specs.push_back(RowSpec{j.seq, 0, j.g + 1});
+        }
+        fill_plan(c, pb.add(&idx[k]), specs, false);
+    }
+    // sequences that drafted nothing still need their input token embedded
+    int embed_idx = -1;
+    {
+        std::vector<RowSpec> specs;
+        for (const Job &j : jobs)
+            if (j.g == 0) specs.push_back(RowSpec{j.seq, 0, 1});
+        if (!specs.empty()) fill_plan(c, pb.add(&embed_idx), specs, false);
+    }
+    rc = plan_commit(c, pb);
+    if (rc) return rc;
+    if (embed_idx >= 0) {
+        CtlArgs ca = ctl_base(c, embed_idx);
+        LAUNCH(launch_embed(ca, c->plan_host[embed_idx].m, c->st, pdl(c)));
+    }
+    int l = 1;
+    for (size_t k = 0; k <= Es.size(); ++k) {
+        const int l_last = k < Es.size() ? Es[k] : c->D.L;
+        const PassInfo pi = pass_info(c, idx[k]);
+        for (; l <= l_last; ++l) {
+            rc = run_layer(c, pi, l, false);
+            if (rc) return rc;
+        }
+    }
+    return DEL_OK;
+}
+
+// ---- stacked LM head + arg-max over all layers' hidden rows (a6), then accept / counts (a7-a8)
+int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bool do_select) {
+    UpdatePlan *up = &c->up_host[0];
+    memset(up, 0, sizeof(*up));
+    int rows = 0;
+    for (const Job &j : jobs) {
+        auto &e = up->s[up->n_seq++];
+        e.seq = j.seq; e.row0 = rows; e.g = j.g; e.E = j.E; e.n_valid_init = W;
+        rows += c->D.L * (mode ? W : j.g + 1);
+    }
+    up->n_rows = rows;
+    if (rows > c->R_max) return DEL_EINVAL;
+    CK(cudaMemcpyAsync(c->up_dev, up, sizeof(UpdatePlan), cudaMemcpyHostToDevice, c->st));
+    const bool P = pdl(c);
+    CtlArgs ca = ctl_base(c, -1);
+    ca.mode = mode;
+    ca.n_rows = rows;
+    LAUNCH(launch_prep_rows(ca, c->up_dev, rows, c->st, P));
+    // streaming LM head in chunks of 64 stacked rows
+    const int n_chunks = (rows + DEL_ROWS_MAX - 1) / DEL_ROWS_MAX;
+    int rc = plan_begin(c, n_chunks);
+    if (rc) return rc;
+    PlanBatch pb(c);
+    std::vector<int> pidx(n_chunks);
+    for (int k = 0; k < n_chunks; ++k) {
+        PassPlan *p = pb.add(&pidx[k]);
+        memset(p, 0, sizeof(*p));
+        p->m = std::min(DEL_ROWS_MAX, rows - k * DEL_ROWS_MAX);
+    }
+    rc = plan_commit(c, pb);
+    if (rc) return rc;
+    for (int k = 0; k < n_chunks; ++k) {
+        const int m = c->plan_host[pidx[k]].m;
+        GemmArgs a = gemm_base(c, pidx[k], 0);
+        a.K = c->D.d;
+        a.n_items = c->D.V / 16;
+        a.X = c->B.XN + (size_t)k * DEL_ROWS_MAX * c->D.d;
+        a.W0 = c->lm_head;
+        a.x_by_row = 1;
+        LAUNCH(launch_rowgemm(EPI_LMHEAD, a, m, c->n_sms, c->st, P));
+        const int n_part = rowgemm_lmhead_grid(a.n_items, m, c->n_sms);
+        LAUNCH(launch_shadow_reduce(ca, c->up_dev, c->B.LPV, c->B.LPI, n_part, DEL_ROWS_MAX, 1, k * DEL_ROWS_MAX, m, c->st, P));
+    }
+    LAUNCH(launch_update(ca, c->up_dev, c->out_dev, up->n_seq, c->st, P));
+    if (do_select) LAUNCH(launch_select(ca, c->up_dev, c->out_dev, up->n_seq, c->st, P));
+    return DEL_OK;
+}
+
+int read_out(del_ctx *c) {
+    CK(cudaMemcpyAsync(c->out_host, c->out_dev, sizeof(del_round_out) * c->D.B, cudaMemcpyDeviceToHost, c->st));
+    CK(cudaStreamSynchronize(c->st));
+    return DEL_OK;
+}
+
+int clip_gamma(const SeqHost &s, int gamma) { return std::max(0, std::min(gamma, s.remaining - 1)); }
+
+bool seq_ok(const del_ctx *c, int sq) { return c && sq >= 0 && sq < c->D.B; }
+
+}  // namespace
+
+// =====================================================================================  C ABI
+extern "C" {
+
+size_t del_workspace_bytes(const del_shape *shape) {
+    if (validate(shape) != DEL_OK) return 0;
+    Dims D; Buffers B; int R, nv; PassPlan *p; UpdatePlan *u; del_round_out *o; float *dbg;
+    return carve_all(*shape, nullptr, D, B, R, nv, &p, &u, &o, &dbg);
+}
+
+int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const del_kv *kv, void *workspace,
+             size_t ws_bytes, void *cuda_stream) {
+    if (!out || !w || !kv || !workspace) return DEL_EINVAL;
+    int rc = validate(shape);
+    if (rc) return rc;
+    if (!w->tok_emb || !w->final_norm || !w->lm_head || !w->attn_norm || !w->wq || !w->wk || !w->wv || !w->wo ||
+        !w->ffn_norm || !w->w_gate || !w->w_up || !w->w_down || !w->rope_cos || !w->rope_sin)
+        return DEL_EINVAL;
+    if (!kv->k_pages || !kv->v_pages || !kv->page_table) return DEL_EINVAL;
+    if (ws_bytes < del_workspace_bytes(shape)) return DEL_ENOSPC;
+    del_ctx *c = new (std::nothrow) del_ctx();
+    if (!c) return DEL_ENOSPC;
+    c->sh = *shape;
+    carve_all(*shape, workspace, c->D, c->B, c->R_max, c->n_vtiles, &c->plan_dev, &c->up_dev, &c->out_dev, &c->dbg_dev);
+    c->B.KP = (bf16 *)kv->k_pages; c->B.VP = (bf16 *)kv->v_pages; c->B.PT = kv->page_table;
+    c->B.rope_cos = w->rope_cos; c->B.rope_sin = w->rope_sin;
+    c->tok_emb = (const bf16 *)w->tok_emb; c->final_norm = (const bf16 *)w->final_norm; c->lm_head = (const bf16 *)w->lm_head;
+    const int L = shape->n_layers;
+    auto grab = [&](std::vector<const bf16 *> &dst, const void *const *src) {
+        dst.resize(L);
+        for (int l = 0; l < L; ++l) {
+            dst[l] = (const bf16 *)src[l];
+            if (!dst[l]) return false;
+        }
+        return true;
+    };
+    if (!grab(c->attn_norm, w->attn_norm) || !grab(c->wq, w->wq) || !grab(c->wk, w->wk) || !grab(c->wv, w->wv) ||
+        !grab(c->wo, w->wo) || !grab(c->ffn_norm, w->ffn_norm) || !grab(c->w_gate, w->w_gate) || !grab(c->w_up, w->w_up) ||
+        !grab(c->w_down, w->w_down)) {
+        delete c;
+        return DEL_EINVAL;
+    }
+    c->st = (cudaStream_t)cuda_stream;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->plan_host, sizeof(PassPlan) * PLAN_RING, cudaHostAllocDefault);
+    if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->up_host, sizeof(UpdatePlan) * 2, cudaHostAllocDefault);
+    if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->out_host, sizeof(del_round_out) * DEL_SEQ_MAX, cudaHostAllocDefault);
+    if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->stage_host, 1 << 16, cudaHostAllocDefault);
+    // zero the workspace (counters, statistics) and the KV pages (stale bit patterns must stay finite)
+    if (e == cudaSuccess) e = cudaMemsetAsync(workspace, 0, del_workspace_bytes(shape), c->st);
+    const size_t kv_bytes = (size_t)shape->n_pages * L * shape->n_kv_heads * 16 * shape->head_dim * sizeof(bf16);
+    if (e == cudaSuccess) e = cudaMemsetAsync(kv->k_pages, 0, kv_bytes, c->st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(kv->v_pages, 0, kv_bytes, c->st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->st);
+    if (e != cudaSuccess) {
+        del_destroy(c);
+        return DEL_ECUDA;
+    }
+    c->pt_host.assign((size_t)c->D.B * c->D.pages_per_seq, 0);
+    for (int p = shape->n_pages - 1; p >= 0; --p) c->free_pages.push_back(p);
+    *out = c;
+    return DEL_OK;
+}
+
+void del_destroy(del_ctx *c) {
+    if (!c) return;
+    if (c->plan_host) cudaFreeHost(c->plan_host);
+    if (c->up_host) cudaFreeHost(c->up_host);
+    if (c->out_host) cudaFreeHost(c->out_host);
+    if (c->stage_host) cudaFreeHost(c->stage_host);
+    delete c;
+}
+
+int del_release(del_ctx *c, int sq) {
+    if (!seq_ok(c, sq)) return DEL_EINVAL;
+    release_seq(c, sq);
+    return DEL_OK;
+}
+
+int del_prefill(del_ctx *c, int sq, const int32_t *prompt, int n_prompt, int max_new_tokens, del_round_out *first_out) {
+    if (!seq_ok(c, sq) || !prompt || n_prompt < 1 || max_new_tokens < 1) return DEL_EINVAL;
+    for (int i = 0; i < n_prompt; ++i)
+        if (prompt[i] < 0 || prompt[i] >= c->D.V) return DEL_EINVAL;
+    if (n_prompt + max_new_tokens + c->sh.g_max + 1 > c->D.max_seq) return DEL_ENOSPC;
+    release_seq(c, sq);
+    SeqHost &s = c->seq[sq];
+    int rc = ensure_pages(c, sq, n_prompt + 1);
+    if (rc) { release_seq(c, sq); return rc; }
+    CK(cudaMemcpyAsync(c->B.PROMPT_ALL, prompt, sizeof(int32_t) * n_prompt, cudaMemcpyHostToDevice, c->st));
+    SeqState st0;
+    memset(&st0, 0, sizeof(st0));
+    memcpy(c->stage_host, &st0, sizeof(st0));
+    CK(cudaMemcpyAsync(c->B.ST + sq, c->stage_host, sizeof(SeqState), cudaMemcpyHostToDevice, c->st));
+    const int S = c->D.S, W = std::min(c->sh.init_window, n_prompt);
+    // chunks of <= S positions; the last chunk is exactly the window so that its hidden states stay
+    // in slots 0..W-1 of the stack
+    std::vector<std::pair<int, int>> chunks;
+    for (int p0 = 0; p0 < n_prompt - W; p0 += S) chunks.push_back({p0, std::min(S, n_prompt - W - p0)});
+    chunks.push_back({n_prompt - W, W});
+    s.T = 0;
+    for (auto ch : chunks) {
+        rc = plan_begin(c, 1);
+        if (rc) return rc;
+        PlanBatch pb(c);
+        int idx;
+        s.T = ch.first;                      // rows are addressed relative to the committed length
+        fill_plan(c, pb.add(&idx), {RowSpec{sq, 0, ch.second}}, true);
+        rc = plan_commit(c, pb);
+        if (rc) return rc;
+        CtlArgs ca = ctl_base(c, idx);
+        ca.tok_src = c->B.PROMPT_ALL;
+        LAUNCH(launch_embed(ca, ch.second, c->st, pdl(c)));
+        const PassInfo pi = pass_info(c, idx);
+        for (int l = 1; l <= c->D.L; ++l) {
+            rc = run_layer(c, pi, l, false);
+            if (rc) return rc;
+        }
+    }
+    s.T = n_prompt;
+    s.active = true;
+    s.remaining = max_new_tokens;
+    s.phase = 0;
+    rc = enqueue_update(c, {Job{sq, 0, 0}}, 1, W, true);
+    if (rc) return rc;
+    rc = read_out(c);
+    if (rc) return rc;
+    const del_round_out &o = c->out_host[sq];
+    s.remaining -= 1;
+    s.E = o.next_E;
+    s.gamma = o.next_gamma;
+    if (first_out) {
+        memset(first_out, 0, sizeof(*first_out));
+        first_out->n_emitted = 1;
+        first_out->tokens[0] = o.tokens[0];
+        first_out->next_E = o.next_E;
+        first_out->next_gamma = o.next_gamma;
+    }
+    return DEL_OK;
+}
+
+int del_draft(del_ctx *c, int sq, int E, int gamma) {
+    if (!seq_ok(c, sq)) return DEL_EINVAL;
+    SeqHost &s = c->seq[sq];
+    if (E < 1 || E >= c->D.L || gamma < 0 || gamma > c->sh.g_max) return DEL_EINVAL;
+    if (!s.active || s.remaining < 1 || s.phase != 0) return DEL_ESTATE;
+    const int g = clip_gamma(s, gamma);
+    int rc = ensure_pages(c, sq, s.T + g + 1);
+    if (rc) return rc;
+    rc = enqueue_draft(c, {Job{sq, E, g}});
+    if (rc) return rc;
+    s.cur_E = E; s.cur_g = g; s.cur_gamma = gamma; s.phase = 1;
+    return DEL_OK;
+}
+
+int del_verify(del_ctx *c, int sq) {
+    if (!seq_ok(c, sq)) return DEL_EINVAL;
+    SeqHost &s = c->seq[sq];
+    if (!s.active || s.phase != 1) return DEL_ESTATE;
+    int rc = enqueue_verify(c, {Job{sq, s.cur_E, s.cur_g}});
+    if (rc) return rc;
+    s.phase = 2;
+    return DEL_OK;
+}
+
+static void finish_round(del_ctx *c, int sq, del_round_out *dst, bool with_next) {
+    SeqHost &s = c->seq[sq];
+    const del_round_out &o = c->out_host[sq];
+    s.T += o.n_emitted;
+    s.remaining -= o.n_emitted;
+    s.phase = 0;
+    if (with_next) { s.E = o.next_E; s.gamma = o.next_gamma; }
+    if (dst) {
+        *dst = o;
+        dst->E = s.cur_E; dst->gamma = s.cur_gamma; dst->g = s.cur_g;
+        dst->status = 0;
+        if (!with_next) { dst->next_E = 0; dst->next_gamma = 0; }
+    }
+}
+
+int del_layer_accept(del_ctx *c, int sq, del_round_out *out) {
+    if (!seq_ok(c, sq)) return DEL_EINVAL;
+    SeqHost &s = c->seq[sq];
+    if (!s.active || s.phase != 2) return DEL_ESTATE;
+    int rc = enqueue_update(c, {Job{sq, s.cur_E, s.cur_g}}, 0, 0, false);
+    if (rc) return rc;
+    rc = read_out(c);
+    if (rc) return rc;
+    finish_round(c, sq, out, false);
+    return DEL_OK;
+}
+
+int del_select(del_ctx *c, int sq, int32_t *E, int32_t *gamma) {
+    if (!seq_ok(c, sq)) return DEL_EINVAL;
+    SeqHost &s = c->seq[sq];
+    if (!s.active) return DEL_ESTATE;
+    UpdatePlan *up = &c->up_host[1];
+    memset(up, 0, sizeof(*up));
+    up->n_seq = 1;
+    up->s[0].seq = sq;
+    CK(cudaMemcpyAsync(c->up_dev + 1, up, sizeof(UpdatePlan), cudaMemcpyHostToDevice, c->st));
+    CtlArgs ca = ctl_base(c, -1);
+    LAUNCH(launch_select(ca, c->up_dev + 1, c->out_dev, 1, c->st, pdl(c)));
+    int rc = read_out(c);
+    if (rc) return rc;
+    s.E = c->out_host[sq].next_E;
+    s.gamma = c->out_host[sq].next_gamma;
+    if (E) *E = s.E;
+    if (gamma) *gamma = s.gamma;
+    return DEL_OK;
+}
+
+int del_round(del_ctx *c, del_round_out *out) {
+    if (!c || !out) return DEL_EINVAL;
+    std::vector<Job> jobs;
+    for (int sq = 0; sq < c->D.B; ++sq) {
+        SeqHost &s = c->seq[sq];
+        memset(&out[sq], 0, sizeof(out[sq]));
+        if (!s.active || s.remaining < 1) continue;
+        if (s.phase != 0) return DEL_ESTATE;
+        const int E = s.fixed_E > 0 ? s.fixed_E : s.E;
+        const int gamma = s.fixed_E > 0 ? s.fixed_gamma : s.gamma;
+        const int g = clip_gamma(s, gamma);
+        int rc = ensure_pages(c, sq, s.T + g + 1);
+        if (rc) return rc;
+        s.cur_E = E; s.cur_g = g; s.cur_gamma = gamma;
+        jobs.push_back(Job{sq, E, g});
+    }
+    if (jobs.empty()) return DEL_ESTATE;
+    int rc = enqueue_draft(c, jobs);
+    if (rc) return rc;
+    rc = enqueue_verify(c, jobs);
+    if (rc) return rc;
+    rc = enqueue_update(c, jobs, 0, 0, true);
+    if (rc) return rc;
+    rc = read_out(c);
+    if (rc) return rc;
+    for (const Job &j : jobs) finish_round(c, j.seq, &out[j.seq], true);
+    return DEL_OK;
+}
+
+int del_set_policy(del_ctx *c, int sq, int E, int gamma) {
+    if (!seq_ok(c, sq)) return DEL_EINVAL;
+    if (E > 0 && (E >= c->D.L || gamma < 0 || gamma > c->sh.g_max)) return DEL_EINVAL;
+    SeqHost &s = c->seq[sq];
+    s.fixed_E = E > 0 ? E : 0;
+    s.fixed_gamma = E > 0 ? gamma : 0;
+    CK(cudaStreamSynchronize(c->st));
+    SeqState st;
+    CK(cudaMemcpy(&st, c->B.ST + sq, sizeof(st), cudaMemcpyDeviceToHost));
+    st.fixed_E = s.fixed_E;
+    st.fixed_gamma = s.fixed_gamma;
+    CK(cudaMemcpy(c->B.ST + sq, &st, sizeof(st), cudaMemcpyHostToDevice));
+    return DEL_OK;
+}
+
+int del_get_stats(del_ctx *c, int sq, double *Sc, double *Sn, int32_t *E, int32_t *gamma) {
+    if (!seq_ok(c, sq)) return DEL_EINVAL;
+    CK(cudaStreamSynchronize(c->st));
+    if (Sc) CK(cudaMemcpy(Sc, c->B.SC + (size_t)sq * c->D.L, sizeof(double) * c->D.L, cudaMemcpyDeviceToHost));
+    SeqState st;
+    CK(cudaMemcpy(&st, c->B.ST + sq, sizeof(st), cudaMemcpyDeviceToHost));
+    if (Sn) *Sn = st.Sn;
+    if (E) *E = c->seq[sq].E;
+    if (gamma) *gamma = c->seq[sq].gamma;
+    return DEL_OK;
+}
+
+int del_set_stats(del_ctx *c, int sq, const double *Sc, double Sn, int32_t E, int32_t gamma) {
+    if (!seq_ok(c, sq) || !Sc) return DEL_EINVAL;
+    CK(cudaStreamSynchronize(c->st));
+    CK(cudaMemcpy(c->B.SC + (size_t)sq * c->D.L, Sc, sizeof(double) * c->D.L, cudaMemcpyHostToDevice));
+    SeqState st;
+    CK(cudaMemcpy(&st, c->B.ST + sq, sizeof(st), cudaMemcpyDeviceToHost));
+    st.Sn = Sn; st.E = E; st.gamma = gamma;
+    CK(cudaMemcpy(c->B.ST + sq, &st, sizeof(st), cudaMemcpyHostToDevice));
+    c->seq[sq].E = E;
+    c->seq[sq].gamma = gamma;
+    return DEL_OK;
+}
+
+int del_get_shadow(del_ctx *c, int sq, int32_t *shadow, int32_t *counts) {
+    if (!seq_ok(c, sq)) return DEL_EINVAL;
+    CK(cudaStreamSynchronize(c->st));
+    const int L = c->D.L, S = c->D.S, G = c->sh.g_max + 1;
+    if (shadow) {
+        std::vector<int32_t> tmp((size_t)L * S);
+        CK(cudaMemcpy(tmp.data(), c->B.SHADOW + (size_t)sq * L * S, sizeof(int32_t) * L * S, cudaMemcpyDeviceToHost));
+        for (int l = 0; l < L; ++l)
+            for (int i = 0; i < G; ++i) shadow[l * G + i] = tmp[(size_t)l * S + i];
+    }
+    if (counts) CK(cudaMemcpy(counts, c->B.COUNTS + (size_t)sq * L, sizeof(int32_t) * L, cudaMemcpyDeviceToHost));
+    return DEL_OK;
+}
+
+int del_get_drafts(del_ctx *c, int sq, int32_t *drafts) {
+    if (!seq_ok(c, sq) || !drafts) return DEL_EINVAL;
+    CK(cudaStreamSynchronize(c->st));
+    if (c->sh.g_max > 0)
+        CK(cudaMemcpy(drafts, c->B.TOK + (size_t)sq * (c->D.S + 1) + 1, sizeof(int32_t) * c->sh.g_max, cudaMemcpyDeviceToHost));
+    return DEL_OK;
+}
+
+int del_force_token(del_ctx *c, int sq, int32_t token) {
+    if (!seq_ok(c, sq) || token < 0 || token >= c->D.V) return DEL_EINVAL;
+    CK(cudaStreamSynchronize(c->st));
+    CK(cudaMemcpy(c->B.TOK + (size_t)sq * (c->D.S + 1), &token, sizeof(int32_t), cudaMemcpyHostToDevice));
+    return DEL_OK;
+}
+
+int del_get_hidden(del_ctx *c, int sq, int layer, int row, float *out) {
+    if (!seq_ok(c, sq) || !out || layer < 0 || layer > c->D.L || row < 0 || row >= c->D.S) return DEL_EINVAL;
+    CK(cudaStreamSynchronize(c->st));
+    const size_t sr = ((size_t)layer * c->D.B + sq) * c->D.S + row;
+    CK(cudaMemcpy(out, c->B.H + sr * c->D.d, sizeof(float) * c->D.d, cudaMemcpyDeviceToHost));
+    return DEL_OK;
+}
+
+int del_debug_logits(del_ctx *c, int sq, int layer, int row, float *out) {
+    if (!seq_ok(c, sq) || !out || layer < 0 || layer > c->D.L || row < 0 || row >= c->D.S) return DEL_EINVAL;
+    CtlArgs ca = ctl_base(c, -1);
+    LAUNCH(launch_debug_logits(ca, layer, sq, row, c->dbg_dev, c->st));
+    CK(cudaStreamSynchronize(c->st));
+    CK(cudaMemcpy(out, c->dbg_dev, sizeof(float) * c->D.V, cudaMemcpyDeviceToHost));
+    return DEL_OK;
+}
+
+int del_get_kv(del_ctx *c, int sq, int layer, int pos, float *k_out, float *v_out) {
+    if (!seq_ok(c, sq) || layer < 1 || layer > c->D.L || pos < 0) return DEL_EINVAL;
+    if (pos >= (int)c->seq[sq].pages.size() * 16) return DEL_EINVAL;
+    const int n = c->D.nkv * c->D.hd;
+    CtlArgs ca = ctl_base(c, -1);
+    LAUNCH(launch_gather_kv(ca, layer, sq, pos, c->dbg_dev, c->dbg_dev + n, c->st));
+    CK(cudaStreamSynchronize(c->st));
+    if (k_out) CK(cudaMemcpy(k_out, c->dbg_dev, sizeof(float) * n, cudaMemcpyDeviceToHost));
+    if (v_out) CK(cudaMemcpy(v_out, c->dbg_dev + n, sizeof(float) * n, cudaMemcpyDeviceToHost));
+    return DEL_OK;
+}
+
+int del_committed_len(del_ctx *c, int sq) {
+    if (!seq_ok(c, sq)) return DEL_EINVAL;
+    return c->seq[sq].active ? c->seq[sq].T : DEL_ESTATE;
+}
+
+int64_t del_launch_count(const del_ctx *c) { return c ? c->launches : 0; }
+
+int del_set_flags(del_ctx *c, int flags) {
+    if (!c) return DEL_EINVAL;
+    const int old = c->flags;
+    c->flags = flags;
+    return old;
+}
+
+const char *del_strerror(int code) {
+    switch (code) {
+        case DEL_OK: return "ok";
+        case DEL_EINVAL: return "invalid argument or shape";
+        case DEL_ENOSPC: return "out of KV pages, sequence length or workspace";
+        case DEL_ESTATE: return "call order wrong for the sequence's state";
+        case DEL_ETIMEOUT: return "a bounded device-side wait expired";
+        case DEL_ECUDA: return "CUDA error (see del_last_cuda_error)";
+    }
+    return "unknown error";
+}
+
+const char *del_last_cuda_error(const del_ctx *c) { return c ? c->err : ""; }
+
+}  // extern "C"

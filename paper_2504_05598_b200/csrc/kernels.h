@@ -1,0 +1,81 @@
+// Internal launch interface between the host-side round scheduler (del_api.cu) and the kernels.
+#pragma once
+
+#include "common.cuh"
+
+enum { EPI_QKV = 0, EPI_OPROJ = 1, EPI_GATEUP = 2, EPI_DOWN = 3, EPI_LMHEAD = 4 };
+
+struct GemmArgs {
+    Dims D;
+    Buffers B;
+    const PassPlan *plan;      // device
+    int32_t layer;             // 1-based layer the op belongs to (LMHEAD: the exit layer)
+    int32_t K;                 // in-features
+    int32_t n_items;           // work items: tile pairs (QKV, GATEUP) or 16-row tiles
+    const bf16 *X;             // activations (see rowgemm.cu for the indexing per epilogue)
+    const bf16 *W0, *W1, *W2;
+    const bf16 *gain_a, *gain_b;
+    int32_t x_by_row;          // LMHEAD: activations are X[c] (stacked rows) instead of XE[seq][slot]
+};
+
+cudaError_t launch_rowgemm(int epi, const GemmArgs &a, int m, int n_sms, cudaStream_t st, bool pdl);
+int rowgemm_lmhead_grid(int n_items, int m, int n_sms);
+
+struct AttnArgs {
+    Dims D;
+    Buffers B;
+    const PassPlan *plan;
+    int32_t layer;
+    int32_t n_splits;          // key-range splits per (segment, kv head)
+    int32_t max_rows;          // largest segment (rows), decides the number of query tiles
+};
+cudaError_t launch_attention(const AttnArgs &a, int n_seg, cudaStream_t st, bool pdl);
+
+// control kernels
+struct CtlArgs {
+    Dims D;
+    Buffers B;
+    const PassPlan *plan;
+    const bf16 *tok_emb, *gain0, *final_gain, *lm_head;
+    const int32_t *tok_src;    // token buffer the embedding reads (B.TOK or B.PROMPT)
+    int32_t n_part;            // LM-head partials to reduce
+    int32_t draft_index;       // which draft the finalised token is
+    int32_t e_min, e_max, g_min, g_max;
+    int32_t mode;              // accept: 0 = round, 1 = prefill initialisation
+    int32_t do_select;
+    int32_t n_rows;            // rows of the stacked LM-head problem
+    int32_t n_vtiles;
+    double omega;
+};
+
+// rows of the stacked LM head: (seq, layer, slot) per row, plus per-sequence bookkeeping of the update
+struct UpdatePlan {
+    int32_t n_seq, n_rows, pad0, pad1;
+    struct {
+        int32_t seq, row0, g, E;     // rows row0 + (l-1)*(g+1) + i ; E = draft layer of the round
+        int32_t n_valid_init;        // prefill: window width W (rows per layer = W)
+        int32_t pad[3];
+    } s[DEL_SEQ_MAX];
+};
+
+cudaError_t launch_embed(const CtlArgs &a, int m, cudaStream_t st, bool pdl);
+cudaError_t launch_draft_finalize_embed(const CtlArgs &a, int m, bool embed_next, cudaStream_t st, bool pdl);
+cudaError_t launch_prep_rows(const CtlArgs &a, const UpdatePlan *up, int n_rows, cudaStream_t st, bool pdl);
+cudaError_t launch_shadow_reduce(const CtlArgs &a, const UpdatePlan *up, const float *pv, const int32_t *pi, int n_part,
+                                 int pstride, int cstride, int row_base, int n_rows, cudaStream_t st, bool pdl);
+cudaError_t launch_update(const CtlArgs &a, const UpdatePlan *up, void *out_dev, int n_seq, cudaStream_t st, bool pdl);
+cudaError_t launch_select(const CtlArgs &a, const UpdatePlan *up, void *out_dev, int n_seq, cudaStream_t st, bool pdl);
+cudaError_t launch_debug_logits(const CtlArgs &a, int layer, int seq, int slot, float *out_dev, cudaStream_t st);
+cudaError_t launch_gather_kv(const CtlArgs &a, int layer, int seq, int pos, float *k_out, float *v_out, cudaStream_t st);
+
+// streaming LM head over stacked rows (chunks of <= 64 rows through the rowgemm kernel is the
+// host's job); tensor-core version:
+struct LmTcArgs {
+    const void *tmap_x, *tmap_w;   // CUtensorMap in device-visible param space (passed by value below)
+    float *part_v;
+    int32_t *part_i;
+    int32_t n_rows, V, d, n_vtiles;
+    int32_t *err;
+};
+cudaError_t launch_lmhead_tc(const void *tmap_x_host, const void *tmap_w_host, float *part_v, int32_t *part_i,
+                             int n_rows, int V, int d, int32_t *err, int n_sms, cudaStream_t st, bool pdl);

@@ -1,0 +1,356 @@
+// Weight-streaming skinny GEMM  Y[m, N] = X[m, K] * W[N, K]^T  for m <= 64 activation rows, with the
+// layer's element-wise work fused into its epilogues.  It is bound by HBM: every weight byte is read
+// exactly once per pass, straight from global memory into tensor-core fragments.
+//
+// Mapping.  A tile is 16 consecutive weight rows (output features) over the whole K.  The 8 warps of a
+// CTA split K in 32-element steps (warp w takes steps w, w+8, ...), so at any time the CTA reads 512
+// contiguous bytes of each of the 16 rows.  Per step a thread issues one 16-byte load for row g and one
+// for row g+8 (g = lane/4) at column offset 8*(lane%4): the eight bf16 values feed two m16n8k16 MMAs.
+// The tensor core sums over k, so any permutation of k applied to both operands gives the same
+// product; the activation fragment is therefore loaded with the same 16-byte pattern from the row's
+// bf16 vector, and no shared-memory staging or ldmatrix is needed.  Loads are software-pipelined in two
+// register batches that run ahead across tile boundaries, and the weight loads of the first batches
+// are issued before the kernel waits for its producer (programmatic dependent launch).
+// Partial sums of the 8 warps are added in a fixed order through shared memory: results do not depend
+// on the grid size or on how many rows share the pass.
+//
+// Epilogues (one per use in the decoder layer):
+//   QKV    scale by the row's 1/rms, rotary embedding on q and k, q -> Q buffer, k and v -> paged cache
+//   OPROJ  + residual -> HM, XM = bf16(HM * ffn gain), partial sums of squares
+//   GATEUP scale by 1/rms, silu(gate) * up -> ACT
+//   DOWN   + residual -> hidden stack, XS/XE = bf16(h * next gain), partial sums of squares
+//   LMHEAD running arg-max over the vocabulary tiles of this CTA (1/rms > 0 cannot change it)
+// RMSNorm is split: the producer stores bf16(h * gain) and per-tile sums of h^2, the consumer scales
+// its accumulators by rsqrt(mean(h^2) + eps) (the scale is a per-row scalar, so it commutes with W).
+#include "kernels.h"
+
+namespace {
+
+template <int EPI> struct EpiTraits { static constexpr int TPI = 1; };
+template <> struct EpiTraits<EPI_QKV> { static constexpr int TPI = 2; };
+template <> struct EpiTraits<EPI_GATEUP> { static constexpr int TPI = 2; };
+
+// weight row base of tile `which` of work item `item`
+template <int EPI>
+__device__ __forceinline__ const bf16 *tile_rows(const GemmArgs &a, int item, int which) {
+    if (EPI == EPI_QKV) {
+        const int hp = a.D.hd >> 5;                 // pairs per head
+        const int nq = a.D.nh * hp, nk = a.D.nkv * hp;
+        if (item < nq + nk) {
+            const bf16 *W = item < nq ? a.W0 : a.W1;
+            const int it = item < nq ? item : item - nq;
+            const int head = it / hp, jb = it - head * hp;
+            const int row = head * a.D.hd + jb * 16 + which * (a.D.hd >> 1);
+            return W + (size_t)row * a.K;
+        }
+        const int it = item - nq - nk;
+        return a.W2 + (size_t)(32 * it + 16 * which) * a.K;
+    }
+    if (EPI == EPI_GATEUP) return (which ? a.W1 : a.W0) + (size_t)(16 * item) * a.K;
+    return a.W0 + (size_t)(16 * item) * a.K;
+}
+
+template <int NT, int D, int EPI>
+__global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_kernel(const GemmArgs a) {
+    constexpr int TPI = EpiTraits<EPI>::TPI;
+    constexpr int HB = D / 2;
+    constexpr int NC = NT * 8;                      // activation-row columns handled
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float4 *red = reinterpret_cast<float4 *>(smem_raw);                       // [8 warps][NT][32]
+    float *res = reinterpret_cast<float *>(smem_raw + sizeof(float4) * 8 * NT * 32);  // [TPI][NC][16]
+    float *rscale = res + TPI * NC * 16;                                      // [NC]
+    float *best_v = rscale + NC;                                              // [NC]
+    int *best_i = reinterpret_cast<int *>(best_v + NC);                       // [NC]
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
+    const int K = a.K;
+    const int n_ksteps = (K + 31) >> 5;
+    const int nkw = (n_ksteps - warp + 7) >> 3;     // k-steps of this warp per tile (>= 1 since K >= 256)
+    const int my_items = (a.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int my_tiles = my_items * TPI;
+    const int total = my_tiles * nkw;
+
+    uint4 wv[2][HB][2];
+    uint4 xv[2][HB][NT];
+
+    // ---- producer cursors
+    int p_tile = 0, p_ksi = 0;                      // weights
+    const bf16 *p_w = nullptr;
+    auto p_enter_tile = [&]() {
+        if (p_tile < my_tiles) {
+            const int item = blockIdx.x + (p_tile / TPI) * gridDim.x;
+            p_w = tile_rows<EPI>(a, item, p_tile % TPI) + (size_t)g * K + 8 * t;
+        }
+    };
+    p_enter_tile();
+    auto load_w = [&](uint4 (&dst)[2]) {
+        if (p_tile < my_tiles) {
+            const int k0 = ((warp + 8 * p_ksi) << 5) + 8 * t;
+            if (k0 < K) {
+                dst[0] = ldg_stream16(p_w + (k0 - 8 * t));
+                dst[1] = ldg_stream16(p_w + (size_t)8 * K + (k0 - 8 * t));
+            } else {
+                dst[0] = make_uint4(0, 0, 0, 0);
+                dst[1] = make_uint4(0, 0, 0, 0);
+            }
+            if (++p_ksi == nkw) { p_ksi = 0; ++p_tile; p_enter_tile(); }
+        }
+    };
+    // activations: same k sequence, tile-independent
+    int x_units = 0, x_ksi = 0;
+    const bf16 *xrow[NT];
+    auto load_x = [&](uint4 (&dst)[NT]) {
+        if (x_units < total) {
+            const int k0 = ((warp + 8 * x_ksi) << 5) + 8 * t;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+                dst[nt] = (xrow[nt] != nullptr && k0 < K) ? ldg_act16(xrow[nt] + k0) : make_uint4(0, 0, 0, 0);
+            if (++x_ksi == nkw) x_ksi = 0;
+            ++x_units;
+        }
+    };
+
+    // weights of the first two batches go out before the producer kernel has finished
+#pragma unroll
+    for (int b = 0; b < 2; ++b)
+#pragma unroll
+        for (int j = 0; j < HB; ++j) load_w(wv[b][j]);
+    pdl_launch();
+    pdl_wait();
+
+    const PassPlan *plan = a.plan;
+    const int m = plan->m;
+    // activation row pointers of this thread's columns
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        const int c = nt * 8 + g;
+        xrow[nt] = nullptr;
+        if (c < m) {
+            size_t r;
+            if (EPI == EPI_QKV) r = stack_row(a.D, a.layer - 1, plan->rows[c].seq, plan->rows[c].slot);
+            else if (EPI == EPI_LMHEAD) r = a.x_by_row ? (size_t)c : (size_t)plan->rows[c].seq * a.D.S + plan->rows[c].slot;
+            else r = c;
+            xrow[nt] = a.X + r * (size_t)K;
+        }
+    }
+#pragma unroll
+    for (int b = 0; b < 2; ++b)
+#pragma unroll
+        for (int j = 0; j < HB; ++j) load_x(xv[b][j]);
+
+    // per-row 1/rms from the producer's partial sums of squares
+    if (EPI == EPI_QKV || EPI == EPI_GATEUP) {
+        for (int c = warp; c < NC; c += DEL_GEMM_WARPS) {
+            float s = 0.f;
+            if (c < m) {
+                const float *ss;
+                if (EPI == EPI_GATEUP) ss = a.B.SSM + (size_t)c * a.D.n_sst;
+                else ss = a.B.SS + stack_row(a.D, a.layer - 1, plan->rows[c].seq, plan->rows[c].slot) * a.D.n_sst;
+                for (int i = lane; i < a.D.n_sst; i += 32) s += ldg_cg_f32(ss + i);
+            }
+            s = warp_sum(s);
+            if (lane == 0) rscale[c] = rsqrtf(s / (float)a.D.d + a.D.eps);
+        }
+    }
+    if (EPI == EPI_LMHEAD) {
+        for (int c = tid; c < NC; c += DEL_GEMM_THREADS) { best_v[c] = -INFINITY; best_i[c] = 0x7fffffff; }
+    }
+    __syncthreads();
+
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+
+    int c_tile = 0, c_ksi = 0, consumed = 0;
+
+    auto tile_end = [&]() {
+        // fixed-order sum of the 8 warps' partials
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            red[(warp * NT + nt) * 32 + lane] = make_float4(acc[nt][0], acc[nt][1], acc[nt][2], acc[nt][3]);
+            acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+        }
+        __syncthreads();
+        const int which = c_tile % TPI;
+        for (int e = tid; e < NT * 32; e += DEL_GEMM_THREADS) {
+            float4 s = red[e];
+#pragma unroll
+            for (int w = 1; w < DEL_GEMM_WARPS; ++w) {
+                const float4 v = red[w * NT * 32 + e];
+                s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+            }
+            const int nt = e >> 5, l2 = e & 31, g2 = l2 >> 2, t2 = l2 & 3;
+            float *r0 = res + ((which * NC) + nt * 8 + 2 * t2) * 16;
+            r0[g2] = s.x; r0[16 + g2] = s.y; r0[g2 + 8] = s.z; r0[16 + g2 + 8] = s.w;
+        }
+        __syncthreads();
+        if (which != TPI - 1) return;
+        const int item = blockIdx.x + (c_tile / TPI) * gridDim.x;
+        const int i = tid & 15;
+        for (int c = tid >> 4; c < NC; c += DEL_GEMM_THREADS / 16) {
+            const bool valid = c < m;
+            const RowDesc rd = valid ? plan->rows[c] : RowDesc{0, 0, 0, 0};
+            const float ra = res[c * 16 + i];
+            if (EPI == EPI_QKV) {
+                if (!valid) continue;
+                const float r = rscale[c];
+                const float va = r * ra, vb = r * res[(NC + c) * 16 + i];
+                const int hd = a.D.hd, half = hd >> 1, hp = hd >> 5;
+                const int nq = a.D.nh * hp, nk = a.D.nkv * hp;
+                const int pg = a.B.PT[rd.seq * a.D.pages_per_seq + (rd.pos >> 4)];
+                const int sl = rd.pos & 15;
+                if (item < nq + nk) {
+                    const bool isq = item < nq;
+                    const int it = isq ? item : item - nq;
+                    const int head = it / hp, j = (it - head * hp) * 16 + i;
+                    const float cs = a.B.rope_cos[(size_t)rd.pos * half + j], sn = a.B.rope_sin[(size_t)rd.pos * half + j];
+                    const float oa = va * cs - vb * sn, ob = vb * cs + va * sn;
+                    if (isq) {
+                        bf16 *q = a.B.Q + (size_t)c * (a.D.nh * hd) + head * hd + j;
+                        q[0] = __float2bfloat16_rn(oa);
+                        q[half] = __float2bfloat16_rn(ob);
+                    } else {
+                        bf16 *kp = a.B.KP + ((((size_t)pg * a.D.L + (a.layer - 1)) * a.D.nkv + head) * 16 + sl) * hd + j;
+                        kp[0] = __float2bfloat16_rn(oa);
+                        kp[half] = __float2bfloat16_rn(ob);
+                    }
+                } else {
+                    const int n0 = 32 * (item - nq - nk) + i;      // value feature of tile 0; tile 1 is +16
+                    const int kvh = n0 / hd, dim = n0 - kvh * hd;
+                    bf16 *vp = a.B.VP + ((((size_t)pg * a.D.L + (a.layer - 1)) * a.D.nkv + kvh) * hd + dim) * 16 + sl;
+                    vp[0] = __float2bfloat16_rn(va);
+                    vp[16 * 16] = __float2bfloat16_rn(vb);
+                }
+            } else if (EPI == EPI_GATEUP) {
+                if (!valid) continue;
+                const float r = rscale[c];
+                const float gate = r * ra, up = r * res[(NC + c) * 16 + i];
+                const float act = gate / (1.f + __expf(-gate)) * up;
+                a.B.ACT[(size_t)c * a.D.F + 16 * item + i] = __float2bfloat16_rn(act);
+            } else if (EPI == EPI_OPROJ || EPI == EPI_DOWN) {
+                const int o = 16 * item + i;
+                float h = 0.f;
+                if (valid) {
+                    if (EPI == EPI_OPROJ) {
+                        h = ldg_cg_f32(a.B.H + stack_row(a.D, a.layer - 1, rd.seq, rd.slot) * a.D.d + o) + ra;
+                        a.B.HM[(size_t)c * a.D.d + o] = h;
+                        a.B.XM[(size_t)c * a.D.d + o] = __float2bfloat16_rn(h * bf16_to_f(a.gain_a[o]));
+                    } else {
+                        h = ldg_cg_f32(a.B.HM + (size_t)c * a.D.d + o) + ra;
+                        const size_t sr = stack_row(a.D, a.layer, rd.seq, rd.slot);
+                        a.B.H[sr * a.D.d + o] = h;
+                        if (a.gain_a) a.B.XS[sr * a.D.d + o] = __float2bfloat16_rn(h * bf16_to_f(a.gain_a[o]));
+                        if (a.gain_b)
+                            a.B.XE[((size_t)rd.seq * a.D.S + rd.slot) * a.D.d + o] = __float2bfloat16_rn(h * bf16_to_f(a.gain_b[o]));
+                    }
+                }
+                float ss = h * h;
+                ss += __shfl_xor_sync(0xffffffffu, ss, 8);
+                ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+                ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+                ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+                if (valid && i == 0) {
+                    if (EPI == EPI_OPROJ) a.B.SSM[(size_t)c * a.D.n_sst + item] = ss;
+                    else a.B.SS[stack_row(a.D, a.layer, rd.seq, rd.slot) * a.D.n_sst + item] = ss;
+                }
+            } else if (EPI == EPI_LMHEAD) {
+                float v = valid ? ra : -INFINITY;      // the row's 1/rms is positive: it cannot change the arg-max
+                int idx = 16 * item + i;
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) {
+                    const float v2 = __shfl_xor_sync(0xffffffffu, v, o);
+                    const int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
+                    if (v2 > v || (v2 == v && i2 < idx)) { v = v2; idx = i2; }
+                }
+                if (valid && i == 0 && (v > best_v[c] || (v == best_v[c] && idx < best_i[c]))) { best_v[c] = v; best_i[c] = idx; }
+            }
+        }
+        // `res` and `best_*` are next written after the following tile's first barrier
+    };
+
+    auto consume = [&](uint4 (&w)[2], uint4 (&x)[NT]) {
+        if (consumed < total) {
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                mma_bf16_16816(acc[nt], w[0].x, w[1].x, w[0].y, w[1].y, x[nt].x, x[nt].y);
+                mma_bf16_16816(acc[nt], w[0].z, w[1].z, w[0].w, w[1].w, x[nt].z, x[nt].w);
+            }
+            ++consumed;
+            if (++c_ksi == nkw) { c_ksi = 0; tile_end(); ++c_tile; }
+        }
+    };
+
+    for (int base = 0; base < total; base += D) {
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+#pragma unroll
+            for (int j = 0; j < HB; ++j) consume(wv[b][j], xv[b][j]);
+#pragma unroll
+            for (int j = 0; j < HB; ++j) { load_w(wv[b][j]); load_x(xv[b][j]); }
+        }
+    }
+
+    if (EPI == EPI_LMHEAD) {
+        __syncthreads();
+        for (int c = tid; c < m; c += DEL_GEMM_THREADS) {
+            a.B.LPV[(size_t)blockIdx.x * DEL_ROWS_MAX + c] = best_v[c];
+            a.B.LPI[(size_t)blockIdx.x * DEL_ROWS_MAX + c] = best_i[c];
+        }
+    }
+}
+
+template <int NT> constexpr int depth_for() { return NT == 1 ? 8 : 4; }
+
+template <int NT, int EPI>
+cudaError_t launch_nt(const GemmArgs &a, int grid, cudaStream_t st, bool pdl) {
+    constexpr int D = depth_for<NT>();
+    constexpr int TPI = EpiTraits<EPI>::TPI;
+    constexpr int NC = NT * 8;
+    const size_t smem = sizeof(float4) * 8 * NT * 32 + sizeof(float) * (TPI * NC * 16 + 3 * NC);
+    auto kern = rowgemm_kernel<NT, D, EPI>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(DEL_GEMM_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+template <int EPI>
+cudaError_t launch_epi(const GemmArgs &a, int m, int n_sms, cudaStream_t st, bool pdl) {
+    const int nt = (m + 7) / 8;
+    if (nt <= 1) return launch_nt<1, EPI>(a, min(a.n_items, 2 * n_sms), st, pdl);
+    if (nt <= 2) return launch_nt<2, EPI>(a, min(a.n_items, 2 * n_sms), st, pdl);
+    if (nt <= 4) return launch_nt<4, EPI>(a, min(a.n_items, n_sms), st, pdl);
+    return launch_nt<8, EPI>(a, min(a.n_items, n_sms), st, pdl);
+}
+
+}  // namespace
+
+cudaError_t launch_rowgemm(int epi, const GemmArgs &a, int m, int n_sms, cudaStream_t st, bool pdl) {
+    switch (epi) {
+        case EPI_QKV: return launch_epi<EPI_QKV>(a, m, n_sms, st, pdl);
+        case EPI_OPROJ: return launch_epi<EPI_OPROJ>(a, m, n_sms, st, pdl);
+        case EPI_GATEUP: return launch_epi<EPI_GATEUP>(a, m, n_sms, st, pdl);
+        case EPI_DOWN: return launch_epi<EPI_DOWN>(a, m, n_sms, st, pdl);
+        case EPI_LMHEAD: return launch_epi<EPI_LMHEAD>(a, m, n_sms, st, pdl);
+    }
+    return cudaErrorInvalidValue;
+}
+
+int rowgemm_lmhead_grid(int n_items, int m, int n_sms) {
+    const int nt = (m + 7) / 8;
+    const int cap = nt <= 2 ? 2 * n_sms : n_sms;
+    return n_items < cap ? n_items : cap;
+}

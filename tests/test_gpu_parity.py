@@ -1,0 +1,207 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle.  Needs a B200."""
+import json
+import os
+
+import numpy as np
+import pytest
+
+import synth
+from cases import TINY, TINY_GQA, TINY_SHORT
+from parity import MARGIN, ref_from_golden, ref_from_oracle, run_sequence
+
+pytestmark = pytest.mark.gpu
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def make_ctx(cfg, weights, **kw):
+    import paper_2504_05598_b200 as dl
+    dev = dl.upload_weights(weights)
+    return dl.DelContext(dl.make_shape(cfg, **kw), dev)
+
+
+@pytest.fixture(scope="module", params=[TINY, TINY_GQA, TINY_SHORT], ids=lambda c: c.name)
+def small(request):
+    cfg = request.param
+    w = synth.make_weights(cfg)
+    return cfg, w, make_ctx(cfg, w)
+
+
+def test_prefill_hidden_kv_and_logits(small):
+    """Element-wise: hidden states of every layer, cached K/V rows and exit-head logits after a prefill."""
+    import oracle
+    cfg, w, ctx = small
+    prompt = synth.make_prompt(cfg)
+    o = oracle.OracleSeq(cfg, w)
+    o.prefill(prompt)
+    ctx.prefill(0, prompt, cfg.gen_len)
+    W = min(cfg.init_window, len(prompt))
+    P = len(prompt)
+    for l in range(cfg.n_layers + 1):
+        for j in (0, W - 1):
+            ref = o.hidden(l, j)
+            got = ctx.get_hidden(0, l, j)
+            scale = np.abs(ref).max()
+            assert np.abs(got - ref).max() <= 2e-2 * scale + 1e-6, (l, j, np.abs(got - ref).max(), scale)
+    for l in (1, cfg.n_layers):
+        for pos in (0, P // 2, P - 1):
+            k, v = ctx.get_kv(0, l, pos)
+            kr, vr = o.k_row(l, pos), o.v_row(l, pos)
+            assert np.abs(k - kr).max() <= 2e-2 * np.abs(kr).max() + 1e-6, ("k", l, pos)
+            assert np.abs(v - vr).max() <= 2e-2 * np.abs(vr).max() + 1e-6, ("v", l, pos)
+    # per-layer logits of the exit head: max-abs 3e-2 after bf16
+    for l in (1, cfg.n_layers // 2, cfg.n_layers):
+        _, _, ref = o.exit_head(o.hidden(l, W - 1), want_logits=True)
+        got = ctx.debug_logits(0, l, W - 1)
+        assert np.abs(got - ref).max() <= 3e-2, (l, np.abs(got - ref).max())
+        if np.sort(ref)[-1] - np.sort(ref)[-2] > MARGIN:
+            assert int(np.argmax(got)) == int(np.argmax(ref))
+
+
+def test_dynamic_rounds_match_oracle(small):
+    cfg, w, ctx = small
+    ref = ref_from_oracle(cfg, w, synth.make_prompt(cfg))
+    rep = run_sequence(ctx, 0, ref, cfg.gen_len)
+    print(f"{cfg.name}: rounds {rep.rounds} compared {rep.compared} flips {rep.flips} resyncs {rep.resyncs}")
+    assert rep.ok(), rep.failures[:5]
+    assert rep.rounds == len(ref.rounds)
+    assert rep.flips <= max(3, rep.compared // 50)          # flips are rare, not the rule
+
+
+def test_every_fixed_setting_reproduces_the_greedy_stream(small):
+    """Speculative greedy output equals plain greedy output for every (E, gamma), gamma = 0 included."""
+    cfg, w, ctx = small
+    prompt = synth.make_prompt(cfg)
+    settings = [(1, 0)] + [(E, g) for E in range(cfg.e_min, cfg.e_max + 1) for g in range(max(1, cfg.g_min), cfg.g_max + 1)]
+    for E, g in settings:
+        ref = ref_from_oracle(cfg, w, prompt, policy=(E, g))
+        rep = run_sequence(ctx, 0, ref, cfg.gen_len, policy=(E, g))
+        assert rep.ok(), ((E, g), rep.failures[:5])
+        assert rep.rounds == len(ref.rounds)
+
+
+def test_step_calls_equal_round_call(small):
+    cfg, w, ctx = small
+    prompt = synth.make_prompt(cfg)
+    first = ctx.prefill(0, prompt, 24)
+    a_tokens, E, g = [first.tokens[0]], first.next_E, first.next_gamma
+    a_trace = []
+    while len(a_tokens) < 24:
+        ctx.draft(0, E, g)
+        ctx.verify(0)
+        out = ctx.layer_accept(0)
+        sh, cn = ctx.get_shadow(0)
+        E, g = ctx.select(0)
+        a_tokens += out.emitted()
+        a_trace.append((out.E, out.g, out.n_accept, sh.copy(), cn.copy(), E, g))
+    first = ctx.prefill(0, prompt, 24)
+    b_tokens = [first.tokens[0]]
+    k = 0
+    while len(b_tokens) < 24:
+        out = ctx.round()[0]
+        sh, cn = ctx.get_shadow(0)
+        b_tokens += out.emitted()
+        t = a_trace[k]
+        assert (out.E, out.g, out.n_accept, out.next_E, out.next_gamma) == (t[0], t[1], t[2], t[5], t[6])
+        assert np.array_equal(sh[:, :out.g + 1], t[3][:, :out.g + 1]) and np.array_equal(cn, t[4])
+        k += 1
+    assert a_tokens == b_tokens and len(a_tokens) == 24
+    # run-to-run determinism: a third pass gives the same tokens
+    first = ctx.prefill(0, prompt, 24)
+    c_tokens = [first.tokens[0]]
+    while len(c_tokens) < 24:
+        c_tokens += ctx.round()[0].emitted()
+    assert c_tokens == b_tokens
+
+
+def test_error_codes(small):
+    import paper_2504_05598_b200 as dl
+    cfg, w, ctx = small
+    lib, h = ctx.lib, ctx._h
+    prompt = synth.make_prompt(cfg)
+    p = np.ascontiguousarray(prompt, dtype=np.int32)
+    assert lib.del_prefill(h, 99, p.ctypes.data, len(p), 8, None) == dl.EINVAL
+    assert lib.del_prefill(h, 0, p.ctypes.data, 0, 8, None) == dl.EINVAL
+    assert lib.del_prefill(h, 0, p.ctypes.data, len(p), 10 ** 6, None) == dl.ENOSPC
+    bad = p.copy()
+    bad[3] = cfg.vocab
+    assert lib.del_prefill(h, 0, bad.ctypes.data, len(bad), 8, None) == dl.EINVAL
+    ctx.release(0)
+    assert lib.del_draft(h, 0, 1, 1) == dl.ESTATE                      # no prefill yet
+    ctx.prefill(0, prompt, 8)
+    assert lib.del_verify(h, 0) == dl.ESTATE                           # verify before draft
+    assert lib.del_draft(h, 0, cfg.n_layers, 1) == dl.EINVAL           # E must leave layers to verify with
+    assert lib.del_draft(h, 0, 1, cfg.g_max + 1) == dl.EINVAL
+    assert lib.del_layer_accept(h, 0, None) == dl.ESTATE
+    ctx.draft(0, 1, 1)
+    assert lib.del_draft(h, 0, 1, 1) == dl.ESTATE                      # round in progress
+    ctx.verify(0)
+    ctx.layer_accept(0)
+    # the context is still healthy
+    assert ctx.round()[0].n_emitted >= 1
+
+
+def test_generation_stops_at_budget(small):
+    cfg, w, ctx = small
+    import paper_2504_05598_b200 as dl
+    first = ctx.prefill(0, synth.make_prompt(cfg), 9)
+    n = 1
+    while True:
+        rc, outs = ctx.try_round()
+        if rc != dl.OK:
+            assert rc == dl.ESTATE
+            break
+        assert 1 <= outs[0].n_emitted <= outs[0].g + 1
+        n += outs[0].n_emitted
+    assert n == 9
+
+
+def test_batch_of_independent_sequences():
+    """Three sequences with their own prompts, (E, gamma) and statistics share the layer passes."""
+    cfg = synth.small_variant(TINY_GQA, batch=3)
+    w = synth.make_weights(cfg)
+    ctx = make_ctx(cfg, w)
+    refs = [ref_from_oracle(cfg, w, synth.make_prompt(cfg, s), gen_len=20 + 7 * s) for s in range(3)]
+    for s in range(3):
+        out = ctx.prefill(s, refs[s].prompt, 20 + 7 * s)
+        assert out.tokens[0] == refs[s].first_token
+    got = [[r.first_token] for r in refs]
+    k = [0, 0, 0]
+    import paper_2504_05598_b200 as dl
+    while True:
+        rc, outs = ctx.try_round()
+        if rc != dl.OK:
+            break
+        for s in range(3):
+            if outs[s].n_emitted == 0:
+                continue
+            r = refs[s].rounds[k[s]]
+            clean = (r.margin > MARGIN).all()
+            if clean:
+                assert (outs[s].E, outs[s].g, outs[s].n_accept) == (r.E, r.g, r.n), (s, k[s])
+                assert outs[s].emitted() == list(r.emitted)
+                assert (outs[s].next_E, outs[s].next_gamma) == (r.next_E, r.next_gamma)
+            k[s] += 1
+            got[s] += outs[s].emitted()
+    for s in range(3):
+        assert len(got[s]) == 20 + 7 * s
+        low = any((r.margin <= MARGIN).any() for r in refs[s].rounds) or (refs[s].init_margin <= MARGIN).any()
+        if not low:
+            assert got[s] == refs[s].tokens
+
+
+@pytest.mark.parametrize("name,max_rounds", [("llama2_7b", None), ("llama32_1b", 60)])
+def test_full_size_config_against_stored_trace(name, max_rounds):
+    """The benchmark shapes, in the configuration bench.py times, against the oracle's stored trace."""
+    path = os.path.join(GOLDEN, f"trace_{name}.json")
+    if not os.path.exists(path):
+        pytest.skip("no stored trace")
+    doc = json.load(open(path))
+    cfg = synth.CONFIGS[name]
+    assert doc["seed"] == cfg.seed and doc["prompt_len"] == cfg.prompt_len
+    w = synth.make_weights(cfg)
+    ctx = make_ctx(cfg, w)
+    ref = ref_from_golden(doc, 0, synth.make_prompt(cfg, 0))
+    rep = run_sequence(ctx, 0, ref, doc["gen_len"], max_rounds=max_rounds)
+    print(f"{name}: rounds {rep.rounds} compared {rep.compared} flips {rep.flips} resyncs {rep.resyncs}")
+    assert rep.ok(), rep.failures[:8]
+    assert rep.flips <= rep.compared // 20
