@@ -186,10 +186,18 @@ int del_committed_len(del_ctx *ctx, int seq);
 int del_release(del_ctx *ctx, int seq);
 /* Kernel launches enqueued since del_init (for launch accounting). */
 int64_t del_launch_count(const del_ctx *ctx);
+/* Bytes the library itself copied host->device (plans, page-table entries, prompts) and
+ * device->host (round results) since del_init. */
+int del_get_traffic(const del_ctx *ctx, int64_t *h2d_bytes, int64_t *d2h_bytes);
 /* Switches of the launch machinery (bit 0: programmatic dependent launch, bit 1: CUDA graphs for
- * single-sequence rounds, bit 2: tcgen05 LM head instead of the streaming one).  Returns the
- * previous flags. */
+ * single-sequence rounds, bit 2: tcgen05 LM head instead of the streaming one, bit 3: record CUDA
+ * events around every launch).  Returns the previous flags. */
 int del_set_flags(del_ctx *ctx, int flags);
+
+/* With flag bit 3 set, per kernel class (0 QKV, 1 attention, 2 O-proj, 3 gate/up, 4 down, 5 draft LM
+ * head, 6 stacked LM head, 7 other): summed device time in ms, launches, and algorithmic bytes (weights
+ * or KV the launches had to read).  HOST arrays of 8 (any may be NULL); reset != 0 clears the sums. */
+int del_get_kernel_times(del_ctx *ctx, double *ms, int64_t *launches, double *bytes, int reset);
 
 const char *del_strerror(int code);
 /* Text of the last CUDA error seen by this context ("" if none). */

@@ -21,12 +21,13 @@ MAX_GAMMA = 31
 MAX_ROWS = 64
 
 OK, EINVAL, ENOSPC, ESTATE, ETIMEOUT, ECUDA = 0, -1, -2, -3, -4, -5
-FLAG_PDL, FLAG_GRAPH, FLAG_TC = 1, 2, 4
+FLAG_PDL, FLAG_GRAPH, FLAG_TC, FLAG_TIMING = 1, 2, 4, 8
+KERNEL_CLASSES = ["qkv_rope", "attention", "o_proj", "gate_up", "down", "lm_head_draft", "lm_head_stacked", "other"]
 
 EXPORTS = ["del_workspace_bytes", "del_init", "del_prefill", "del_draft", "del_verify", "del_layer_accept",
            "del_select", "del_round", "del_set_policy", "del_get_stats", "del_set_stats", "del_get_shadow",
            "del_get_drafts", "del_force_token", "del_get_hidden", "del_debug_logits", "del_get_kv", "del_committed_len", "del_release",
-           "del_launch_count", "del_set_flags", "del_strerror", "del_last_cuda_error", "del_destroy"]
+           "del_launch_count", "del_get_traffic", "del_set_flags", "del_get_kernel_times", "del_strerror", "del_last_cuda_error", "del_destroy"]
 
 
 class Shape(C.Structure):
@@ -111,8 +112,12 @@ def load_library(build_if_missing: bool = True):
     L.del_release.argtypes = [vp, ci]
     L.del_launch_count.restype = C.c_int64
     L.del_launch_count.argtypes = [vp]
+    L.del_get_traffic.restype = ci
+    L.del_get_traffic.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
     L.del_set_flags.restype = ci
     L.del_set_flags.argtypes = [vp, ci]
+    L.del_get_kernel_times.restype = ci
+    L.del_get_kernel_times.argtypes = [vp, vp, vp, vp, ci]
     L.del_strerror.restype = C.c_char_p
     L.del_strerror.argtypes = [ci]
     L.del_last_cuda_error.restype = C.c_char_p
@@ -295,6 +300,19 @@ class DelContext:
 
     def launch_count(self) -> int:
         return int(self.lib.del_launch_count(self._h))
+
+    def traffic(self):
+        a, b = C.c_int64(), C.c_int64()
+        self._ck(self.lib.del_get_traffic(self._h, C.byref(a), C.byref(b)), "del_get_traffic")
+        return a.value, b.value
+
+    def kernel_times(self, reset: bool = True):
+        ms = np.zeros(8, dtype=np.float64)
+        n = np.zeros(8, dtype=np.int64)
+        by = np.zeros(8, dtype=np.float64)
+        self._ck(self.lib.del_get_kernel_times(self._h, ms.ctypes.data, n.ctypes.data, by.ctypes.data, int(reset)),
+                 "del_get_kernel_times")
+        return {k: {"ms": float(ms[i]), "launches": int(n[i]), "bytes": float(by[i])} for i, k in enumerate(KERNEL_CLASSES)}
 
     def set_flags(self, flags: int) -> int:
         return self.lib.del_set_flags(self._h, flags)

@@ -13,7 +13,8 @@
 namespace {
 
 constexpr int PLAN_RING = 192;
-constexpr int FLAG_PDL = 1, FLAG_GRAPH = 2, FLAG_TC = 4;
+constexpr int FLAG_PDL = 1, FLAG_GRAPH = 2, FLAG_TC = 4, FLAG_TIMING = 8;
+enum { CLS_QKV = 0, CLS_ATTN, CLS_OPROJ, CLS_GATEUP, CLS_DOWN, CLS_LMHEAD, CLS_LMSTACK, CLS_OTHER, CLS_N };
 
 struct SeqHost {
     bool active = false;
@@ -58,7 +59,15 @@ struct del_ctx {
     del_round_out *out_host = nullptr, *out_dev = nullptr; // [B]
     void *stage_host = nullptr;                            // small pinned scratch
     float *dbg_dev = nullptr;                              // [V] debug logits / kv rows
-    int64_t launches = 0;
+    int64_t launches = 0, h2d_bytes = 0, d2h_bytes = 0;
+    // optional per-launch timing (FLAG_TIMING): events around every launch, summed per kernel class
+    struct TimeRec { int cls, ev; double bytes; };
+    std::vector<cudaEvent_t> ev_pool;
+    std::vector<TimeRec> recs;
+    int ev_used = 0, cur_cls = CLS_OTHER;
+    double cur_bytes = 0.0;
+    double cls_ms[CLS_N] = {0}, cls_bytes[CLS_N] = {0};
+    int64_t cls_n[CLS_N] = {0};
     char err[256] = {0};
     cudaError_t last = cudaSuccess;
 };
@@ -139,12 +148,47 @@ int fail(del_ctx *c, cudaError_t e) {
         cudaError_t e__ = (call);                  \
         if (e__ != cudaSuccess) return fail(c, e__); \
     } while (0)
+int timing_begin(del_ctx *c) {
+    if (!(c->flags & FLAG_TIMING)) return -1;
+    while ((int)c->ev_pool.size() < 2 * (c->ev_used + 1)) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) return -1;
+        c->ev_pool.push_back(e);
+    }
+    const int i = c->ev_used++;
+    cudaEventRecord(c->ev_pool[2 * i], c->st);
+    return i;
+}
+void timing_end(del_ctx *c, int i) {
+    if (i >= 0) {
+        cudaEventRecord(c->ev_pool[2 * i + 1], c->st);
+        c->recs.push_back({c->cur_cls, i, c->cur_bytes});
+    }
+    c->cur_cls = CLS_OTHER;
+    c->cur_bytes = 0.0;
+}
+// call after the stream has been synchronised
+void timing_collect(del_ctx *c) {
+    for (const auto &r : c->recs) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, c->ev_pool[2 * r.ev], c->ev_pool[2 * r.ev + 1]) == cudaSuccess) {
+            c->cls_ms[r.cls] += ms;
+            c->cls_bytes[r.cls] += r.bytes;
+            c->cls_n[r.cls] += 1;
+        }
+    }
+    c->recs.clear();
+    c->ev_used = 0;
+}
 #define LAUNCH(call)                               \
     do {                                           \
+        const int t__ = timing_begin(c);           \
         cudaError_t e__ = (call);                  \
         if (e__ != cudaSuccess) return fail(c, e__); \
         ++c->launches;                             \
+        timing_end(c, t__);                        \
     } while (0)
+#define TAG(cls, bytes) (c->cur_cls = (cls), c->cur_bytes = (double)(bytes))
 
 bool pdl(const del_ctx *c) { return (c->flags & FLAG_PDL) != 0; }
 
@@ -171,6 +215,7 @@ int plan_begin(del_ctx *c, int need) {
 int plan_commit(del_ctx *c, const PlanBatch &b) {
     if (b.count == 0) return DEL_OK;
     CK(cudaMemcpyAsync(c->plan_dev + b.first, c->plan_host + b.first, sizeof(PassPlan) * b.count, cudaMemcpyHostToDevice, c->st));
+    c->h2d_bytes += sizeof(PassPlan) * b.count;
     c->plan_cur = b.first + b.count;
     return DEL_OK;
 }
@@ -210,6 +255,7 @@ int ensure_pages(del_ctx *c, int sq, int positions) {
     CK(cudaMemcpyAsync(c->B.PT + (size_t)sq * c->D.pages_per_seq + first_new,
                        c->pt_host.data() + (size_t)sq * c->D.pages_per_seq + first_new,
                        sizeof(int32_t) * (need - first_new), cudaMemcpyHostToDevice, c->st));
+    c->h2d_bytes += sizeof(int32_t) * (need - first_new);
     return DEL_OK;
 }
 
@@ -270,6 +316,7 @@ int run_layer(del_ctx *c, const PassInfo &pi, int l, bool write_exit) {
         a.n_items = (D.nh + 2 * D.nkv) * (D.hd / 32);
         a.X = c->B.XS;
         a.W0 = c->wq[l - 1]; a.W1 = c->wk[l - 1]; a.W2 = c->wv[l - 1];
+        TAG(CLS_QKV, 2.0 * (D.nh + 2 * D.nkv) * D.hd * D.d);
         LAUNCH(launch_rowgemm(EPI_QKV, a, pi.m, c->n_sms, c->st, P));
     }
     {
@@ -281,6 +328,12 @@ int run_layer(del_ctx *c, const PassInfo &pi, int l, bool write_exit) {
         ns = std::max(1, std::min(std::min(ns, 16), (pages + 1) / 2));
         a.n_splits = ns;
         a.max_rows = pi.max_rows;
+        {
+            double kvb = 0.0;
+            const PassPlan &pp = c->plan_host[pi.plan_idx];
+            for (int i = 0; i < pp.n_seg; ++i) kvb += 4.0 * (pp.seg[i].pos0 + pp.seg[i].nrows) * D.nkv * D.hd;
+            TAG(CLS_ATTN, kvb);
+        }
         LAUNCH(launch_attention(a, pi.n_seg, c->st, P));
     }
     {
@@ -290,6 +343,7 @@ int run_layer(del_ctx *c, const PassInfo &pi, int l, bool write_exit) {
         a.X = c->B.ATT;
         a.W0 = c->wo[l - 1];
         a.gain_a = c->ffn_norm[l - 1];
+        TAG(CLS_OPROJ, 2.0 * D.d * D.nh * D.hd);
         LAUNCH(launch_rowgemm(EPI_OPROJ, a, pi.m, c->n_sms, c->st, P));
     }
     {
@@ -298,6 +352,7 @@ int run_layer(del_ctx *c, const PassInfo &pi, int l, bool write_exit) {
         a.n_items = D.F / 16;
         a.X = c->B.XM;
         a.W0 = c->w_gate[l - 1]; a.W1 = c->w_up[l - 1];
+        TAG(CLS_GATEUP, 4.0 * D.F * D.d);
         LAUNCH(launch_rowgemm(EPI_GATEUP, a, pi.m, c->n_sms, c->st, P));
     }
     {
@@ -308,6 +363,7 @@ int run_layer(del_ctx *c, const PassInfo &pi, int l, bool write_exit) {
         a.W0 = c->w_down[l - 1];
         a.gain_a = l < D.L ? c->attn_norm[l] : nullptr;
         a.gain_b = write_exit ? c->final_norm : nullptr;
+        TAG(CLS_DOWN, 2.0 * D.d * D.F);
         LAUNCH(launch_rowgemm(EPI_DOWN, a, pi.m, c->n_sms, c->st, P));
     }
     return DEL_OK;
@@ -376,6 +432,7 @@ int enqueue_draft(del_ctx *c, const std::vector<Job> &jobs) {
         a.n_items = c->D.V / 16;
         a.X = c->B.XE;
         a.W0 = c->lm_head;
+        TAG(CLS_LMHEAD, 2.0 * c->D.V * c->D.d);
         LAUNCH(launch_rowgemm(EPI_LMHEAD, a, full.m, c->n_sms, c->st, P));
         CtlArgs ca = ctl_base(c, full.plan_idx);
         ca.n_part = rowgemm_lmhead_grid(a.n_items, full.m, c->n_sms);
@@ -444,6 +501,7 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
     up->n_rows = rows;
     if (rows > c->R_max) return DEL_EINVAL;
     CK(cudaMemcpyAsync(c->up_dev, up, sizeof(UpdatePlan), cudaMemcpyHostToDevice, c->st));
+    c->h2d_bytes += sizeof(UpdatePlan);
     const bool P = pdl(c);
     CtlArgs ca = ctl_base(c, -1);
     ca.mode = mode;
@@ -470,6 +528,7 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
         a.X = c->B.XN + (size_t)k * DEL_ROWS_MAX * c->D.d;
         a.W0 = c->lm_head;
         a.x_by_row = 1;
+        TAG(CLS_LMSTACK, 2.0 * c->D.V * c->D.d);
         LAUNCH(launch_rowgemm(EPI_LMHEAD, a, m, c->n_sms, c->st, P));
         const int n_part = rowgemm_lmhead_grid(a.n_items, m, c->n_sms);
         LAUNCH(launch_shadow_reduce(ca, c->up_dev, c->B.LPV, c->B.LPI, n_part, DEL_ROWS_MAX, 1, k * DEL_ROWS_MAX, m, c->st, P));
@@ -481,7 +540,9 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
 
 int read_out(del_ctx *c) {
     CK(cudaMemcpyAsync(c->out_host, c->out_dev, sizeof(del_round_out) * c->D.B, cudaMemcpyDeviceToHost, c->st));
+    c->d2h_bytes += sizeof(del_round_out) * c->D.B;
     CK(cudaStreamSynchronize(c->st));
+    timing_collect(c);
     return DEL_OK;
 }
 
@@ -562,6 +623,7 @@ void del_destroy(del_ctx *c) {
     if (c->up_host) cudaFreeHost(c->up_host);
     if (c->out_host) cudaFreeHost(c->out_host);
     if (c->stage_host) cudaFreeHost(c->stage_host);
+    for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
     delete c;
 }
 
@@ -581,6 +643,7 @@ int del_prefill(del_ctx *c, int sq, const int32_t *prompt, int n_prompt, int max
     int rc = ensure_pages(c, sq, n_prompt + 1);
     if (rc) { release_seq(c, sq); return rc; }
     CK(cudaMemcpyAsync(c->B.PROMPT_ALL, prompt, sizeof(int32_t) * n_prompt, cudaMemcpyHostToDevice, c->st));
+    c->h2d_bytes += sizeof(int32_t) * n_prompt;
     SeqState st0;
     memset(&st0, 0, sizeof(st0));
     memcpy(c->stage_host, &st0, sizeof(st0));
@@ -836,6 +899,24 @@ int del_committed_len(del_ctx *c, int sq) {
 }
 
 int64_t del_launch_count(const del_ctx *c) { return c ? c->launches : 0; }
+
+int del_get_traffic(const del_ctx *c, int64_t *h2d_bytes, int64_t *d2h_bytes) {
+    if (!c) return DEL_EINVAL;
+    if (h2d_bytes) *h2d_bytes = c->h2d_bytes;
+    if (d2h_bytes) *d2h_bytes = c->d2h_bytes;
+    return DEL_OK;
+}
+
+int del_get_kernel_times(del_ctx *c, double *ms, int64_t *launches, double *bytes, int reset) {
+    if (!c) return DEL_EINVAL;
+    for (int i = 0; i < CLS_N; ++i) {
+        if (ms) ms[i] = c->cls_ms[i];
+        if (launches) launches[i] = c->cls_n[i];
+        if (bytes) bytes[i] = c->cls_bytes[i];
+        if (reset) { c->cls_ms[i] = 0; c->cls_n[i] = 0; c->cls_bytes[i] = 0; }
+    }
+    return DEL_OK;
+}
 
 int del_set_flags(del_ctx *c, int flags) {
     if (!c) return DEL_EINVAL;
