@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_kernel(const AttnArgs a
             ri[h] = rv[h] ? rr[h] - rh[h] * ms : 0;
             const bf16 *qp = a.B.Q + (size_t)(seg.row0 + ri[h]) * qdim + (kvh * group + rh[h]) * HD + 8 * t;
 #pragma unroll
-            for (int ks = 0; ks < KS; ++ks) qf[h][ks] = rv[h] ? ldg_act16(qp + 32 * ks) : make_uint4(0, 0, 0, 0);
+            for (int ks = 0; ks < KS; ++ks) qf[h][ks] = ldg_act16_pred(qp + 32 * ks, rv[h]);
         }
         const int rpos[2] = {seg.pos0 + ri[0], seg.pos0 + ri[1]};
         float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};

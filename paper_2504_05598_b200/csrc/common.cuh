@@ -101,6 +101,23 @@ __device__ __forceinline__ uint4 ldg_act16(const void *p) {
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
 }
+// Predicated forms: zero when `pred` is false.  The destination is cleared first and the load itself is
+// predicated, so no select instruction has to wait for the loaded value (which would serialise the
+// software pipeline on the load latency).
+__device__ __forceinline__ uint4 ldg_stream16_pred(const void *p, bool pred) {
+    uint4 v;
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %5, 0;\n\tmov.u32 %0, 0;\n\tmov.u32 %1, 0;\n\tmov.u32 %2, 0;\n\tmov.u32 %3, 0;\n\t"
+                 "@q ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n\t}"
+                 : "=&r"(v.x), "=&r"(v.y), "=&r"(v.z), "=&r"(v.w) : "l"(p), "r"((uint32_t)pred));
+    return v;
+}
+__device__ __forceinline__ uint4 ldg_act16_pred(const void *p, bool pred) {
+    uint4 v;
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %5, 0;\n\tmov.u32 %0, 0;\n\tmov.u32 %1, 0;\n\tmov.u32 %2, 0;\n\tmov.u32 %3, 0;\n\t"
+                 "@q ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];\n\t}"
+                 : "=&r"(v.x), "=&r"(v.y), "=&r"(v.z), "=&r"(v.w) : "l"(p), "r"((uint32_t)pred));
+    return v;
+}
 __device__ __forceinline__ uint2 ldg_act8(const void *p) {
     uint2 v;
     asm volatile("ld.global.cg.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));

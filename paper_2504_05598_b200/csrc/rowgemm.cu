@@ -8,9 +8,10 @@
 // for row g+8 (g = lane/4) at column offset 8*(lane%4): the eight bf16 values feed two m16n8k16 MMAs.
 // The tensor core sums over k, so any permutation of k applied to both operands gives the same
 // product; the activation fragment is therefore loaded with the same 16-byte pattern from the row's
-// bf16 vector, and no shared-memory staging or ldmatrix is needed.  Loads are software-pipelined in two
-// register batches that run ahead across tile boundaries, and the weight loads of the first batches
-// are issued before the kernel waits for its producer (programmatic dependent launch).
+// bf16 vector, and no shared-memory staging or ldmatrix is needed.  Loads are issued in bursts of U
+// k-steps (all loads of a burst before its first MMA); the two resident CTAs per SM overlap each
+// other's bursts, and the first burst of weights is issued before the kernel waits for its producer
+// (programmatic dependent launch).
 // Partial sums of the 8 warps are added in a fixed order through shared memory: results do not depend
 // on the grid size or on how many rows share the pass.
 //
@@ -50,10 +51,9 @@ __device__ __forceinline__ const bf16 *tile_rows(const GemmArgs &a, int item, in
     return a.W0 + (size_t)(16 * item) * a.K;
 }
 
-template <int NT, int D, int EPI>
+template <int NT, int U, int EPI>
 __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_kernel(const GemmArgs a) {
     constexpr int TPI = EpiTraits<EPI>::TPI;
-    constexpr int HB = D / 2;
     constexpr int NC = NT * 8;                      // activation-row columns handled
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float4 *red = reinterpret_cast<float4 *>(smem_raw);                       // [8 warps][NT][32]
@@ -65,56 +65,41 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int K = a.K;
     const int n_ksteps = (K + 31) >> 5;
-    const int nkw = (n_ksteps - warp + 7) >> 3;     // k-steps of this warp per tile (>= 1 since K >= 256)
+    const int nkw = (n_ksteps + 7) >> 3;            // k-steps per warp and tile (the last ones may be empty)
     const int my_items = (a.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     const int my_tiles = my_items * TPI;
-    const int total = my_tiles * nkw;
 
-    uint4 wv[2][HB][2];
-    uint4 xv[2][HB][NT];
-
-    // ---- producer cursors
-    int p_tile = 0, p_ksi = 0;                      // weights
-    const bf16 *p_w = nullptr;
-    auto p_enter_tile = [&]() {
-        if (p_tile < my_tiles) {
-            const int item = blockIdx.x + (p_tile / TPI) * gridDim.x;
-            p_w = tile_rows<EPI>(a, item, p_tile % TPI) + (size_t)g * K + 8 * t;
-        }
-    };
-    p_enter_tile();
-    auto load_w = [&](uint4 (&dst)[2]) {
-        if (p_tile < my_tiles) {
-            const int k0 = ((warp + 8 * p_ksi) << 5) + 8 * t;
-            if (k0 < K) {
-                dst[0] = ldg_stream16(p_w + (k0 - 8 * t));
-                dst[1] = ldg_stream16(p_w + (size_t)8 * K + (k0 - 8 * t));
-            } else {
-                dst[0] = make_uint4(0, 0, 0, 0);
-                dst[1] = make_uint4(0, 0, 0, 0);
-            }
-            if (++p_ksi == nkw) { p_ksi = 0; ++p_tile; p_enter_tile(); }
-        }
-    };
-    // activations: same k sequence, tile-independent
-    int x_units = 0, x_ksi = 0;
+    uint4 wa[U], wb[U];
+    uint4 xv[U][NT];
     const bf16 *xrow[NT];
-    auto load_x = [&](uint4 (&dst)[NT]) {
-        if (x_units < total) {
-            const int k0 = ((warp + 8 * x_ksi) << 5) + 8 * t;
+
+    auto tile_base = [&](int ti) {
+        const int item = blockIdx.x + (ti / TPI) * gridDim.x;
+        return tile_rows<EPI>(a, item, ti % TPI) + (size_t)g * K + 8 * t;
+    };
+    // one burst: U k-steps of this warp, all loads issued before the first use
+    auto load_w = [&](const bf16 *base, int u0) {
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
-                dst[nt] = (xrow[nt] != nullptr && k0 < K) ? ldg_act16(xrow[nt] + k0) : make_uint4(0, 0, 0, 0);
-            if (++x_ksi == nkw) x_ksi = 0;
-            ++x_units;
+        for (int u = 0; u < U; ++u) {
+            const int k0 = (warp + 8 * (u0 + u)) << 5;
+            const bool ok = (u0 + u < nkw) && (k0 + 8 * t < K);
+            wa[u] = ldg_stream16_pred(base + k0, ok);
+            wb[u] = ldg_stream16_pred(base + (size_t)8 * K + k0, ok);
+        }
+    };
+    auto load_x = [&](int u0) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int k0 = ((warp + 8 * (u0 + u)) << 5) + 8 * t;
+            const bool ok = (u0 + u < nkw) && (k0 < K);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) xv[u][nt] = ldg_act16_pred(xrow[nt] + k0, ok && xrow[nt] != nullptr);
         }
     };
 
-    // weights of the first two batches go out before the producer kernel has finished
-#pragma unroll
-    for (int b = 0; b < 2; ++b)
-#pragma unroll
-        for (int j = 0; j < HB; ++j) load_w(wv[b][j]);
+    // the first burst of weights goes out before the producer kernel has finished
+    const bf16 *base = tile_base(0);
+    load_w(base, 0);
     pdl_launch();
     pdl_wait();
 
@@ -133,10 +118,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
             xrow[nt] = a.X + r * (size_t)K;
         }
     }
-#pragma unroll
-    for (int b = 0; b < 2; ++b)
-#pragma unroll
-        for (int j = 0; j < HB; ++j) load_x(xv[b][j]);
+    load_x(0);
 
     // per-row 1/rms from the producer's partial sums of squares
     if (EPI == EPI_QKV || EPI == EPI_GATEUP) {
@@ -161,7 +143,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
 
-    int c_tile = 0, c_ksi = 0, consumed = 0;
+    int c_tile = 0;
 
     auto tile_end = [&]() {
         // fixed-order sum of the 8 warps' partials
@@ -268,26 +250,28 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
         // `res` and `best_*` are next written after the following tile's first barrier
     };
 
-    auto consume = [&](uint4 (&w)[2], uint4 (&x)[NT]) {
-        if (consumed < total) {
+    auto mma_burst = [&]() {
+#pragma unroll
+        for (int u = 0; u < U; ++u)
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-                mma_bf16_16816(acc[nt], w[0].x, w[1].x, w[0].y, w[1].y, x[nt].x, x[nt].y);
-                mma_bf16_16816(acc[nt], w[0].z, w[1].z, w[0].w, w[1].w, x[nt].z, x[nt].w);
+                mma_bf16_16816(acc[nt], wa[u].x, wb[u].x, wa[u].y, wb[u].y, xv[u][nt].x, xv[u][nt].y);
+                mma_bf16_16816(acc[nt], wa[u].z, wb[u].z, wa[u].w, wb[u].w, xv[u][nt].z, xv[u][nt].w);
             }
-            ++consumed;
-            if (++c_ksi == nkw) { c_ksi = 0; tile_end(); ++c_tile; }
-        }
     };
 
-    for (int base = 0; base < total; base += D) {
-#pragma unroll
-        for (int b = 0; b < 2; ++b) {
-#pragma unroll
-            for (int j = 0; j < HB; ++j) consume(wv[b][j], xv[b][j]);
-#pragma unroll
-            for (int j = 0; j < HB; ++j) { load_w(wv[b][j]); load_x(xv[b][j]); }
+    mma_burst();
+    int u0 = U;
+    for (;;) {
+        for (; u0 < nkw; u0 += U) {
+            load_w(base, u0);
+            load_x(u0);
+            mma_burst();
         }
+        tile_end();
+        if (++c_tile == my_tiles) break;
+        base = tile_base(c_tile);
+        u0 = 0;
     }
 
     if (EPI == EPI_LMHEAD) {
@@ -299,7 +283,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     }
 }
 
-template <int NT> constexpr int depth_for() { return NT == 1 ? 8 : 4; }
+template <int NT> constexpr int depth_for() { return NT == 1 ? 8 : (NT == 2 ? 4 : 2); }
 
 template <int NT, int EPI>
 cudaError_t launch_nt(const GemmArgs &a, int grid, cudaStream_t st, bool pdl) {
