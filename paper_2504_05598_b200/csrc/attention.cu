@@ -1,33 +1,39 @@
 // Multi-query decode attention over the paged bf16 KV cache.
 //
-// One CTA = (key-range split, kv head, sequence segment).  The query rows of the segment (its 1..32
-// consecutive positions times the query heads sharing this kv head) form 16-row tiles; keys are walked
-// one 16-token page at a time.  Scores and the P*V product run on bf16 tensor-core MMAs with fp32
-// accumulation; the softmax is the online (running max / running sum) form, its row reductions done
-// with warp shuffles inside the 4-lane groups that own a row.
+// One CTA = (key-range split, kv head, sequence segment), 8 warps.  The query rows of the segment (its
+// 1..32 consecutive positions times the query heads sharing this kv head) form 16-row tiles; the warps
+// are divided among up to 4 query tiles, and the warps of one tile walk the key pages (16 tokens each)
+// of the CTA's key range in a strided fashion.  Scores and the P*V product run on bf16 tensor-core
+// MMAs with fp32 accumulation; the softmax is the online (running max / running sum) form, its row
+// reductions done with warp shuffles inside the 4-lane groups that own a row.
 //
 // Fragment loading without shared memory: the MMA sums over its k index, so any permutation of k used
 // for both operands is allowed.  For Q*K^T a thread loads 16 contiguous bytes of a key row (and the
 // same bytes of the query row) and feeds them to two MMAs.  For P*V the page stores V transposed
 // ([head_dim][16 tokens]); the score tile's columns are assigned to tokens such that a thread's four
-// probabilities belong to tokens 4t..4t+3, which are 8 contiguous bytes of a V^T row.
+// probabilities belong to tokens 4t..4t+3, which are 8 contiguous bytes of a V^T row.  The page ids of
+// a warp are fetched up front, and all loads of a page (keys and values) are issued before their
+// first use.
 //
-// Splits write (max, sum, unnormalised output) partials; the last CTA to arrive for a (segment, kv
-// head) merges them in split order, so the result does not depend on scheduling.
+// The warps of a query tile merge their (max, sum, output) states through shared memory, every warp
+// of the CTA merging a slice of the output columns.  With one split the result is final; otherwise
+// splits write partials and the last CTA to arrive for a (segment, kv head) merges them in split
+// order, so the result does not depend on scheduling.
 #include "kernels.h"
 
 namespace {
 
-constexpr int ATT_THREADS = 128;
 constexpr float LOG2E = 1.4426950408889634f;
+constexpr int NW = 8;                 // warps per CTA
+constexpr int PG = 4;                 // page ids fetched ahead per warp
 
 template <int HD>
-__global__ void __launch_bounds__(ATT_THREADS) attention_kernel(const AttnArgs a) {
+__global__ void __launch_bounds__(NW * 32) attention_kernel(const AttnArgs a) {
     constexpr int KS = HD / 32;       // 16-byte chunks per thread along head_dim
     constexpr int NJ = HD / 8;        // output n-tiles
     extern __shared__ __align__(16) float sm[];
-    float *sm_o = sm;                               // [4][32][NJ*4]
-    float *sm_ml = sm + 4 * 32 * NJ * 4;            // [4][32][4]
+    float *sm_o = sm;                               // [NW][32][NJ*4]
+    float *sm_ml = sm + NW * 32 * NJ * 4;           // [NW][32][4]
     __shared__ int s_last;
 
     pdl_launch();
@@ -43,23 +49,26 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_kernel(const AttnArgs a
     const int n_pages = (kv_len + 15) >> 4;
     const int pps = (n_pages + n_splits - 1) / n_splits;
     const int p_begin = split * pps, p_end = min(n_pages, p_begin + pps);
-    const int P = n_mt >= 4 ? 4 : (n_mt >= 2 ? (n_mt == 2 ? 2 : 4) : 1);
-    const int n_kl = 4 / P, kl = warp / P;
+    const int P = n_mt >= 3 ? 4 : n_mt;             // query tiles handled concurrently: 1, 2 or 4
+    const int n_kl = NW / P, kl = warp / P;
     const float sc = rsqrtf((float)HD) * LOG2E;
     const int32_t *pt = a.B.PT + seg.seq * a.D.pages_per_seq;
     const size_t page_stride = (size_t)a.D.L * a.D.nkv * 16 * HD;
     const size_t head_off = ((size_t)(a.layer - 1) * a.D.nkv + kvh) * 16 * HD;
     const int qdim = a.D.nh * HD;
+    const int n_iter = (n_mt + P - 1) / P;
+    const int key0 = 4 * (g >> 1) + (g & 1);        // token of score-tile 0 column g; tile 1: +2
 
-    for (int mt = warp % P; mt < n_mt; mt += P) {
+    for (int it = 0; it < n_iter; ++it) {
+        const int mt = it * P + warp % P;
         // rows of this thread: rr0 = mt*16+g, rr1 = rr0+8, ordered head-major: rr = hq*ms + i
-        int rr[2] = {mt * 16 + g, mt * 16 + g + 8};
+        const int rr[2] = {mt * 16 + g, mt * 16 + g + 8};
         int ri[2], rh[2];
         bool rv[2];
         uint4 qf[2][KS];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
-            rv[h] = rr[h] < R;
+            rv[h] = mt < n_mt && rr[h] < R;
             rh[h] = rv[h] ? rr[h] / ms : 0;
             ri[h] = rv[h] ? rr[h] - rh[h] * ms : 0;
             const bf16 *qp = a.B.Q + (size_t)(seg.row0 + ri[h]) * qdim + (kvh * group + rh[h]) * HD + 8 * t;
@@ -72,54 +81,65 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_kernel(const AttnArgs a
 #pragma unroll
         for (int j = 0; j < NJ; ++j) O[j][0] = O[j][1] = O[j][2] = O[j][3] = 0.f;
 
-        for (int p = p_begin + kl; p < p_end; p += n_kl) {
-            const int pg = pt[p];
-            const bf16 *kpage = a.B.KP + (size_t)pg * page_stride + head_off;
-            const bf16 *vpage = a.B.VP + (size_t)pg * page_stride + head_off;
-            const int key0 = 4 * (g >> 1) + (g & 1);       // token of score-tile 0 column g; tile 1: +2
-            uint4 kf[2][KS];
+        if (mt < n_mt) {
+            for (int pb = p_begin + kl; pb < p_end; pb += n_kl * PG) {
+                int pgs[PG];
 #pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                kf[0][ks] = ldg_act16(kpage + key0 * HD + 32 * ks + 8 * t);
-                kf[1][ks] = ldg_act16(kpage + (key0 + 2) * HD + 32 * ks + 8 * t);
-            }
-            float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int q = 0; q < PG; ++q) {
+                    const int p = pb + q * n_kl;
+                    pgs[q] = p < p_end ? pt[p] : 0;
+                }
 #pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                mma_bf16_16816(s0, qf[0][ks].x, qf[1][ks].x, qf[0][ks].y, qf[1][ks].y, kf[0][ks].x, kf[0][ks].y);
-                mma_bf16_16816(s0, qf[0][ks].z, qf[1][ks].z, qf[0][ks].w, qf[1][ks].w, kf[0][ks].z, kf[0][ks].w);
-                mma_bf16_16816(s1, qf[0][ks].x, qf[1][ks].x, qf[0][ks].y, qf[1][ks].y, kf[1][ks].x, kf[1][ks].y);
-                mma_bf16_16816(s1, qf[0][ks].z, qf[1][ks].z, qf[0][ks].w, qf[1][ks].w, kf[1][ks].z, kf[1][ks].w);
-            }
-            // this thread's scores: tokens 4t, 4t+1 (s0) and 4t+2, 4t+3 (s1) of the page, rows g / g+8
-            const int tok0 = p * 16 + 4 * t;
-            float pr[2][4];
+                for (int q = 0; q < PG; ++q) {
+                    const int p = pb + q * n_kl;
+                    if (p >= p_end) break;
+                    const bf16 *kpage = a.B.KP + (size_t)pgs[q] * page_stride + head_off;
+                    const bf16 *vpage = a.B.VP + (size_t)pgs[q] * page_stride + head_off;
+                    uint4 kf[2][KS];
+                    uint2 vf[NJ];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                float v[4] = {s0[2 * h] * sc, s0[2 * h + 1] * sc, s1[2 * h] * sc, s1[2 * h + 1] * sc};
+                    for (int ks = 0; ks < KS; ++ks) {
+                        kf[0][ks] = ldg_act16(kpage + key0 * HD + 32 * ks + 8 * t);
+                        kf[1][ks] = ldg_act16(kpage + (key0 + 2) * HD + 32 * ks + 8 * t);
+                    }
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (!rv[h] || tok0 + e > rpos[h]) v[e] = -INFINITY;
-                float mx = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3]));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float m_new = fmaxf(m_run[h], mx);
-                const float base = (m_new == -INFINITY) ? 0.f : m_new;
-                const float alpha = exp2f(m_run[h] - base);
-                m_run[h] = m_new;
-                float psum = 0.f;
+                    for (int j = 0; j < NJ; ++j) vf[j] = ldg_act8(vpage + (8 * j + g) * 16 + 4 * t);
+                    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int e = 0; e < 4; ++e) { pr[h][e] = exp2f(v[e] - base); psum += pr[h][e]; }
-                l_run[h] = l_run[h] * alpha + psum;
+                    for (int ks = 0; ks < KS; ++ks) {
+                        mma_bf16_16816(s0, qf[0][ks].x, qf[1][ks].x, qf[0][ks].y, qf[1][ks].y, kf[0][ks].x, kf[0][ks].y);
+                        mma_bf16_16816(s0, qf[0][ks].z, qf[1][ks].z, qf[0][ks].w, qf[1][ks].w, kf[0][ks].z, kf[0][ks].w);
+                        mma_bf16_16816(s1, qf[0][ks].x, qf[1][ks].x, qf[0][ks].y, qf[1][ks].y, kf[1][ks].x, kf[1][ks].y);
+                        mma_bf16_16816(s1, qf[0][ks].z, qf[1][ks].z, qf[0][ks].w, qf[1][ks].w, kf[1][ks].z, kf[1][ks].w);
+                    }
+                    // this thread's scores: tokens 4t, 4t+1 (s0) and 4t+2, 4t+3 (s1) of the page, rows g / g+8
+                    const int tok0 = p * 16 + 4 * t;
+                    float pr[2][4];
 #pragma unroll
-                for (int j = 0; j < NJ; ++j) { O[j][2 * h] *= alpha; O[j][2 * h + 1] *= alpha; }
-            }
-            const uint32_t pa0 = pack_bf16(pr[0][0], pr[0][1]), pa1 = pack_bf16(pr[1][0], pr[1][1]);
-            const uint32_t pa2 = pack_bf16(pr[0][2], pr[0][3]), pa3 = pack_bf16(pr[1][2], pr[1][3]);
+                    for (int h = 0; h < 2; ++h) {
+                        float v[4] = {s0[2 * h] * sc, s0[2 * h + 1] * sc, s1[2 * h] * sc, s1[2 * h + 1] * sc};
 #pragma unroll
-            for (int j = 0; j < NJ; ++j) {
-                const uint2 vf = ldg_act8(vpage + (8 * j + g) * 16 + 4 * t);
-                mma_bf16_16816(O[j], pa0, pa1, pa2, pa3, vf.x, vf.y);
+                        for (int e = 0; e < 4; ++e)
+                            if (!rv[h] || tok0 + e > rpos[h]) v[e] = -INFINITY;
+                        float mx = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3]));
+                        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                        const float m_new = fmaxf(m_run[h], mx);
+                        const float base = (m_new == -INFINITY) ? 0.f : m_new;
+                        const float alpha = exp2f(m_run[h] - base);
+                        m_run[h] = m_new;
+                        float psum = 0.f;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) { pr[h][e] = exp2f(v[e] - base); psum += pr[h][e]; }
+                        l_run[h] = l_run[h] * alpha + psum;
+#pragma unroll
+                        for (int j = 0; j < NJ; ++j) { O[j][2 * h] *= alpha; O[j][2 * h + 1] *= alpha; }
+                    }
+                    const uint32_t pa0 = pack_bf16(pr[0][0], pr[0][1]), pa1 = pack_bf16(pr[1][0], pr[1][1]);
+                    const uint32_t pa2 = pack_bf16(pr[0][2], pr[0][3]), pa3 = pack_bf16(pr[1][2], pr[1][3]);
+#pragma unroll
+                    for (int j = 0; j < NJ; ++j) mma_bf16_16816(O[j], pa0, pa1, pa2, pa3, vf[j].x, vf[j].y);
+                }
             }
         }
 #pragma unroll
@@ -128,59 +148,55 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_kernel(const AttnArgs a
             l_run[h] += __shfl_xor_sync(0xffffffffu, l_run[h], 2);
         }
 
-        if (n_kl > 1) {          // warps that share this query tile merge through shared memory
-            float *so = sm_o + (size_t)(warp * 32 + lane) * NJ * 4;
+        // ---- merge the warps of each query tile; every warp merges some output column tiles
+        {
+            // layout [column tile][warp][lane]: consecutive lanes write consecutive 16-byte words
 #pragma unroll
-            for (int j = 0; j < NJ; ++j) *reinterpret_cast<float4 *>(so + 4 * j) = make_float4(O[j][0], O[j][1], O[j][2], O[j][3]);
+            for (int j = 0; j < NJ; ++j)
+                *reinterpret_cast<float4 *>(sm_o + (size_t)((j * NW + warp) * 32 + lane) * 4) = make_float4(O[j][0], O[j][1], O[j][2], O[j][3]);
             *reinterpret_cast<float4 *>(sm_ml + (warp * 32 + lane) * 4) = make_float4(m_run[0], l_run[0], m_run[1], l_run[1]);
-            __syncthreads();
-            if (kl == 0) {
-                float M[2] = {m_run[0], m_run[1]};
-                for (int k2 = 1; k2 < n_kl; ++k2) {
-                    const float4 ml = *reinterpret_cast<float4 *>(sm_ml + ((warp + k2 * P) * 32 + lane) * 4);
-                    M[0] = fmaxf(M[0], ml.x);
-                    M[1] = fmaxf(M[1], ml.z);
-                }
-                const float b0 = M[0] == -INFINITY ? 0.f : M[0], b1 = M[1] == -INFINITY ? 0.f : M[1];
-                float f0 = exp2f(m_run[0] - b0), f1 = exp2f(m_run[1] - b1);
-                l_run[0] *= f0; l_run[1] *= f1;
-#pragma unroll
-                for (int j = 0; j < NJ; ++j) { O[j][0] *= f0; O[j][1] *= f0; O[j][2] *= f1; O[j][3] *= f1; }
-                for (int k2 = 1; k2 < n_kl; ++k2) {
-                    const int w2 = warp + k2 * P;
-                    const float4 ml = *reinterpret_cast<float4 *>(sm_ml + (w2 * 32 + lane) * 4);
-                    f0 = exp2f(ml.x - b0); f1 = exp2f(ml.z - b1);
-                    l_run[0] += ml.y * f0; l_run[1] += ml.w * f1;
-                    const float *so2 = sm_o + (size_t)(w2 * 32 + lane) * NJ * 4;
-#pragma unroll
-                    for (int j = 0; j < NJ; ++j) {
-                        const float4 o2 = *reinterpret_cast<const float4 *>(so2 + 4 * j);
-                        O[j][0] += o2.x * f0; O[j][1] += o2.y * f0; O[j][2] += o2.z * f1; O[j][3] += o2.w * f1;
-                    }
-                }
-                m_run[0] = M[0]; m_run[1] = M[1];
-            }
         }
-        if (kl == 0) {
+        __syncthreads();
+        for (int task = warp; task < P * NJ; task += NW) {
+            const int mp = task / NJ, j = task - mp * NJ;      // query-tile slot of this iteration, column tile
+            const int mt2 = it * P + mp;
+            if (mt2 >= n_mt) continue;
+            float M0 = -INFINITY, M1 = -INFINITY;
+            for (int k2 = 0; k2 < n_kl; ++k2) {
+                const float4 ml = *reinterpret_cast<const float4 *>(sm_ml + ((mp + k2 * P) * 32 + lane) * 4);
+                M0 = fmaxf(M0, ml.x);
+                M1 = fmaxf(M1, ml.z);
+            }
+            const float b0 = M0 == -INFINITY ? 0.f : M0, b1 = M1 == -INFINITY ? 0.f : M1;
+            float L0 = 0.f, L1 = 0.f, o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;
+            for (int k2 = 0; k2 < n_kl; ++k2) {
+                const int w2 = mp + k2 * P;
+                const float4 ml = *reinterpret_cast<const float4 *>(sm_ml + (w2 * 32 + lane) * 4);
+                const float f0 = exp2f(ml.x - b0), f1 = exp2f(ml.z - b1);
+                L0 += ml.y * f0;
+                L1 += ml.w * f1;
+                const float4 ov = *reinterpret_cast<const float4 *>(sm_o + (size_t)((j * NW + w2) * 32 + lane) * 4);
+                o0 += ov.x * f0; o1 += ov.y * f0; o2 += ov.z * f1; o3 += ov.w * f1;
+            }
+            const float Mv[2] = {M0, M1}, Lv[2] = {L0, L1}, ov2[2][2] = {{o0, o1}, {o2, o3}};
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                if (!rv[h]) continue;
-                const int c = seg.row0 + ri[h], qh = kvh * group + rh[h];
+                const int r2 = mt2 * 16 + g + 8 * h;
+                if (r2 >= R) continue;
+                const int hq = r2 / ms, i = r2 - hq * ms;
+                const int c = seg.row0 + i, qh = kvh * group + hq;
                 if (n_splits == 1) {
-                    const float inv = 1.f / l_run[h];
-                    bf16 *op = a.B.ATT + (size_t)c * qdim + qh * HD + 2 * t;
-#pragma unroll
-                    for (int j = 0; j < NJ; ++j)
-                        *reinterpret_cast<uint32_t *>(op + 8 * j) = pack_bf16(O[j][2 * h] * inv, O[j][2 * h + 1] * inv);
+                    const float inv = 1.f / Lv[h];
+                    *reinterpret_cast<uint32_t *>(a.B.ATT + (size_t)c * qdim + qh * HD + 8 * j + 2 * t) =
+                        pack_bf16(ov2[h][0] * inv, ov2[h][1] * inv);
                 } else {
                     const size_t pi = ((size_t)c * a.D.nh + qh) * n_splits + split;
-                    float *op = a.B.APO + pi * HD + 2 * t;
-#pragma unroll
-                    for (int j = 0; j < NJ; ++j) *reinterpret_cast<float2 *>(op + 8 * j) = make_float2(O[j][2 * h], O[j][2 * h + 1]);
-                    if (t == 0) *reinterpret_cast<float2 *>(a.B.APML + pi * 2) = make_float2(m_run[h], l_run[h]);
+                    *reinterpret_cast<float2 *>(a.B.APO + pi * HD + 8 * j + 2 * t) = make_float2(ov2[h][0], ov2[h][1]);
+                    if (j == 0 && t == 0) *reinterpret_cast<float2 *>(a.B.APML + pi * 2) = make_float2(Mv[h], Lv[h]);
                 }
             }
         }
+        __syncthreads();
     }
 
     if (n_splits > 1) {
@@ -195,20 +211,33 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_kernel(const AttnArgs a
         if (s_last) {
             __threadfence();
             // merge the splits of every (row, head) of this kv head in split order
-            for (int e = tid; e < R * (HD / 4); e += ATT_THREADS) {
+            for (int e = tid; e < R * (HD / 4); e += NW * 32) {
                 const int row = e / (HD / 4), d4 = (e - row * (HD / 4)) * 4;
                 const int hq = row / ms, i = row - hq * ms;
                 const int c = seg.row0 + i, qh = kvh * group + hq;
                 const size_t pi = ((size_t)c * a.D.nh + qh) * n_splits;
+                // all loads first (n_splits <= 16), then the arithmetic: two memory latencies in total
+                uint2 mlv[16];
+                uint4 ovv[16];
+#pragma unroll
+                for (int s = 0; s < 16; ++s) {
+                    const int se = s < n_splits ? s : n_splits - 1;        // clamped: unused slots are masked below
+                    mlv[s] = ldg_act8(a.B.APML + (pi + se) * 2);
+                    ovv[s] = ldg_act16(a.B.APO + (pi + se) * HD + d4);
+                }
                 float M = -INFINITY;
-                for (int s = 0; s < n_splits; ++s) M = fmaxf(M, ldg_cg_f32(a.B.APML + (pi + s) * 2));
+#pragma unroll
+                for (int s = 0; s < 16; ++s) {
+                    if (s >= n_splits) mlv[s].x = 0xff800000u;              // -inf: weight 0
+                    M = fmaxf(M, __uint_as_float(mlv[s].x));
+                }
                 float l = 0.f, o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;
-                for (int s = 0; s < n_splits; ++s) {
-                    const float f = exp2f(ldg_cg_f32(a.B.APML + (pi + s) * 2) - M);
-                    l += f * ldg_cg_f32(a.B.APML + (pi + s) * 2 + 1);
-                    const float *op = a.B.APO + (pi + s) * HD + d4;
-                    o0 += f * ldg_cg_f32(op); o1 += f * ldg_cg_f32(op + 1);
-                    o2 += f * ldg_cg_f32(op + 2); o3 += f * ldg_cg_f32(op + 3);
+#pragma unroll
+                for (int s = 0; s < 16; ++s) {
+                    const float f = exp2f(__uint_as_float(mlv[s].x) - M);
+                    l += f * __uint_as_float(mlv[s].y);
+                    o0 += f * __uint_as_float(ovv[s].x); o1 += f * __uint_as_float(ovv[s].y);
+                    o2 += f * __uint_as_float(ovv[s].z); o3 += f * __uint_as_float(ovv[s].w);
                 }
                 const float inv = 1.f / l;
                 uint2 pk;
@@ -220,14 +249,19 @@ __global__ void __launch_bounds__(ATT_THREADS) attention_kernel(const AttnArgs a
     }
 }
 
-}  // namespace
-
-cudaError_t launch_attention(const AttnArgs &a, int n_seg, cudaStream_t st, bool pdl) {
-    const int HD = a.D.hd;
-    const size_t smem = sizeof(float) * (4 * 32 * (HD / 8) * 4 + 4 * 32 * 4);
+template <int HD>
+cudaError_t launch_one(const AttnArgs &a, int n_seg, cudaStream_t st, bool pdl) {
+    const size_t smem = sizeof(float) * ((size_t)NW * 32 * (HD / 8) * 4 + (size_t)NW * 32 * 4);
+    auto kern = attention_kernel<HD>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(a.n_splits, a.D.nkv, n_seg);
-    cfg.blockDim = dim3(ATT_THREADS);
+    cfg.blockDim = dim3(NW * 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute at[1];
@@ -235,15 +269,26 @@ cudaError_t launch_attention(const AttnArgs &a, int n_seg, cudaStream_t st, bool
     at[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = at;
     cfg.numAttrs = pdl ? 1 : 0;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
-        if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
-    if (HD == 128) return cudaLaunchKernelEx(&cfg, attention_kernel<128>, a);
-    if (HD == 64) return cudaLaunchKernelEx(&cfg, attention_kernel<64>, a);
+    return cudaLaunchKernelEx(&cfg, kern, a);
+}
+
+}  // namespace
+
+// Key-range splits for a pass whose longest sequence holds `pages` pages, with `n_units` (segment, kv
+// head) pairs and query tiles processed `tiles_par` at a time (so 8 / tiles_par warps walk the pages).
+int attention_splits(int pages, int n_units, int tiles_par, int n_sms) {
+    const int lanes = NW / tiles_par;
+    const int per_warp = (pages + lanes - 1) / lanes;   // pages a warp walks if the key range is not split
+    if (per_warp <= 2) return 1;                        // one or two page latencies, no cross-CTA merge
+    // the kernel keeps one CTA per SM resident: stay within one wave, aim at two pages per warp
+    int ns = (per_warp + 1) / 2;
+    const int one_wave = n_sms / n_units;
+    if (ns > one_wave) ns = one_wave;
+    return ns > 16 ? 16 : (ns < 1 ? 1 : ns);
+}
+
+cudaError_t launch_attention(const AttnArgs &a, int n_seg, cudaStream_t st, bool pdl) {
+    if (a.D.hd == 128) return launch_one<128>(a, n_seg, st, pdl);
+    if (a.D.hd == 64) return launch_one<64>(a, n_seg, st, pdl);
     return cudaErrorInvalidValue;
 }

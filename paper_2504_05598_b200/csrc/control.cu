@@ -9,24 +9,41 @@ namespace {
 constexpr int CTL_THREADS = 256;
 
 __device__ __forceinline__ void write_embedding(const CtlArgs &a, int token, int seq, int slot) {
-    // h^0 = embedding row; also the bf16 input of layer 1's attention norm and its partial sums of squares
+    // h^0 = embedding row; also the bf16 input of layer 1's attention norm and its partial sums of squares.
+    // A thread owns 8 consecutive features; two neighbouring threads make one 16-feature partial.
     const int d = a.D.d;
     const bf16 *e = a.tok_emb + (size_t)token * d;
     const size_t sr = stack_row(a.D, 0, seq, slot);
-    for (int o0 = 0; o0 < d; o0 += CTL_THREADS) {
-        const int o = o0 + threadIdx.x;
-        float h = 0.f;
-        if (o < d) {
-            h = bf16_to_f(e[o]);
-            a.B.H[sr * d + o] = h;
-            a.B.XS[sr * d + o] = __float2bfloat16_rn(h * bf16_to_f(a.gain0[o]));
+    for (int o0 = 0; o0 < d; o0 += 2 * 8 * CTL_THREADS) {
+        uint4 ev[2], gv[2];
+        int o[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            o[r] = o0 + (r * CTL_THREADS + threadIdx.x) * 8;
+            ev[r] = ldg_stream16_pred(e + o[r], o[r] < d);
+            gv[r] = ldg_stream16_pred(a.gain0 + o[r], o[r] < d);
         }
-        float ss = h * h;
-        ss += __shfl_xor_sync(0xffffffffu, ss, 8);
-        ss += __shfl_xor_sync(0xffffffffu, ss, 4);
-        ss += __shfl_xor_sync(0xffffffffu, ss, 2);
-        ss += __shfl_xor_sync(0xffffffffu, ss, 1);
-        if (o < d && (o & 15) == 0) a.B.SS[sr * a.D.n_sst + (o >> 4)] = ss;
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const uint32_t ew[4] = {ev[r].x, ev[r].y, ev[r].z, ev[r].w}, gw[4] = {gv[r].x, gv[r].y, gv[r].z, gv[r].w};
+            float h[8], ss = 0.f;
+            uint32_t xs[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                h[2 * q] = __uint_as_float(ew[q] << 16);
+                h[2 * q + 1] = __uint_as_float(ew[q] & 0xffff0000u);
+                xs[q] = pack_bf16(h[2 * q] * __uint_as_float(gw[q] << 16), h[2 * q + 1] * __uint_as_float(gw[q] & 0xffff0000u));
+                ss += h[2 * q] * h[2 * q] + h[2 * q + 1] * h[2 * q + 1];
+            }
+            ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+            if (o[r] < d) {
+                float4 *hp = reinterpret_cast<float4 *>(a.B.H + sr * d + o[r]);
+                hp[0] = make_float4(h[0], h[1], h[2], h[3]);
+                hp[1] = make_float4(h[4], h[5], h[6], h[7]);
+                *reinterpret_cast<uint4 *>(a.B.XS + sr * d + o[r]) = make_uint4(xs[0], xs[1], xs[2], xs[3]);
+                if ((threadIdx.x & 1) == 0) a.B.SS[sr * a.D.n_sst + (o[r] >> 4)] = ss;
+            }
+        }
     }
 }
 

@@ -324,8 +324,8 @@ int run_layer(del_ctx *c, const PassInfo &pi, int l, bool write_exit) {
         memset(&a, 0, sizeof(a));
         a.D = D; a.B = c->B; a.plan = c->plan_dev + pi.plan_idx; a.layer = l;
         const int pages = (pi.max_kv + 15) / 16;
-        int ns = (2 * c->n_sms + pi.n_seg * D.nkv - 1) / (pi.n_seg * D.nkv);
-        ns = std::max(1, std::min(std::min(ns, 16), (pages + 1) / 2));
+        const int R = pi.max_rows * (D.nh / D.nkv), n_mt = (R + 15) / 16;
+        const int ns = attention_splits(pages, pi.n_seg * D.nkv, n_mt >= 3 ? 4 : n_mt, c->n_sms);
         a.n_splits = ns;
         a.max_rows = pi.max_rows;
         {

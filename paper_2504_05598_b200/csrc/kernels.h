@@ -30,6 +30,7 @@ struct AttnArgs {
     int32_t max_rows;          // largest segment (rows), decides the number of query tiles
 };
 cudaError_t launch_attention(const AttnArgs &a, int n_seg, cudaStream_t st, bool pdl);
+int attention_splits(int pages, int n_units, int tiles_par, int n_sms);
 
 // control kernels
 struct CtlArgs {

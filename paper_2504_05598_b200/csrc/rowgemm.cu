@@ -78,20 +78,20 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
         return tile_rows<EPI>(a, item, ti % TPI) + (size_t)g * K + 8 * t;
     };
     // one burst: U k-steps of this warp, all loads issued before the first use
-    auto load_w = [&](const bf16 *base, int u0) {
+    auto load_w = [&](const bf16 *base, int u0, bool live) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int k0 = (warp + 8 * (u0 + u)) << 5;
-            const bool ok = (u0 + u < nkw) && (k0 + 8 * t < K);
+            const bool ok = live && (u0 + u < nkw) && (k0 + 8 * t < K);
             wa[u] = ldg_stream16_pred(base + k0, ok);
             wb[u] = ldg_stream16_pred(base + (size_t)8 * K + k0, ok);
         }
     };
-    auto load_x = [&](int u0) {
+    auto load_x = [&](int u0, bool live) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int k0 = ((warp + 8 * (u0 + u)) << 5) + 8 * t;
-            const bool ok = (u0 + u < nkw) && (k0 < K);
+            const bool ok = live && (u0 + u < nkw) && (k0 < K);
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) xv[u][nt] = ldg_act16_pred(xrow[nt] + k0, ok && xrow[nt] != nullptr);
         }
@@ -99,7 +99,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
 
     // the first burst of weights goes out before the producer kernel has finished
     const bf16 *base = tile_base(0);
-    load_w(base, 0);
+    load_w(base, 0, true);
     pdl_launch();
     pdl_wait();
 
@@ -118,7 +118,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
             xrow[nt] = a.X + r * (size_t)K;
         }
     }
-    load_x(0);
+    load_x(0, true);
 
     // per-row 1/rms from the producer's partial sums of squares
     if (EPI == EPI_QKV || EPI == EPI_GATEUP) {
@@ -264,14 +264,20 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     int u0 = U;
     for (;;) {
         for (; u0 < nkw; u0 += U) {
-            load_w(base, u0);
-            load_x(u0);
+            load_w(base, u0, true);
+            load_x(u0, true);
             mma_burst();
         }
+        // the next tile's first burst is in flight while this tile is reduced and written out
+        const bool more = c_tile + 1 < my_tiles;
+        if (more) base = tile_base(c_tile + 1);
+        load_w(base, 0, more);
+        load_x(0, more);
         tile_end();
-        if (++c_tile == my_tiles) break;
-        base = tile_base(c_tile);
-        u0 = 0;
+        if (!more) break;
+        ++c_tile;
+        mma_burst();
+        u0 = U;
     }
 
     if (EPI == EPI_LMHEAD) {
