@@ -922,6 +922,7 @@ int del_set_flags(del_ctx *c, int flags) {
     if (!c) return DEL_EINVAL;
     const int old = c->flags;
     c->flags = flags;
+    rowgemm_set_ctas_per_sm((flags & 16) ? 1 : 2);
     return old;
 }
 

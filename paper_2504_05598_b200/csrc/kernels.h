@@ -20,6 +20,7 @@ struct GemmArgs {
 
 cudaError_t launch_rowgemm(int epi, const GemmArgs &a, int m, int n_sms, cudaStream_t st, bool pdl);
 int rowgemm_lmhead_grid(int n_items, int m, int n_sms);
+void rowgemm_set_ctas_per_sm(int n);
 
 struct AttnArgs {
     Dims D;

@@ -317,11 +317,13 @@ cudaError_t launch_nt(const GemmArgs &a, int grid, cudaStream_t st, bool pdl) {
     return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
+int g_cta_per_sm = 2;
+
 template <int EPI>
 cudaError_t launch_epi(const GemmArgs &a, int m, int n_sms, cudaStream_t st, bool pdl) {
     const int nt = (m + 7) / 8;
-    if (nt <= 1) return launch_nt<1, EPI>(a, min(a.n_items, 2 * n_sms), st, pdl);
-    if (nt <= 2) return launch_nt<2, EPI>(a, min(a.n_items, 2 * n_sms), st, pdl);
+    if (nt <= 1) return launch_nt<1, EPI>(a, min(a.n_items, g_cta_per_sm * n_sms), st, pdl);
+    if (nt <= 2) return launch_nt<2, EPI>(a, min(a.n_items, g_cta_per_sm * n_sms), st, pdl);
     if (nt <= 4) return launch_nt<4, EPI>(a, min(a.n_items, n_sms), st, pdl);
     return launch_nt<8, EPI>(a, min(a.n_items, n_sms), st, pdl);
 }
@@ -339,8 +341,10 @@ cudaError_t launch_rowgemm(int epi, const GemmArgs &a, int m, int n_sms, cudaStr
     return cudaErrorInvalidValue;
 }
 
+void rowgemm_set_ctas_per_sm(int n) { g_cta_per_sm = n < 1 ? 1 : (n > 2 ? 2 : n); }
+
 int rowgemm_lmhead_grid(int n_items, int m, int n_sms) {
     const int nt = (m + 7) / 8;
-    const int cap = nt <= 2 ? 2 * n_sms : n_sms;
+    const int cap = nt <= 2 ? g_cta_per_sm * n_sms : n_sms;
     return n_items < cap ? n_items : cap;
 }
