@@ -253,12 +253,12 @@ def run_ours(a):
     prefill_all()
     for _ in range(3):
         ctx.round()
-    ctx.set_flags(dl.FLAG_PDL | dl.FLAG_TIMING)
+    ctx.set_flags(dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_TIMING)
     ctx.kernel_times(reset=True)
     for _ in range(min(K, 24)):
         ctx.round()
     kt = ctx.kernel_times(reset=True)
-    ctx.set_flags(dl.FLAG_PDL)
+    ctx.set_flags(dl.FLAG_PDL | dl.FLAG_TC)
     peak, peak_kind = measured_peaks()
     kernels = {}
     for name, v in kt.items():

@@ -48,7 +48,7 @@ struct del_ctx {
     std::vector<const bf16 *> attn_norm, wq, wk, wv, wo, ffn_norm, w_gate, w_up, w_down;
     cudaStream_t st = nullptr;
     int n_sms = 148;
-    int flags = FLAG_PDL;
+    int flags = FLAG_PDL | FLAG_TC;
     SeqHost seq[DEL_SEQ_MAX];
     std::vector<int> free_pages;
     std::vector<int32_t> pt_host;
@@ -59,6 +59,8 @@ struct del_ctx {
     del_round_out *out_host = nullptr, *out_dev = nullptr; // [B]
     void *stage_host = nullptr;                            // small pinned scratch
     float *dbg_dev = nullptr;                              // [V] debug logits / kv rows
+    alignas(64) unsigned char map_x[128], map_w[128];     // tensor maps of the stacked rows and of W_lm
+    bool tc_ok = false;
     int64_t launches = 0, h2d_bytes = 0, d2h_bytes = 0;
     // optional per-launch timing (FLAG_TIMING): events around every launch, summed per kernel class
     struct TimeRec { int cls, ev; double bytes; };
@@ -507,6 +509,16 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
     ca.mode = mode;
     ca.n_rows = rows;
     LAUNCH(launch_prep_rows(ca, c->up_dev, rows, c->st, P));
+    if ((c->flags & FLAG_TC) && c->tc_ok) {
+        // one pass over W_lm on the tensor cores, arg-max fused; partials [row][vocabulary tile]
+        const int nvt = lmhead_tc_vtiles(c->D.V);
+        TAG(CLS_LMSTACK, 2.0 * c->D.V * c->D.d);
+        LAUNCH(launch_lmhead_tc(c->map_x, c->map_w, c->B.TPV, c->B.TPI, rows, c->D.V, c->D.d, c->B.ERR, c->n_sms, c->st, P));
+        LAUNCH(launch_shadow_reduce(ca, c->up_dev, c->B.TPV, c->B.TPI, nvt, 1, nvt, 0, rows, c->st, P));
+        LAUNCH(launch_update(ca, c->up_dev, c->out_dev, up->n_seq, c->st, P));
+        if (do_select) LAUNCH(launch_select(ca, c->up_dev, c->out_dev, up->n_seq, c->st, P));
+        return DEL_OK;
+    }
     // streaming LM head in chunks of 64 stacked rows
     const int n_chunks = (rows + DEL_ROWS_MAX - 1) / DEL_ROWS_MAX;
     int rc = plan_begin(c, n_chunks);
@@ -541,8 +553,16 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
 int read_out(del_ctx *c) {
     CK(cudaMemcpyAsync(c->out_host, c->out_dev, sizeof(del_round_out) * c->D.B, cudaMemcpyDeviceToHost, c->st));
     c->d2h_bytes += sizeof(del_round_out) * c->D.B;
+    int32_t *err_host = reinterpret_cast<int32_t *>(c->stage_host) + 1024;
+    CK(cudaMemcpyAsync(err_host, c->B.ERR, sizeof(int32_t), cudaMemcpyDeviceToHost, c->st));
     CK(cudaStreamSynchronize(c->st));
     timing_collect(c);
+    if (*err_host != 0) {
+        // a bounded device-side wait expired; clear the word so that the context stays usable
+        snprintf(c->err, sizeof(c->err), "device wait expired (code %d)", *err_host);
+        cudaMemsetAsync(c->B.ERR, 0, sizeof(int32_t), c->st);
+        return DEL_ETIMEOUT;
+    }
     return DEL_OK;
 }
 
@@ -611,6 +631,9 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
         del_destroy(c);
         return DEL_ECUDA;
     }
+    c->tc_ok = (shape->d_model % 64 == 0) &&
+               lmhead_tc_make_map(c->map_x, c->B.XN, (uint64_t)c->R_max + 128, (uint64_t)shape->d_model, 128) == 0 &&
+               lmhead_tc_make_map(c->map_w, c->lm_head, (uint64_t)shape->vocab, (uint64_t)shape->d_model, 256) == 0;
     c->pt_host.assign((size_t)c->D.B * c->D.pages_per_seq, 0);
     for (int p = shape->n_pages - 1; p >= 0; --p) c->free_pages.push_back(p);
     *out = c;

@@ -70,14 +70,9 @@ cudaError_t launch_select(const CtlArgs &a, const UpdatePlan *up, void *out_dev,
 cudaError_t launch_debug_logits(const CtlArgs &a, int layer, int seq, int slot, float *out_dev, cudaStream_t st);
 cudaError_t launch_gather_kv(const CtlArgs &a, int layer, int seq, int pos, float *k_out, float *v_out, cudaStream_t st);
 
-// streaming LM head over stacked rows (chunks of <= 64 rows through the rowgemm kernel is the
-// host's job); tensor-core version:
-struct LmTcArgs {
-    const void *tmap_x, *tmap_w;   // CUtensorMap in device-visible param space (passed by value below)
-    float *part_v;
-    int32_t *part_i;
-    int32_t n_rows, V, d, n_vtiles;
-    int32_t *err;
-};
-cudaError_t launch_lmhead_tc(const void *tmap_x_host, const void *tmap_w_host, float *part_v, int32_t *part_i,
-                             int n_rows, int V, int d, int32_t *err, int n_sms, cudaStream_t st, bool pdl);
+// Stacked LM head on tcgen05 / TMEM with fused arg-max (lmhead_tc.cu).  The tensor maps are 128-byte
+// opaque blobs (CUtensorMap) kept by the host context.
+int lmhead_tc_make_map(void *map_out, const void *base, uint64_t rows, uint64_t d, uint32_t box_rows);
+int lmhead_tc_vtiles(int V);
+cudaError_t launch_lmhead_tc(const void *map_x, const void *map_w, float *part_v, int32_t *part_i, int n_rows, int V, int d,
+                             int32_t *err, int n_sms, cudaStream_t st, bool pdl);

@@ -31,6 +31,7 @@ def main():
     ap.add_argument("--no-timing", action="store_true")
     ap.add_argument("--no-pdl", action="store_true")
     ap.add_argument("--one-cta", action="store_true")
+    ap.add_argument("--no-tc", action="store_true")
     a = ap.parse_args()
     base = synth.CONFIGS[a.config]
     L = a.layers
@@ -43,7 +44,7 @@ def main():
         if a.policy:
             E, G = (int(v) for v in a.policy.split(","))
             ctx.set_policy(s, E, G)
-    flags = (0 if a.no_pdl else dl.FLAG_PDL) | (16 if a.one_cta else 0)
+    flags = (0 if a.no_pdl else dl.FLAG_PDL) | (16 if a.one_cta else 0) | (0 if a.no_tc else dl.FLAG_TC)
     ctx.set_flags(flags)
     ctx.round()
     ctx.round()

@@ -205,3 +205,32 @@ def test_full_size_config_against_stored_trace(name, max_rounds):
     print(f"{name}: rounds {rep.rounds} compared {rep.compared} flips {rep.flips} resyncs {rep.resyncs}")
     assert rep.ok(), rep.failures[:8]
     assert rep.flips <= rep.compared // 20
+
+
+def test_streaming_lm_head_against_oracle(small):
+    """The stacked LM head also exists as a streaming (mma.sync) kernel; it must match the oracle too."""
+    import paper_2504_05598_b200 as dl
+    cfg, w, ctx = small
+    ref = ref_from_oracle(cfg, w, synth.make_prompt(cfg))
+    old = ctx.set_flags(dl.FLAG_PDL)
+    try:
+        rep = run_sequence(ctx, 0, ref, cfg.gen_len)
+    finally:
+        ctx.set_flags(old)
+    print(f"{cfg.name} (streaming head): rounds {rep.rounds} compared {rep.compared} flips {rep.flips}")
+    assert rep.ok(), rep.failures[:5]
+    assert rep.rounds == len(ref.rounds)
+
+
+def test_streaming_lm_head_full_size():
+    import paper_2504_05598_b200 as dl
+    name = "llama2_7b"
+    doc = json.load(open(os.path.join(GOLDEN, f"trace_{name}.json")))
+    cfg = synth.CONFIGS[name]
+    w = synth.make_weights(cfg)
+    ctx = make_ctx(cfg, w)
+    ctx.set_flags(dl.FLAG_PDL)
+    ref = ref_from_golden(doc, 0, synth.make_prompt(cfg, 0))
+    rep = run_sequence(ctx, 0, ref, doc["gen_len"], max_rounds=40)
+    print(f"{name} (streaming head): rounds {rep.rounds} compared {rep.compared} flips {rep.flips} resyncs {rep.resyncs}")
+    assert rep.ok(), rep.failures[:8]
