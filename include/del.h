@@ -199,6 +199,24 @@ int del_set_flags(del_ctx *ctx, int flags);
  * or KV the launches had to read).  HOST arrays of 8 (any may be NULL); reset != 0 clears the sums. */
 int del_get_kernel_times(del_ctx *ctx, double *ms, int64_t *launches, double *bytes, int reset);
 
+/* Exit-head arg-max without any allocation (the paper has no counterpart: this entry point exists for
+ * callers that cannot call cudaMalloc — a serving loop whose device memory pool is frozen after
+ * start-up, a plug-in that receives tensors but no allocator, a process that has filled the GPU).
+ * Needs no context.  x: DEVICE bf16 [rows][d_model], hidden rows already multiplied by the final norm's
+ * gain (the norm's 1/rms is positive and cannot change the arg-max); lm_head: DEVICE bf16
+ * [vocab][d_model]; tokens: DEVICE int32 [rows], token id of the largest logit per row (lowest id on
+ * ties).  Async on cuda_stream.  The kernel's scratch (per-CTA arg-max partials) lives in a fixed
+ * array inside the library image, DEL_STATIC_SCRATCH_BYTES per GPU that loads the library, held until
+ * the process exits.  Limits: 1 <= rows <= DEL_MAX_ROWS, vocab % 16 == 0, d_model >= 256 and % 8 == 0;
+ * anything larger than the fixed array can serve returns DEL_EINVAL.  No cudaMalloc / cudaFree or
+ * allocating library routine is called.  All calls on a device share the array: calls that overlap on
+ * the GPU (different streams) race, calls on one stream are safe; what a call reads from the array it
+ * has written first.  The first call on each device looks up the array's device address: make that
+ * call before any stream capture begins. */
+#define DEL_STATIC_SCRATCH_BYTES ((1 << 19) + 4096)
+int del_head_argmax_static(const void *x, const void *lm_head, int rows, int vocab, int d_model, int32_t *tokens,
+                           void *cuda_stream);
+
 const char *del_strerror(int code);
 /* Text of the last CUDA error seen by this context ("" if none). */
 const char *del_last_cuda_error(const del_ctx *ctx);

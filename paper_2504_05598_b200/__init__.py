@@ -27,7 +27,7 @@ KERNEL_CLASSES = ["qkv_rope", "attention", "o_proj", "gate_up", "down", "lm_head
 EXPORTS = ["del_workspace_bytes", "del_init", "del_prefill", "del_draft", "del_verify", "del_layer_accept",
            "del_select", "del_round", "del_set_policy", "del_get_stats", "del_set_stats", "del_get_shadow",
            "del_get_drafts", "del_force_token", "del_get_hidden", "del_debug_logits", "del_get_kv", "del_committed_len", "del_release",
-           "del_launch_count", "del_get_traffic", "del_set_flags", "del_get_kernel_times", "del_strerror", "del_last_cuda_error", "del_destroy"]
+           "del_launch_count", "del_get_traffic", "del_set_flags", "del_get_kernel_times", "del_head_argmax_static", "del_strerror", "del_last_cuda_error", "del_destroy"]
 
 
 class Shape(C.Structure):
@@ -118,6 +118,8 @@ def load_library(build_if_missing: bool = True):
     L.del_set_flags.argtypes = [vp, ci]
     L.del_get_kernel_times.restype = ci
     L.del_get_kernel_times.argtypes = [vp, vp, vp, vp, ci]
+    L.del_head_argmax_static.restype = ci
+    L.del_head_argmax_static.argtypes = [vp, vp, ci, ci, ci, vp, vp]
     L.del_strerror.restype = C.c_char_p
     L.del_strerror.argtypes = [ci]
     L.del_last_cuda_error.restype = C.c_char_p
@@ -327,3 +329,13 @@ def upload_weights(w, device="cuda:0") -> Dict:
 
     return {"tok_emb": up(w.tok_emb), "final_norm": up(w.final_norm), "lm_head": up(w.lm_head),
             "layers": [{k: up(v) for k, v in lw.items()} for lw in w.layers]}
+
+
+def head_argmax_static(x, lm_head, tokens_out, stream=None) -> int:
+    """del_head_argmax_static on torch CUDA tensors: x bf16 [rows, d], lm_head bf16 [vocab, d],
+    tokens_out int32 [rows].  Allocates nothing (the kernel's scratch is a fixed array in the library);
+    returns the library's status code."""
+    import torch
+    st = stream or torch.cuda.current_stream(x.device)
+    return load_library().del_head_argmax_static(x.data_ptr(), lm_head.data_ptr(), x.shape[0], lm_head.shape[0], x.shape[1],
+                                                 tokens_out.data_ptr(), C.c_void_p(st.cuda_stream))
