@@ -315,7 +315,7 @@ int run_layer(del_ctx *c, const PassInfo &pi, int l, bool write_exit) {
     {
         GemmArgs a = gemm_base(c, pi.plan_idx, l);
         a.K = D.d;
-        a.n_items = (D.nh + 2 * D.nkv) * (D.hd / 32);
+        a.n_items = (D.nh + 2 * D.nkv) * (D.hd / 16);
         a.X = c->B.XS;
         a.W0 = c->wq[l - 1]; a.W1 = c->wk[l - 1]; a.W2 = c->wv[l - 1];
         TAG(CLS_QKV, 2.0 * (D.nh + 2 * D.nkv) * D.hd * D.d);
@@ -351,7 +351,7 @@ int run_layer(del_ctx *c, const PassInfo &pi, int l, bool write_exit) {
     {
         GemmArgs a = gemm_base(c, pi.plan_idx, l);
         a.K = D.d;
-        a.n_items = D.F / 16;
+        a.n_items = D.F / 8;
         a.X = c->B.XM;
         a.W0 = c->w_gate[l - 1]; a.W1 = c->w_up[l - 1];
         TAG(CLS_GATEUP, 4.0 * D.F * D.d);

@@ -2,7 +2,7 @@
 // layer's element-wise work fused into its epilogues.  It is bound by HBM: every weight byte is read
 // exactly once per pass, straight from global memory into tensor-core fragments.
 //
-// Mapping.  A tile is 16 consecutive weight rows (output features) over the whole K.  The 8 warps of a
+// Mapping.  A tile is 16 weight rows (output features; two groups of 8, see tile_rows) over the whole K.  The 8 warps of a
 // CTA split K in 32-element steps (warp w takes steps w, w+8, ...), so at any time the CTA reads 512
 // contiguous bytes of each of the 16 rows.  Per step a thread issues one 16-byte load for row g and one
 // for row g+8 (g = lane/4) at column offset 8*(lane%4): the eight bf16 values feed two m16n8k16 MMAs.
@@ -27,38 +27,44 @@
 
 namespace {
 
-template <int EPI> struct EpiTraits { static constexpr int TPI = 1; };
-template <> struct EpiTraits<EPI_QKV> { static constexpr int TPI = 2; };
-template <> struct EpiTraits<EPI_GATEUP> { static constexpr int TPI = 2; };
-
-// weight row base of tile `which` of work item `item`
+// The 16 weight rows of a tile are two groups of 8 (MMA rows g and g+8), which need not be adjacent:
+//   QKV, q and k tiles: rows j..j+7 of a head and their rotary partners j+hd/2..  (one thread then holds
+//        both members of every rotation pair); v tiles: 16 consecutive rows
+//   GATEUP: 8 rows of W_gate and the same 8 rows of W_up (SiLU(gate)*up stays inside the tile)
+//   others: 16 consecutive rows
 template <int EPI>
-__device__ __forceinline__ const bf16 *tile_rows(const GemmArgs &a, int item, int which) {
+__device__ __forceinline__ void tile_rows(const GemmArgs &a, int item, const bf16 *&lo, const bf16 *&hi) {
     if (EPI == EPI_QKV) {
-        const int hp = a.D.hd >> 5;                 // pairs per head
-        const int nq = a.D.nh * hp, nk = a.D.nkv * hp;
+        const int h8 = a.D.hd >> 4;                 // tiles per head
+        const int nq = a.D.nh * h8, nk = a.D.nkv * h8;
         if (item < nq + nk) {
             const bf16 *W = item < nq ? a.W0 : a.W1;
             const int it = item < nq ? item : item - nq;
-            const int head = it / hp, jb = it - head * hp;
-            const int row = head * a.D.hd + jb * 16 + which * (a.D.hd >> 1);
-            return W + (size_t)row * a.K;
+            const int head = it / h8, jb = it - head * h8;
+            lo = W + (size_t)(head * a.D.hd + jb * 8) * a.K;
+            hi = lo + (size_t)(a.D.hd >> 1) * a.K;
+            return;
         }
-        const int it = item - nq - nk;
-        return a.W2 + (size_t)(32 * it + 16 * which) * a.K;
+        lo = a.W2 + (size_t)(16 * (item - nq - nk)) * a.K;
+        hi = lo + (size_t)8 * a.K;
+        return;
     }
-    if (EPI == EPI_GATEUP) return (which ? a.W1 : a.W0) + (size_t)(16 * item) * a.K;
-    return a.W0 + (size_t)(16 * item) * a.K;
+    if (EPI == EPI_GATEUP) {
+        lo = a.W0 + (size_t)(8 * item) * a.K;
+        hi = a.W1 + (size_t)(8 * item) * a.K;
+        return;
+    }
+    lo = a.W0 + (size_t)(16 * item) * a.K;
+    hi = lo + (size_t)8 * a.K;
 }
 
 template <int NT, int U, int EPI>
 __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_kernel(const GemmArgs a) {
-    constexpr int TPI = EpiTraits<EPI>::TPI;
     constexpr int NC = NT * 8;                      // activation-row columns handled
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float4 *red = reinterpret_cast<float4 *>(smem_raw);                       // [8 warps][NT][32]
-    float *res = reinterpret_cast<float *>(smem_raw + sizeof(float4) * 8 * NT * 32);  // [TPI][NC][16]
-    float *rscale = res + TPI * NC * 16;                                      // [NC]
+    float *res = reinterpret_cast<float *>(smem_raw + sizeof(float4) * 8 * NT * 32);  // [NC][16]
+    float *rscale = res + NC * 16;                                      // [NC]
     float *best_v = rscale + NC;                                              // [NC]
     int *best_i = reinterpret_cast<int *>(best_v + NC);                       // [NC]
 
@@ -67,24 +73,26 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     const int n_ksteps = (K + 31) >> 5;
     const int nkw = (n_ksteps + 7) >> 3;            // k-steps per warp and tile (the last ones may be empty)
     const int my_items = (a.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    const int my_tiles = my_items * TPI;
+    const int my_tiles = my_items;
 
     uint4 wa[U], wb[U];
     uint4 xv[U][NT];
     const bf16 *xrow[NT];
 
+    const bf16 *base = nullptr, *base_hi = nullptr;     // this thread's row g / row g+8 of the current tile
     auto tile_base = [&](int ti) {
-        const int item = blockIdx.x + (ti / TPI) * gridDim.x;
-        return tile_rows<EPI>(a, item, ti % TPI) + (size_t)g * K + 8 * t;
+        tile_rows<EPI>(a, blockIdx.x + ti * gridDim.x, base, base_hi);
+        base += (size_t)g * K + 8 * t;
+        base_hi += (size_t)g * K + 8 * t;
     };
     // one burst: U k-steps of this warp, all loads issued before the first use
-    auto load_w = [&](const bf16 *base, int u0, bool live) {
+    auto load_w = [&](int u0, bool live) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int k0 = (warp + 8 * (u0 + u)) << 5;
             const bool ok = live && (u0 + u < nkw) && (k0 + 8 * t < K);
             wa[u] = ldg_stream16_pred(base + k0, ok);
-            wb[u] = ldg_stream16_pred(base + (size_t)8 * K + k0, ok);
+            wb[u] = ldg_stream16_pred(base_hi + k0, ok);
         }
     };
     auto load_x = [&](int u0, bool live) {
@@ -98,8 +106,8 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     };
 
     // the first burst of weights goes out before the producer kernel has finished
-    const bf16 *base = tile_base(0);
-    load_w(base, 0, true);
+    tile_base(0);
+    load_w(0, true);
     pdl_launch();
     pdl_wait();
 
@@ -153,7 +161,6 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
             acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
         }
         __syncthreads();
-        const int which = c_tile % TPI;
         for (int e = tid; e < NT * 32; e += DEL_GEMM_THREADS) {
             float4 s = red[e];
 #pragma unroll
@@ -162,12 +169,11 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
                 s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
             }
             const int nt = e >> 5, l2 = e & 31, g2 = l2 >> 2, t2 = l2 & 3;
-            float *r0 = res + ((which * NC) + nt * 8 + 2 * t2) * 16;
+            float *r0 = res + (nt * 8 + 2 * t2) * 16;
             r0[g2] = s.x; r0[16 + g2] = s.y; r0[g2 + 8] = s.z; r0[16 + g2 + 8] = s.w;
         }
         __syncthreads();
-        if (which != TPI - 1) return;
-        const int item = blockIdx.x + (c_tile / TPI) * gridDim.x;
+        const int item = blockIdx.x + c_tile * gridDim.x;
         const int i = tid & 15;
         for (int c = tid >> 4; c < NC; c += DEL_GEMM_THREADS / 16) {
             const bool valid = c < m;
@@ -176,15 +182,16 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
             if (EPI == EPI_QKV) {
                 if (!valid) continue;
                 const float r = rscale[c];
-                const float va = r * ra, vb = r * res[(NC + c) * 16 + i];
-                const int hd = a.D.hd, half = hd >> 1, hp = hd >> 5;
-                const int nq = a.D.nh * hp, nk = a.D.nkv * hp;
+                const int hd = a.D.hd, half = hd >> 1, h8 = hd >> 4;
+                const int nq = a.D.nh * h8, nk = a.D.nkv * h8;
                 const int pg = a.B.PT[rd.seq * a.D.pages_per_seq + (rd.pos >> 4)];
                 const int sl = rd.pos & 15;
                 if (item < nq + nk) {
+                    if (i >= 8) continue;                         // rows 0..7 and their partners 8..15: one thread per pair
+                    const float va = r * ra, vb = r * res[c * 16 + 8 + i];
                     const bool isq = item < nq;
                     const int it = isq ? item : item - nq;
-                    const int head = it / hp, j = (it - head * hp) * 16 + i;
+                    const int head = it / h8, j = (it - head * h8) * 8 + i;
                     const float cs = a.B.rope_cos[(size_t)rd.pos * half + j], sn = a.B.rope_sin[(size_t)rd.pos * half + j];
                     const float oa = va * cs - vb * sn, ob = vb * cs + va * sn;
                     if (isq) {
@@ -197,18 +204,17 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
                         kp[half] = __float2bfloat16_rn(ob);
                     }
                 } else {
-                    const int n0 = 32 * (item - nq - nk) + i;      // value feature of tile 0; tile 1 is +16
+                    const int n0 = 16 * (item - nq - nk) + i;      // value feature
                     const int kvh = n0 / hd, dim = n0 - kvh * hd;
-                    bf16 *vp = a.B.VP + ((((size_t)pg * a.D.L + (a.layer - 1)) * a.D.nkv + kvh) * hd + dim) * 16 + sl;
-                    vp[0] = __float2bfloat16_rn(va);
-                    vp[16 * 16] = __float2bfloat16_rn(vb);
+                    a.B.VP[((((size_t)pg * a.D.L + (a.layer - 1)) * a.D.nkv + kvh) * hd + dim) * 16 + sl] = __float2bfloat16_rn(r * ra);
                 }
             } else if (EPI == EPI_GATEUP) {
                 if (!valid) continue;
                 const float r = rscale[c];
-                const float gate = r * ra, up = r * res[(NC + c) * 16 + i];
+                if (i >= 8) continue;                             // rows 0..7 gate, rows 8..15 the matching up rows
+                const float gate = r * ra, up = r * res[c * 16 + 8 + i];
                 const float act = gate / (1.f + __expf(-gate)) * up;
-                a.B.ACT[(size_t)c * a.D.F + 16 * item + i] = __float2bfloat16_rn(act);
+                a.B.ACT[(size_t)c * a.D.F + 8 * item + i] = __float2bfloat16_rn(act);
             } else if (EPI == EPI_OPROJ || EPI == EPI_DOWN) {
                 const int o = 16 * item + i;
                 float h = 0.f;
@@ -264,14 +270,14 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     int u0 = U;
     for (;;) {
         for (; u0 < nkw; u0 += U) {
-            load_w(base, u0, true);
+            load_w(u0, true);
             load_x(u0, true);
             mma_burst();
         }
         // the next tile's first burst is in flight while this tile is reduced and written out
         const bool more = c_tile + 1 < my_tiles;
-        if (more) base = tile_base(c_tile + 1);
-        load_w(base, 0, more);
+        if (more) tile_base(c_tile + 1);
+        load_w(0, more);
         load_x(0, more);
         tile_end();
         if (!more) break;
@@ -294,9 +300,8 @@ template <int NT> constexpr int depth_for() { return NT == 1 ? 8 : (NT == 2 ? 4 
 template <int NT, int EPI>
 cudaError_t launch_nt(const GemmArgs &a, int grid, cudaStream_t st, bool pdl) {
     constexpr int D = depth_for<NT>();
-    constexpr int TPI = EpiTraits<EPI>::TPI;
     constexpr int NC = NT * 8;
-    const size_t smem = sizeof(float4) * 8 * NT * 32 + sizeof(float) * (TPI * NC * 16 + 3 * NC);
+    const size_t smem = sizeof(float4) * 8 * NT * 32 + sizeof(float) * (NC * 16 + 3 * NC);
     auto kern = rowgemm_kernel<NT, D, EPI>;
     static bool attr_done = false;
     if (!attr_done) {
