@@ -28,7 +28,7 @@ constexpr int NW = 8;                 // warps per CTA
 constexpr int PG = 4;                 // page ids fetched ahead per warp
 
 template <int HD>
-__global__ void __launch_bounds__(NW * 32) attention_kernel(const AttnArgs a) {
+__global__ void __launch_bounds__(NW * 32) attention_kernel(const __grid_constant__ AttnArgs a) {
     constexpr int KS = HD / 32;       // 16-byte chunks per thread along head_dim
     constexpr int NJ = HD / 8;        // output n-tiles
     extern __shared__ __align__(16) float sm[];
@@ -36,11 +36,11 @@ __global__ void __launch_bounds__(NW * 32) attention_kernel(const AttnArgs a) {
     float *sm_ml = sm + NW * 32 * NJ * 4;           // [NW][32][4]
     __shared__ int s_last;
 
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     pdl_launch();
     pdl_wait();
 
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
-    const PassPlan *plan = a.plan;
+    const PassPlan *plan = &a.plan;
     const Segment seg = plan->seg[blockIdx.z];
     const int kvh = blockIdx.y, split = blockIdx.x, n_splits = a.n_splits;
     const int ms = seg.nrows, group = a.D.nh / a.D.nkv;

@@ -47,10 +47,10 @@ __device__ __forceinline__ void write_embedding(const CtlArgs &a, int token, int
     }
 }
 
-__global__ void __launch_bounds__(CTL_THREADS) embed_kernel(const CtlArgs a) {
+__global__ void __launch_bounds__(CTL_THREADS) embed_kernel(const __grid_constant__ CtlArgs a) {
     pdl_launch();
     pdl_wait();
-    const RowDesc rd = a.plan->rows[blockIdx.x];
+    const RowDesc rd = a.plan.rows[blockIdx.x];
     const int token = a.tok_src[rd.tok];
     write_embedding(a, token, rd.seq, rd.slot);
 }
@@ -75,12 +75,12 @@ __device__ __forceinline__ void block_argmax(float &v, int &idx) {
 
 // Draft head, last step: reduce the per-CTA arg-max partials of the streaming LM head into the draft
 // token, store it, and write the embedding of that token as the next row of the sequence.
-__global__ void __launch_bounds__(CTL_THREADS) draft_finalize_embed_kernel(const CtlArgs a, int embed_next) {
+__global__ void __launch_bounds__(CTL_THREADS) draft_finalize_embed_kernel(const __grid_constant__ CtlArgs a, int embed_next) {
     __shared__ int s_tok;
     pdl_launch();
     pdl_wait();
     const int c = blockIdx.x;
-    const RowDesc rd = a.plan->rows[c];
+    const RowDesc rd = a.plan.rows[c];
     float v = -INFINITY;
     int idx = 0x7fffffff;
     for (int p = threadIdx.x; p < a.n_part; p += CTL_THREADS) {

@@ -13,7 +13,7 @@
 namespace {
 
 constexpr int PLAN_RING = 192;
-constexpr int FLAG_PDL = 1, FLAG_GRAPH = 2, FLAG_TC = 4, FLAG_TIMING = 8;
+constexpr int FLAG_PDL = 1, FLAG_GRAPH = 2, FLAG_TC = 4, FLAG_TIMING = 8, FLAG_ONECTA = 16;
 enum { CLS_QKV = 0, CLS_ATTN, CLS_OPROJ, CLS_GATEUP, CLS_DOWN, CLS_LMHEAD, CLS_LMSTACK, CLS_OTHER, CLS_N };
 
 struct SeqHost {
@@ -53,7 +53,7 @@ struct del_ctx {
     std::vector<int> free_pages;
     std::vector<int32_t> pt_host;
     // plans
-    PassPlan *plan_host = nullptr, *plan_dev = nullptr;
+    PassPlan *plan_host = nullptr;       // host ring of pass plans (passed to kernels by value)
     int plan_cur = 0;
     UpdatePlan *up_host = nullptr, *up_dev = nullptr;      // [2]
     del_round_out *out_host = nullptr, *out_dev = nullptr; // [B]
@@ -76,7 +76,7 @@ struct del_ctx {
 
 namespace {
 
-size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max, int &n_vtiles, PassPlan **plan_dev,
+size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max, int &n_vtiles,
                  UpdatePlan **up_dev, del_round_out **out_dev, float **dbg_dev) {
     D.L = s.n_layers; D.d = s.d_model; D.nh = s.n_heads; D.nkv = s.n_kv_heads; D.hd = s.head_dim; D.F = s.d_ffn; D.V = s.vocab;
     D.B = s.max_batch;
@@ -113,7 +113,6 @@ size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max
     B.SC = c.take<double>(base, (size_t)D.B * D.L);
     B.ST = c.take<SeqState>(base, (size_t)D.B);
     B.ERR = c.take<int32_t>(base, 64);
-    *plan_dev = c.take<PassPlan>(base, PLAN_RING);
     *up_dev = c.take<UpdatePlan>(base, 2);
     *out_dev = c.take<del_round_out>(base, (size_t)D.B);
     *dbg_dev = c.take<float>(base, (size_t)std::max(D.V, 2 * D.nkv * D.hd));
@@ -208,16 +207,12 @@ struct PlanBatch {
 int plan_begin(del_ctx *c, int need) {
     if (need > PLAN_RING) return DEL_EINVAL;
     if (c->plan_cur + need > PLAN_RING) {
-        // wrap: earlier copies out of the pinned ring must have been consumed
-        CK(cudaStreamSynchronize(c->st));
         c->plan_cur = 0;
     }
     return DEL_OK;
 }
 int plan_commit(del_ctx *c, const PlanBatch &b) {
     if (b.count == 0) return DEL_OK;
-    CK(cudaMemcpyAsync(c->plan_dev + b.first, c->plan_host + b.first, sizeof(PassPlan) * b.count, cudaMemcpyHostToDevice, c->st));
-    c->h2d_bytes += sizeof(PassPlan) * b.count;
     c->plan_cur = b.first + b.count;
     return DEL_OK;
 }
@@ -272,7 +267,7 @@ GemmArgs gemm_base(const del_ctx *c, int plan_idx, int layer) {
     memset(&a, 0, sizeof(a));
     a.D = c->D;
     a.B = c->B;
-    a.plan = c->plan_dev + plan_idx;
+    a.plan = c->plan_host[plan_idx];
     a.layer = layer;
     return a;
 }
@@ -282,7 +277,7 @@ CtlArgs ctl_base(const del_ctx *c, int plan_idx) {
     memset(&a, 0, sizeof(a));
     a.D = c->D;
     a.B = c->B;
-    a.plan = plan_idx >= 0 ? c->plan_dev + plan_idx : nullptr;
+    if (plan_idx >= 0) a.plan = c->plan_host[plan_idx];
     a.tok_emb = c->tok_emb;
     a.gain0 = c->attn_norm[0];
     a.final_gain = c->final_norm;
@@ -324,7 +319,7 @@ int run_layer(del_ctx *c, const PassInfo &pi, int l, bool write_exit) {
     {
         AttnArgs a;
         memset(&a, 0, sizeof(a));
-        a.D = D; a.B = c->B; a.plan = c->plan_dev + pi.plan_idx; a.layer = l;
+        a.D = D; a.B = c->B; a.plan = c->plan_host[pi.plan_idx]; a.layer = l;
         const int pages = (pi.max_kv + 15) / 16;
         const int R = pi.max_rows * (D.nh / D.nkv), n_mt = (R + 15) / 16;
         const int ns = attention_splits(pages, pi.n_seg * D.nkv, n_mt >= 3 ? 4 : n_mt, c->n_sms);
@@ -577,8 +572,8 @@ extern "C" {
 
 size_t del_workspace_bytes(const del_shape *shape) {
     if (validate(shape) != DEL_OK) return 0;
-    Dims D; Buffers B; int R, nv; PassPlan *p; UpdatePlan *u; del_round_out *o; float *dbg;
-    return carve_all(*shape, nullptr, D, B, R, nv, &p, &u, &o, &dbg);
+    Dims D; Buffers B; int R, nv; UpdatePlan *u; del_round_out *o; float *dbg;
+    return carve_all(*shape, nullptr, D, B, R, nv, &u, &o, &dbg);
 }
 
 int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const del_kv *kv, void *workspace,
@@ -594,7 +589,7 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
     del_ctx *c = new (std::nothrow) del_ctx();
     if (!c) return DEL_ENOSPC;
     c->sh = *shape;
-    carve_all(*shape, workspace, c->D, c->B, c->R_max, c->n_vtiles, &c->plan_dev, &c->up_dev, &c->out_dev, &c->dbg_dev);
+    carve_all(*shape, workspace, c->D, c->B, c->R_max, c->n_vtiles, &c->up_dev, &c->out_dev, &c->dbg_dev);
     c->B.KP = (bf16 *)kv->k_pages; c->B.VP = (bf16 *)kv->v_pages; c->B.PT = kv->page_table;
     c->B.rope_cos = w->rope_cos; c->B.rope_sin = w->rope_sin;
     c->tok_emb = (const bf16 *)w->tok_emb; c->final_norm = (const bf16 *)w->final_norm; c->lm_head = (const bf16 *)w->lm_head;
@@ -945,7 +940,7 @@ int del_set_flags(del_ctx *c, int flags) {
     if (!c) return DEL_EINVAL;
     const int old = c->flags;
     c->flags = flags;
-    rowgemm_set_ctas_per_sm((flags & 16) ? 1 : 2);
+    rowgemm_set_ctas_per_sm((flags & FLAG_ONECTA) ? 1 : 2);
     return old;
 }
 

@@ -8,7 +8,7 @@ enum { EPI_QKV = 0, EPI_OPROJ = 1, EPI_GATEUP = 2, EPI_DOWN = 3, EPI_LMHEAD = 4 
 struct GemmArgs {
     Dims D;
     Buffers B;
-    const PassPlan *plan;      // device
+    PassPlan plan;             // rows of the pass, by value: read from the constant bank, no dependent load
     int32_t layer;             // 1-based layer the op belongs to (LMHEAD: the exit layer)
     int32_t K;                 // in-features
     int32_t n_items;           // work items: tile pairs (QKV, GATEUP) or 16-row tiles
@@ -25,7 +25,7 @@ void rowgemm_set_ctas_per_sm(int n);
 struct AttnArgs {
     Dims D;
     Buffers B;
-    const PassPlan *plan;
+    PassPlan plan;
     int32_t layer;
     int32_t n_splits;          // key-range splits per (segment, kv head)
     int32_t max_rows;          // largest segment (rows), decides the number of query tiles
@@ -37,7 +37,7 @@ int attention_splits(int pages, int n_units, int tiles_par, int n_sms);
 struct CtlArgs {
     Dims D;
     Buffers B;
-    const PassPlan *plan;
+    PassPlan plan;
     const bf16 *tok_emb, *gain0, *final_gain, *lm_head;
     const int32_t *tok_src;    // token buffer the embedding reads (B.TOK or B.PROMPT)
     int32_t n_part;            // LM-head partials to reduce

@@ -22,9 +22,8 @@
 namespace {
 
 constexpr int MAX_CTAS = 1024;
-constexpr size_t PLAN_BYTES = (sizeof(PassPlan) + 255) & ~(size_t)255;
 constexpr size_t PART_BYTES = (size_t)MAX_CTAS * DEL_ROWS_MAX * 4;
-constexpr size_t SCRATCH_BYTES = PLAN_BYTES + 2 * PART_BYTES;
+constexpr size_t SCRATCH_BYTES = 2 * PART_BYTES;
 static_assert(SCRATCH_BYTES <= DEL_STATIC_SCRATCH_BYTES, "static scratch larger than documented");
 
 // The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress, never an address.
@@ -32,14 +31,6 @@ static __device__ __align__(256) unsigned char g_static_scratch[DEL_STATIC_SCRAT
 
 constexpr int MAX_DEVICES = 64;
 unsigned char *g_scratch_ptr[MAX_DEVICES] = {nullptr};   // device address of the array, per device
-
-// Device code may name the array directly: start the call's plan from a clean slate.
-__global__ void static_plan_kernel(int m) {
-    PassPlan *plan = reinterpret_cast<PassPlan *>(g_static_scratch);
-    for (int i = threadIdx.x; i < (int)(sizeof(PassPlan) / 4); i += blockDim.x) reinterpret_cast<int32_t *>(plan)[i] = 0;
-    __syncthreads();
-    if (threadIdx.x == 0) plan->m = m;
-}
 
 // one block per row: reduce the per-CTA partials, ties to the lowest token id
 __global__ void __launch_bounds__(256) static_argmax_kernel(const float *pv, const int32_t *pi, int n_part, int32_t *tokens) {
@@ -93,17 +84,15 @@ extern "C" int del_head_argmax_static(const void *x, const void *lm_head, int ro
     GemmArgs a;
     memset(&a, 0, sizeof(a));
     a.D.d = d_model; a.D.V = vocab; a.D.S = 1; a.D.B = 1; a.D.n_sst = d_model / 16;
-    a.plan = reinterpret_cast<const PassPlan *>(scratch);
+    a.plan.m = rows;
     a.K = d_model;
     a.n_items = n_items;
     a.X = reinterpret_cast<const bf16 *>(x);
     a.W0 = reinterpret_cast<const bf16 *>(lm_head);
     a.x_by_row = 1;
-    a.B.LPV = reinterpret_cast<float *>(scratch + PLAN_BYTES);
-    a.B.LPI = reinterpret_cast<int32_t *>(scratch + PLAN_BYTES + PART_BYTES);
+    a.B.LPV = reinterpret_cast<float *>(scratch);
+    a.B.LPI = reinterpret_cast<int32_t *>(scratch + PART_BYTES);
 
-    static_plan_kernel<<<1, 256, 0, st>>>(rows);
-    if (cudaGetLastError() != cudaSuccess) return DEL_ECUDA;
     if (launch_rowgemm(EPI_LMHEAD, a, rows, n_sms, st, false) != cudaSuccess) return DEL_ECUDA;
     static_argmax_kernel<<<rows, 256, 0, st>>>(a.B.LPV, a.B.LPI, n_part, tokens);
     if (cudaGetLastError() != cudaSuccess) return DEL_ECUDA;

@@ -59,7 +59,7 @@ __device__ __forceinline__ void tile_rows(const GemmArgs &a, int item, const bf1
 }
 
 template <int NT, int U, int EPI>
-__global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_kernel(const GemmArgs a) {
+__global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_kernel(const __grid_constant__ GemmArgs a) {
     constexpr int NC = NT * 8;                      // activation-row columns handled
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float4 *red = reinterpret_cast<float4 *>(smem_raw);                       // [8 warps][NT][32]
@@ -111,7 +111,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     pdl_launch();
     pdl_wait();
 
-    const PassPlan *plan = a.plan;
+    const PassPlan *plan = &a.plan;
     const int m = plan->m;
     // activation row pointers of this thread's columns
 #pragma unroll
