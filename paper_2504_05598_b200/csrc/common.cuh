@@ -74,6 +74,7 @@ struct Buffers {
     double *SC;                  // [B][L] decayed match counts
     SeqState *ST;                // [B]
     int32_t *ERR;                // device error word
+    int32_t *TCNT;               // ring of per-launch tile-claim counters
     bf16 *KP, *VP;               // KV pages
     int32_t *PT;                 // page table [B][pages_per_seq]
     const float *rope_cos, *rope_sin;
@@ -117,6 +118,12 @@ __device__ __forceinline__ uint4 ldg_act16_pred(const void *p, bool pred) {
                  "@q ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];\n\t}"
                  : "=&r"(v.x), "=&r"(v.y), "=&r"(v.z), "=&r"(v.w) : "l"(p), "r"((uint32_t)pred));
     return v;
+}
+// 16-byte asynchronous global -> shared copy (zero fill when `pred` is false)
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src, bool pred) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    const uint32_t n = pred ? 16u : 0u;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(gmem_src), "r"(n) : "memory");
 }
 __device__ __forceinline__ uint2 ldg_act8(const void *p) {
     uint2 v;

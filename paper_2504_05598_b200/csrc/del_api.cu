@@ -13,6 +13,7 @@
 namespace {
 
 constexpr int PLAN_RING = 192;
+constexpr int CTR_RING = 4096;
 constexpr int FLAG_PDL = 1, FLAG_GRAPH = 2, FLAG_TC = 4, FLAG_TIMING = 8, FLAG_ONECTA = 16;
 enum { CLS_QKV = 0, CLS_ATTN, CLS_OPROJ, CLS_GATEUP, CLS_DOWN, CLS_LMHEAD, CLS_LMSTACK, CLS_OTHER, CLS_N };
 
@@ -53,6 +54,7 @@ struct del_ctx {
     std::vector<int> free_pages;
     std::vector<int32_t> pt_host;
     // plans
+    int ctr_cur = 0;                     // next free slot of the tile-claim counter ring
     PassPlan *plan_host = nullptr;       // host ring of pass plans (passed to kernels by value)
     int plan_cur = 0;
     UpdatePlan *up_host = nullptr, *up_dev = nullptr;      // [2]
@@ -113,6 +115,7 @@ size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max
     B.SC = c.take<double>(base, (size_t)D.B * D.L);
     B.ST = c.take<SeqState>(base, (size_t)D.B);
     B.ERR = c.take<int32_t>(base, 64);
+    B.TCNT = c.take<int32_t>(base, CTR_RING);
     *up_dev = c.take<UpdatePlan>(base, 2);
     *out_dev = c.take<del_round_out>(base, (size_t)D.B);
     *dbg_dev = c.take<float>(base, (size_t)std::max(D.V, 2 * D.nkv * D.hd));
@@ -262,9 +265,19 @@ void release_seq(del_ctx *c, int sq) {
     s = SeqHost();
 }
 
-GemmArgs gemm_base(const del_ctx *c, int plan_idx, int layer) {
+// next zeroed tile-claim counter; the ring is cleared (in stream order) each time it wraps
+int32_t *next_counter(del_ctx *c) {
+    if (c->ctr_cur == CTR_RING) {
+        cudaMemsetAsync(c->B.TCNT, 0, sizeof(int32_t) * CTR_RING, c->st);
+        c->ctr_cur = 0;
+    }
+    return c->B.TCNT + c->ctr_cur++;
+}
+
+GemmArgs gemm_base(del_ctx *c, int plan_idx, int layer) {
     GemmArgs a;
     memset(&a, 0, sizeof(a));
+    a.tile_ctr = next_counter(c);
     a.D = c->D;
     a.B = c->B;
     a.plan = c->plan_host[plan_idx];

@@ -15,6 +15,7 @@ struct GemmArgs {
     const bf16 *X;             // activations (see rowgemm.cu for the indexing per epilogue)
     const bf16 *W0, *W1, *W2;
     const bf16 *gain_a, *gain_b;
+    int32_t *tile_ctr;         // per-launch zeroed counter for dynamic tile claims (nullptr: static round-robin)
     int32_t x_by_row;          // LMHEAD: activations are X[c] (stacked rows) instead of XE[seq][slot]
 };
 

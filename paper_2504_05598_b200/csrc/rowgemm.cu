@@ -25,7 +25,18 @@
 // its accumulators by rsqrt(mean(h^2) + eps) (the scale is a per-row scalar, so it commutes with W).
 #include "kernels.h"
 
+// optional per-CTA time stamps for tuning builds (a harness defines the macro); off in the library
+#ifndef DEL_TRACE_STAMP
+#define DEL_TRACE_STAMP(i)
+#endif
+
 namespace {
+
+
+// bytes of the reduction buffer, result tile, row scales and arg-max state (16-byte multiple)
+__host__ __device__ constexpr size_t small_smem_bytes(int nt) {
+    return (sizeof(float4) * 8 * nt * 32 + sizeof(float) * (nt * 8 * 16 + 3 * nt * 8) + 15) & ~(size_t)15;
+}
 
 // The 16 weight rows of a tile are two groups of 8 (MMA rows g and g+8), which need not be adjacent:
 //   QKV, q and k tiles: rows j..j+7 of a head and their rotary partners j+hd/2..  (one thread then holds
@@ -72,20 +83,20 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     const int K = a.K;
     const int n_ksteps = (K + 31) >> 5;
     const int nkw = (n_ksteps + 7) >> 3;            // k-steps per warp and tile (the last ones may be empty)
-    const int my_items = (a.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    const int my_tiles = my_items;
+    __shared__ int s_claim[2];                      // tile claimed for the turn after next (double-buffered)
 
     uint4 wa[U], wb[U];
     uint4 xv[U][NT];
     const bf16 *xrow[NT];
 
     const bf16 *base = nullptr, *base_hi = nullptr;     // this thread's row g / row g+8 of the current tile
-    auto tile_base = [&](int ti) {
-        tile_rows<EPI>(a, blockIdx.x + ti * gridDim.x, base, base_hi);
+    auto tile_base = [&](int item) {
+        tile_rows<EPI>(a, item, base, base_hi);
         base += (size_t)g * K + 8 * t;
         base_hi += (size_t)g * K + 8 * t;
     };
     // one burst: U k-steps of this warp, all loads issued before the first use
+    // (the load sequences are kept free of branches: the compiler batches them only in straight-line code)
     auto load_w = [&](int u0, bool live) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
@@ -106,10 +117,22 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     };
 
     // the first burst of weights goes out before the producer kernel has finished
-    tile_base(0);
+    DEL_TRACE_STAMP(0);
+    // Tiles: two static turns per CTA (b, b + grid), further tiles claimed from a per-launch counter so that
+    // fast CTAs take more and all CTAs finish together.  Results do not depend on who computes a tile.
+    const int grid = (int)gridDim.x;
+    int cur_item = blockIdx.x;
+    int nxt_item = cur_item + grid < a.n_items ? cur_item + grid : -1;
+    int claimed = -1;                               // thread 0: the claim in flight
+    auto claim = [&]() {
+        if (tid == 0 && a.tile_ctr != nullptr && nxt_item >= 0) claimed = 2 * grid + atomicAdd(a.tile_ctr, 1);
+    };
+    tile_base(cur_item);
     load_w(0, true);
+    claim();
     pdl_launch();
     pdl_wait();
+    DEL_TRACE_STAMP(1);
 
     const PassPlan *plan = &a.plan;
     const int m = plan->m;
@@ -128,30 +151,33 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     }
     load_x(0, true);
 
-    // per-row 1/rms from the producer's partial sums of squares
+    // per-row 1/rms from the producer's partial sums of squares: the loads of this warp's first row go
+    // out now, their sum is taken after the first burst of MMAs (it is needed in the first epilogue only)
+    constexpr int SSN = 12;                         // 32 * 12 partials = rows of up to 6144 features
+    float ssv[SSN];
+    auto ss_ptr = [&](int c) -> const float * {
+        if (EPI == EPI_GATEUP) return a.B.SSM + (size_t)c * a.D.n_sst;
+        return a.B.SS + stack_row(a.D, a.layer - 1, plan->rows[c].seq, plan->rows[c].slot) * a.D.n_sst;
+    };
     if (EPI == EPI_QKV || EPI == EPI_GATEUP) {
-        for (int c = warp; c < NC; c += DEL_GEMM_WARPS) {
-            float s = 0.f;
-            if (c < m) {
-                const float *ss;
-                if (EPI == EPI_GATEUP) ss = a.B.SSM + (size_t)c * a.D.n_sst;
-                else ss = a.B.SS + stack_row(a.D, a.layer - 1, plan->rows[c].seq, plan->rows[c].slot) * a.D.n_sst;
-                for (int i = lane; i < a.D.n_sst; i += 32) s += ldg_cg_f32(ss + i);
-            }
-            s = warp_sum(s);
-            if (lane == 0) rscale[c] = rsqrtf(s / (float)a.D.d + a.D.eps);
+        const bool v0 = warp < m;
+        const float *ss = v0 ? ss_ptr(warp) : a.B.SSM;
+#pragma unroll
+        for (int q = 0; q < SSN; ++q) {
+            const int i = lane + 32 * q;
+            ssv[q] = (v0 && i < a.D.n_sst) ? ldg_cg_f32(ss + i) : 0.f;
         }
     }
     if (EPI == EPI_LMHEAD) {
         for (int c = tid; c < NC; c += DEL_GEMM_THREADS) { best_v[c] = -INFINITY; best_i[c] = 0x7fffffff; }
     }
-    __syncthreads();
+    // no barrier here: rscale / best_* are first read in an epilogue, after the two barriers of tile_end
 
     float acc[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
 
-    int c_tile = 0;
+    int turn = 0;
 
     auto tile_end = [&]() {
         // fixed-order sum of the 8 warps' partials
@@ -173,7 +199,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
             r0[g2] = s.x; r0[16 + g2] = s.y; r0[g2 + 8] = s.z; r0[16 + g2 + 8] = s.w;
         }
         __syncthreads();
-        const int item = blockIdx.x + c_tile * gridDim.x;
+        const int item = cur_item;
         const int i = tid & 15;
         for (int c = tid >> 4; c < NC; c += DEL_GEMM_THREADS / 16) {
             const bool valid = c < m;
@@ -267,6 +293,23 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     };
 
     mma_burst();
+    DEL_TRACE_STAMP(2);
+    if (EPI == EPI_QKV || EPI == EPI_GATEUP) {
+        for (int c = warp; c < NC; c += DEL_GEMM_WARPS) {
+            float s = 0.f;
+            if (c == warp) {
+#pragma unroll
+                for (int q = 0; q < SSN; ++q) s += ssv[q];
+                if (c < m)
+                    for (int i = lane + 32 * SSN; i < a.D.n_sst; i += 32) s += ldg_cg_f32(ss_ptr(c) + i);
+            } else if (c < m) {
+                const float *ss = ss_ptr(c);
+                for (int i = lane; i < a.D.n_sst; i += 32) s += ldg_cg_f32(ss + i);
+            }
+            s = warp_sum(s);
+            if (lane == 0) rscale[c] = rsqrtf(s / (float)a.D.d + a.D.eps);
+        }
+    }
     int u0 = U;
     for (;;) {
         for (; u0 < nkw; u0 += U) {
@@ -275,17 +318,25 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
             mma_burst();
         }
         // the next tile's first burst is in flight while this tile is reduced and written out
-        const bool more = c_tile + 1 < my_tiles;
-        if (more) tile_base(c_tile + 1);
+        const bool more = nxt_item >= 0;
+        if (more) tile_base(nxt_item);
         load_w(0, more);
         load_x(0, more);
+        if (tid == 0) s_claim[turn & 1] = claimed;
         tile_end();
         if (!more) break;
-        ++c_tile;
+        int after;
+        if (a.tile_ctr != nullptr) after = s_claim[turn & 1];
+        else after = nxt_item + grid;
+        cur_item = nxt_item;
+        nxt_item = (after >= 0 && after < a.n_items) ? after : -1;
+        ++turn;
+        claim();
         mma_burst();
         u0 = U;
     }
 
+    DEL_TRACE_STAMP(3);
     if (EPI == EPI_LMHEAD) {
         __syncthreads();
         for (int c = tid; c < m; c += DEL_GEMM_THREADS) {
@@ -301,7 +352,7 @@ template <int NT, int EPI>
 cudaError_t launch_nt(const GemmArgs &a, int grid, cudaStream_t st, bool pdl) {
     constexpr int D = depth_for<NT>();
     constexpr int NC = NT * 8;
-    const size_t smem = sizeof(float4) * 8 * NT * 32 + sizeof(float) * (NC * 16 + 3 * NC);
+    const size_t smem = small_smem_bytes(NT);
     auto kern = rowgemm_kernel<NT, D, EPI>;
     static bool attr_done = false;
     if (!attr_done) {
