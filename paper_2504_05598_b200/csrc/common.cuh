@@ -130,6 +130,13 @@ __device__ __forceinline__ uint2 ldg_act8(const void *p) {
     asm volatile("ld.global.cg.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
     return v;
 }
+__device__ __forceinline__ uint2 ldg_act8_pred(const void *p, bool pred) {
+    uint2 v;
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %3, 0;\n\tmov.u32 %0, 0;\n\tmov.u32 %1, 0;\n\t"
+                 "@q ld.global.cg.v2.u32 {%0,%1}, [%2];\n\t}"
+                 : "=&r"(v.x), "=&r"(v.y) : "l"(p), "r"((uint32_t)pred));
+    return v;
+}
 __device__ __forceinline__ float ldg_cg_f32(const float *p) {
     float v;
     asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
