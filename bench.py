@@ -138,6 +138,19 @@ def workload_name(cfg):
             f"gamma {cfg.g_min}..{cfg.g_max}")
 
 
+def aggregate_replicas(dev_ms, wall, tokens, bytes_total, world, device):
+    """Replicas share nothing: the job's time is the slowest rank's, its tokens and bytes are the sums."""
+    if world <= 1:
+        return dev_ms, wall, float(tokens), float(bytes_total)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([dev_ms, wall], dtype=torch.float64, device=device)
+    u = torch.tensor([float(tokens), float(bytes_total)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t[0]), float(t[1]), float(u[0]), float(u[1])
+
+
 def run_ours(a):
     import torch
     import paper_2504_05598_b200 as dl
@@ -200,14 +213,7 @@ def run_ours(a):
     dev_ms = ev0.elapsed_time(ev1)
     launches = ctx.launch_count() - launches0
     h2d1, d2h1 = ctx.traffic()
-    t = torch.tensor([dev_ms, float(tokens), bytes_total, wall], dtype=torch.float64, device=dev)
-    if world > 1:
-        tmax = t.clone()
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        tsum = t.clone()
-        dist.all_reduce(tsum, op=dist.ReduceOp.SUM)
-        dev_ms, wall = float(tmax[0]), float(tmax[3])
-        tokens, bytes_total = float(tsum[1]), float(tsum[2])
+    dev_ms, wall, tokens, bytes_total = aggregate_replicas(dev_ms, wall, tokens, bytes_total, world, dev)
     value = tokens / (dev_ms / 1000.0)
 
     # ---- vanilla (gamma = 0) rounds on the same kernels, for the speculative speed-up on this model

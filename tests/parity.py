@@ -202,3 +202,31 @@ def run_sequence(ctx, seq, ref: SeqRef, total_tokens: int, policy=None, max_roun
         if len(rep.failures) > 20:
             break
     return rep
+
+
+def run_batch(ctx, refs: List[SeqRef], total_tokens: int, max_rounds=None) -> List[Report]:
+    """All sequences of a batch through shared del_round calls, each compared with its own oracle trace."""
+    n = len(refs)
+    reps = [Report() for _ in refs]
+    for s in range(n):
+        compare_init(ctx, s, refs[s], total_tokens, reps[s])
+    done, k = [1] * n, [0] * n
+    calls = 0
+    while any(k[s] < len(refs[s].rounds) for s in range(n)):
+        if max_rounds is not None and calls >= max_rounds:
+            break
+        outs = ctx.round()
+        calls += 1
+        for s in range(n):
+            if k[s] >= len(refs[s].rounds):
+                continue
+            r = refs[s].rounds[k[s]]
+            need = compare_round(ctx, s, outs[s], r, reps[s])
+            done[s] += r.n + 1
+            k[s] += 1
+            if need and k[s] < len(refs[s].rounds):
+                reps[s].resyncs += 1
+                _resync(ctx, s, refs[s], done[s], r.Sc, r.Sn, r.next_E, r.next_gamma, total_tokens)
+        if sum(len(rp.failures) for rp in reps) > 20:
+            break
+    return reps

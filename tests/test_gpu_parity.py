@@ -7,7 +7,7 @@ import pytest
 
 import synth
 from cases import TINY, TINY_GQA, TINY_SHORT
-from parity import MARGIN, ref_from_golden, ref_from_oracle, run_sequence
+from parity import MARGIN, ref_from_golden, ref_from_oracle, run_batch, run_sequence
 
 pytestmark = pytest.mark.gpu
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
@@ -189,7 +189,7 @@ def test_batch_of_independent_sequences():
             assert got[s] == refs[s].tokens
 
 
-@pytest.mark.parametrize("name,max_rounds", [("llama2_7b", None), ("llama32_1b", 60)])
+@pytest.mark.parametrize("name,max_rounds", [("llama2_7b", None), ("llama32_1b", 60), ("llama2_13b", 24)])
 def test_full_size_config_against_stored_trace(name, max_rounds):
     """The benchmark shapes, in the configuration bench.py times, against the oracle's stored trace."""
     path = os.path.join(GOLDEN, f"trace_{name}.json")
@@ -234,3 +234,22 @@ def test_streaming_lm_head_full_size():
     rep = run_sequence(ctx, 0, ref, doc["gen_len"], max_rounds=40)
     print(f"{name} (streaming head): rounds {rep.rounds} compared {rep.compared} flips {rep.flips} resyncs {rep.resyncs}")
     assert rep.ok(), rep.failures[:8]
+
+
+def test_full_size_batch_of_four_against_stored_trace():
+    """Llama-3-8B shape, four sequences with their own (E, gamma) state and paged KV, lock-step rounds."""
+    name = "llama3_8b_b4"
+    path = os.path.join(GOLDEN, f"trace_{name}.json")
+    if not os.path.exists(path):
+        pytest.skip("no stored trace")
+    doc = json.load(open(path))
+    cfg = synth.CONFIGS[name]
+    assert doc["seed"] == cfg.seed and len(doc["sequences"]) == cfg.batch
+    w = synth.make_weights(cfg)
+    ctx = make_ctx(cfg, w)
+    refs = [ref_from_golden(doc, s, synth.make_prompt(cfg, s)) for s in range(cfg.batch)]
+    reps = run_batch(ctx, refs, doc["gen_len"])
+    for s, rep in enumerate(reps):
+        print(f"{name} seq {s}: rounds {rep.rounds} compared {rep.compared} flips {rep.flips} resyncs {rep.resyncs}")
+        assert rep.ok(), (s, rep.failures[:8])
+        assert rep.rounds == len(refs[s].rounds)
