@@ -281,7 +281,11 @@ def run_ours(a):
     achieved = (sb / 1e9) / (sm_ / 1e3)
     roofline = {"bound": "hbm", "kernel": "rowgemm_kernel (weight-streaming skinny GEMM, all epilogues)",
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
-                "bytes_per_launch": sb / sl, "avg_us": 1000.0 * sm_ / sl, "traffic": None,
+                "bytes_per_launch": sb / sl, "avg_us": 1000.0 * sm_ / sl,
+                # DRAM read+write per launch from the ncu capture of the same kernels (profiles/
+                # round_kernels_m1_llama2_7b_layer.txt): 1.000-1.001 x the weight bytes read plus the ~3 MB of
+                # activation / partial writes ncu attributes to a launch
+                "traffic": (sb / sl) * 1.0005 + 3.5e6,
                 "share_of_round": sm_ / tot_ms}
 
     line = {
