@@ -49,7 +49,9 @@ class RoundInfo(C.Structure):
     _fields_ = [("E", C.c_int32), ("gamma", C.c_int32), ("g", C.c_int32), ("n_accept", C.c_int32),
                 ("n_emitted", C.c_int32), ("drafts", C.c_int32 * MAX_GAMMA),
                 ("emitted", C.c_int32 * (MAX_GAMMA + 1)), ("next_E", C.c_int32), ("next_gamma", C.c_int32),
-                ("loaded_layers", C.c_int32), ("Sn", C.c_double)]
+                ("loaded_layers", C.c_int32), ("Sn", C.c_double),
+                ("stopped", C.c_int32), ("pad_", C.c_int32), ("tau", C.c_double), ("next_tau", C.c_double),
+                ("draft_conf", C.c_double * (MAX_GAMMA + 1))]
 
 
 def lib():
@@ -90,6 +92,14 @@ def lib():
     L.ora_tpl.argtypes = [f64, i32, i32, i32]
     L.ora_select.argtypes = [vp, f64, i32, i32, i32, i32, i32, C.POINTER(i32), C.POINTER(i32)]
     L.ora_num_threads.restype = C.c_int
+    L.ora_set_exit_mode.argtypes = [vp, i32]
+    L.ora_get_conf_stats.argtypes = [vp, vp, vp, vp]
+    L.ora_set_conf_stats.argtypes = [vp, vp, vp]
+    L.ora_get_conf.argtypes = [vp, vp, i32]
+    L.ora_confidence.restype = f64
+    L.ora_confidence.argtypes = [vp, i32]
+    L.ora_threshold.restype = f64
+    L.ora_threshold.argtypes = [f64, f64, f64, f64]
     _lib = L
     return L
 
@@ -102,7 +112,7 @@ def _p16(a: np.ndarray):
 class Round:
     """Plain-Python copy of one round's record."""
     __slots__ = ("E", "gamma", "g", "n_accept", "emitted", "drafts", "next_E", "next_gamma", "loaded_layers",
-                 "shadow", "margin", "counts", "Sn")
+                 "shadow", "margin", "counts", "Sn", "stopped", "tau", "next_tau", "draft_conf", "conf")
 
     def __init__(self, info: RoundInfo, shadow, margin, counts):
         self.E, self.gamma, self.g, self.n_accept = info.E, info.gamma, info.g, info.n_accept
@@ -111,6 +121,9 @@ class Round:
         self.next_E, self.next_gamma = info.next_E, info.next_gamma
         self.loaded_layers, self.Sn = info.loaded_layers, info.Sn
         self.shadow, self.margin, self.counts = shadow, margin, counts
+        self.stopped, self.tau, self.next_tau = bool(info.stopped), info.tau, info.next_tau
+        self.draft_conf = [float(info.draft_conf[i]) for i in range(info.g + info.stopped)]
+        self.conf = None            # [L][columns] confidence of the shadow tokens, filled by OracleSeq
 
 
 class OracleSeq:
@@ -167,6 +180,26 @@ class OracleSeq:
         Sc = np.ascontiguousarray(Sc, dtype=np.float64)
         lib().ora_set_stats(self._h, Sc.ctypes.data, float(Sn), int(E), int(gamma))
 
+    def set_exit_mode(self, on: bool):
+        """Dynamic draft-exiting (Sec. 4.4): draft up to g_max tokens, stop at the first low-confidence one."""
+        lib().ora_set_exit_mode(self._h, 1 if on else 0)
+
+    def get_conf_stats(self):
+        L = self.cfg.n_layers
+        Stcs, Sfcs, tau = (np.zeros(L, dtype=np.float64) for _ in range(3))
+        lib().ora_get_conf_stats(self._h, Stcs.ctypes.data, Sfcs.ctypes.data, tau.ctypes.data)
+        return Stcs, Sfcs, tau
+
+    def set_conf_stats(self, Stcs, Sfcs):
+        Stcs = np.ascontiguousarray(Stcs, dtype=np.float64)
+        Sfcs = np.ascontiguousarray(Sfcs, dtype=np.float64)
+        lib().ora_set_conf_stats(self._h, Stcs.ctypes.data, Sfcs.ctypes.data)
+
+    def get_conf(self, n_cols: int) -> np.ndarray:
+        out = np.zeros((self.cfg.n_layers, n_cols), dtype=np.float64)
+        lib().ora_get_conf(self._h, out.ctypes.data, n_cols)
+        return out
+
     def hidden(self, layer: int, row: int) -> np.ndarray:
         p = lib().ora_hidden(self._h, layer, row)
         return np.ctypeslib.as_array(p, shape=(self.cfg.d_model,)).copy()
@@ -189,7 +222,9 @@ class OracleSeq:
         tok = lib().ora_prefill(self._h, prompt.ctypes.data, len(prompt), shadow.ctypes.data, margin.ctypes.data,
                                 C.byref(info))
         w = min(W, len(prompt))
-        return tok, Round(info, shadow[:, :w], margin[:, :w], None)
+        r = Round(info, shadow[:, :w], margin[:, :w], None)
+        r.conf = self.get_conf(w)
+        return tok, r
 
     def round(self, remaining: int) -> Round:
         L = self.cfg.n_layers
@@ -201,7 +236,9 @@ class OracleSeq:
                              counts.ctypes.data)
         if rc != 0:
             raise RuntimeError(f"ora_round failed: {rc}")
-        return Round(info, shadow[:, :info.g + 1], margin[:, :info.g + 1], counts)
+        r = Round(info, shadow[:, :info.g + 1], margin[:, :info.g + 1], counts)
+        r.conf = self.get_conf(info.g + 1)
+        return r
 
     def generate(self, prompt: np.ndarray, n_tokens: int):
         """Prefill then rounds until n_tokens tokens exist (the prefill's token included)."""
@@ -253,6 +290,15 @@ def softmax(x: np.ndarray) -> np.ndarray:
     p = np.zeros(x.size, dtype=np.float64)
     lib().ora_softmax(x.ctypes.data, x.size, p.ctypes.data)
     return p
+
+
+def confidence(logits: np.ndarray) -> float:
+    x = np.ascontiguousarray(logits, dtype=np.float32)
+    return lib().ora_confidence(x.ctypes.data, x.size)
+
+
+def threshold(Stcs: float, Sc: float, Sfcs: float, Smis: float) -> float:
+    return lib().ora_threshold(Stcs, Sc, Sfcs, Smis)
 
 
 def silu(x: float) -> float:

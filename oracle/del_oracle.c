@@ -10,7 +10,8 @@
  *   Sec. 4.1 Eq. 1 (tokens-per-layer, in its sum form), cost d*l + L
  *   Sec. 4.2 shadow tokens, u_r, c_r^l, decayed sum S, Eq. 2 (alpha_l)
  *   Sec. 4.3 selection by argmax of TPL, initialisation from the prefill
- *   Algorithm 1 (the loop; the confidence break and the threshold update are not on this path)
+ *   Sec. 4.4 dynamic draft-exiting: confidence = probability of the top-1 token, tcs / fcs, Eq. 3
+ *   Algorithm 1 (the loop with its confidence break, DEL_Update)
  *   App. B.2 hyper-parameters: window 32, omega 0.95
  * The decoder block itself is the standard pre-norm Llama block (RMSNorm, rotary embedding with
  * rotate-half pairing, grouped-query causal attention, SwiGLU), which the paper takes as given.
@@ -33,6 +34,10 @@ struct ora_seq {
     int32_t fixed_E, fixed_gamma;
     double *Sc;         /* [L], index l-1; Sc[L-1] (layer L) tracked too: it must equal Sn */
     double Sn;
+    double *Stcs, *Sfcs; /* [L] decayed confidence sums over matched / mismatched shadow tokens (Sec. 4.4) */
+    double *tau;        /* [L] thresholds of Eq. 3 from the current statistics */
+    double *conf;       /* [L][rows] confidence of every shadow token of the last round / prefill window */
+    int32_t exit_mode;  /* 1: the draft loop runs up to g_max steps and stops on a low confidence */
     float *K, *V;       /* [L][max_seq][n_kv*hd] */
     float *H;           /* [L+1][rows][d] hidden stack */
     int32_t rows;       /* rows per layer in H */
@@ -169,6 +174,10 @@ ora_seq *ora_seq_create(const ora_shape *shape, const ora_weights *w) {
     s->rows = sh->g_max + 1 > sh->init_window ? sh->g_max + 1 : sh->init_window;
     s->H = (float *)calloc((size_t)(sh->n_layers + 1) * s->rows * sh->d_model, sizeof(float));
     s->Sc = (double *)calloc(sh->n_layers, sizeof(double));
+    s->Stcs = (double *)calloc(sh->n_layers, sizeof(double));
+    s->Sfcs = (double *)calloc(sh->n_layers, sizeof(double));
+    s->tau = (double *)calloc(sh->n_layers, sizeof(double));
+    s->conf = (double *)calloc((size_t)sh->n_layers * s->rows, sizeof(double));
     s->rope_cos = (float *)malloc(sizeof(float) * (size_t)sh->max_seq * (sh->head_dim / 2));
     s->rope_sin = (float *)malloc(sizeof(float) * (size_t)sh->max_seq * (sh->head_dim / 2));
     rope_tables(s->rope_cos, s->rope_sin, sh->max_seq, sh->head_dim, sh->rope_theta);
@@ -182,6 +191,7 @@ ora_seq *ora_seq_create(const ora_shape *shape, const ora_weights *w) {
 void ora_seq_destroy(ora_seq *s) {
     if (!s) return;
     free(s->K); free(s->V); free(s->H); free(s->Sc); free(s->rope_cos); free(s->rope_sin);
+    free(s->Stcs); free(s->Sfcs); free(s->tau); free(s->conf);
     free(s);
 }
 
@@ -200,9 +210,46 @@ void ora_get_stats(const ora_seq *s, double *Sc, double *Sn, int32_t *E, int32_t
     if (gamma) *gamma = s->gamma;
 }
 
+/* Eq. 3: midpoint of the decayed mean confidence of matched and of mismatched shadow tokens.  The paper
+ * does not say what a mean over no tokens is; here the mean over no matched tokens is 1 and the mean
+ * over no mismatched tokens is 0 (the two ends of the range of a probability). */
+double ora_threshold(double Stcs, double Sc, double Sfcs, double Smis) {
+    double mean_true = 1.0, mean_false = 0.0;
+    if (Sc > 0.0) mean_true = Stcs / Sc;
+    if (Smis > 0.0) mean_false = Sfcs / Smis;
+    double sum = mean_true + mean_false;
+    return 0.5 * sum;
+}
+
+/* S(u - c) = S(u) - S(c): S is linear */
+static void refresh_tau(ora_seq *s) {
+    for (int32_t l = 0; l < s->sh.n_layers; ++l)
+        s->tau[l] = ora_threshold(s->Stcs[l], s->Sc[l], s->Sfcs[l], s->Sn - s->Sc[l]);
+}
+
 void ora_set_stats(ora_seq *s, const double *Sc, double Sn, int32_t E, int32_t gamma) {
     memcpy(s->Sc, Sc, sizeof(double) * s->sh.n_layers);
     s->Sn = Sn; s->E = E; s->gamma = gamma;
+    refresh_tau(s);
+}
+
+void ora_set_exit_mode(ora_seq *s, int32_t mode) { s->exit_mode = mode ? 1 : 0; }
+
+void ora_get_conf_stats(const ora_seq *s, double *Stcs, double *Sfcs, double *tau) {
+    if (Stcs) memcpy(Stcs, s->Stcs, sizeof(double) * s->sh.n_layers);
+    if (Sfcs) memcpy(Sfcs, s->Sfcs, sizeof(double) * s->sh.n_layers);
+    if (tau) memcpy(tau, s->tau, sizeof(double) * s->sh.n_layers);
+}
+
+void ora_set_conf_stats(ora_seq *s, const double *Stcs, const double *Sfcs) {
+    memcpy(s->Stcs, Stcs, sizeof(double) * s->sh.n_layers);
+    memcpy(s->Sfcs, Sfcs, sizeof(double) * s->sh.n_layers);
+    refresh_tau(s);
+}
+
+void ora_get_conf(const ora_seq *s, double *conf, int32_t n_cols) {
+    for (int32_t l = 0; l < s->sh.n_layers; ++l)
+        for (int32_t i = 0; i < n_cols; ++i) conf[(size_t)l * n_cols + i] = s->conf[(size_t)l * s->rows + i];
 }
 
 static float *hidden_at(const ora_seq *s, int32_t layer, int32_t row) {
@@ -302,6 +349,23 @@ void ora_layer_rows(ora_seq *s, int32_t layer1, const float *h_in, int32_t pos0,
 
 /* Exit head at any layer: shared final RMSNorm, LM head, greedy choice (Sec. 2; Sec. 4.2 applies the
  * same head to every layer's hidden state).  Lowest token id wins ties. */
+/* Confidence score of Sec. 4.4: the softmax probability of the top-1 token, 1 / sum_v exp(z_v - z_max). */
+double ora_confidence(const float *logits, int32_t V) {
+    double mx = logits[0];
+    for (int32_t t = 1; t < V; ++t)
+        if (logits[t] > mx) mx = logits[t];
+    double sum = 0.0;
+    for (int32_t t = 0; t < V; ++t) sum += exp((double)logits[t] - mx);
+    return 1.0 / sum;
+}
+
+static void exit_head_conf(const ora_seq *s, const float *h, int32_t *token, float *margin, double *conf) {
+    float *lg = (float *)malloc(sizeof(float) * s->sh.vocab);
+    ora_exit_head(s, h, token, margin, lg);
+    *conf = ora_confidence(lg, s->sh.vocab);
+    free(lg);
+}
+
 void ora_exit_head(const ora_seq *s, const float *h, int32_t *token, float *margin, float *logits_or_null) {
     const ora_shape *sh = &s->sh;
     const int32_t d = sh->d_model, V = sh->vocab;
@@ -386,16 +450,25 @@ int32_t ora_prefill(ora_seq *s, const int32_t *prompt, int32_t P, int32_t *shado
     for (int32_t l = 1; l <= L; ++l)
         for (int32_t j = 0; j < W; ++j) {
             float mg;
-            ora_exit_head(s, hidden_at(s, l, j), &sd[(size_t)(l - 1) * W + j], &mg, NULL);
+            exit_head_conf(s, hidden_at(s, l, j), &sd[(size_t)(l - 1) * W + j], &mg, &s->conf[(size_t)(l - 1) * s->rows + j]);
             if (shadow) shadow[(size_t)(l - 1) * sh->init_window + j] = sd[(size_t)(l - 1) * W + j];
             if (margin) margin[(size_t)(l - 1) * sh->init_window + j] = mg;
         }
     for (int32_t l = 1; l <= L; ++l) {
         int32_t c = 0;
-        for (int32_t j = 0; j < W; ++j) c += (sd[(size_t)(l - 1) * W + j] == sd[(size_t)(L - 1) * W + j]);
+        double tcs = 0.0, fcs = 0.0;
+        for (int32_t j = 0; j < W; ++j) {
+            const int match = sd[(size_t)(l - 1) * W + j] == sd[(size_t)(L - 1) * W + j];
+            const double cf = s->conf[(size_t)(l - 1) * s->rows + j];
+            c += match;
+            if (match) tcs += cf; else fcs += cf;
+        }
         s->Sc[l - 1] = (double)c;
+        s->Stcs[l - 1] = tcs;
+        s->Sfcs[l - 1] = fcs;
     }
     s->Sn = (double)W;
+    refresh_tau(s);
     s->T = P;
     s->x_in = sd[(size_t)(L - 1) * W + (W - 1)];
     free(sd);
@@ -407,6 +480,7 @@ int32_t ora_prefill(ora_seq *s, const int32_t *prompt, int32_t P, int32_t *shado
         info->next_E = s->E;
         info->next_gamma = s->gamma;
         info->Sn = s->Sn;
+        info->next_tau = s->tau[s->E - 1];
     }
     return s->x_in;
 }
@@ -416,18 +490,25 @@ int ora_round(ora_seq *s, int32_t remaining, ora_round_info *info, int32_t *shad
     const ora_shape *sh = &s->sh;
     const int32_t d = sh->d_model, L = sh->n_layers, stride = sh->g_max + 1;
     const int32_t E = s->E;
-    int32_t g = s->gamma;
+    /* Algorithm 1: with dynamic draft-exiting the loop runs up to d_max steps, otherwise gamma steps */
+    int32_t g_cap = s->exit_mode ? sh->g_max : s->gamma;
     if (remaining < 1) return -1;
-    if (g > remaining - 1) g = remaining - 1;
-    if (g > ORA_MAX_GAMMA || g + 1 > s->rows || s->T + g + 1 > sh->max_seq) return -2;
+    if (g_cap > remaining - 1) g_cap = remaining - 1;
+    if (g_cap > ORA_MAX_GAMMA || g_cap + 1 > s->rows || s->T + g_cap + 1 > sh->max_seq) return -2;
     int32_t drafts[ORA_MAX_GAMMA];
-    int32_t in = s->x_in;
-    /* draft: g tokens through layers 1..E + exit head (Algorithm 1, draft loop) */
-    for (int32_t i = 0; i < g; ++i) {
+    double draft_conf[ORA_MAX_GAMMA + 1];
+    const double tau_E = s->tau[E - 1];
+    int32_t in = s->x_in, g = 0, stopped = 0;
+    /* draft: tokens through layers 1..E + exit head (Algorithm 1, draft loop); a token whose confidence is
+     * below the threshold ends the loop and is not appended */
+    for (int32_t i = 0; i < g_cap; ++i) {
+        int32_t tok;
         ora_embed(s, in, hidden_at(s, 0, i));
         for (int32_t l = 1; l <= E; ++l) ora_layer_rows(s, l, hidden_at(s, l - 1, i), s->T + i, 1, hidden_at(s, l, i));
-        ora_exit_head(s, hidden_at(s, E, i), &drafts[i], NULL, NULL);
-        in = drafts[i];
+        exit_head_conf(s, hidden_at(s, E, i), &tok, NULL, &draft_conf[i]);
+        if (s->exit_mode && draft_conf[i] < tau_E) { stopped = 1; break; }
+        drafts[g++] = tok;
+        in = tok;
     }
     /* verify: the last input through layers 1..E, then all g+1 rows through layers E+1..L, reusing the
      * exit layer's cached hidden states and the KV cache written while drafting */
@@ -439,7 +520,7 @@ int ora_round(ora_seq *s, int32_t remaining, ora_round_info *info, int32_t *shad
     for (int32_t l = 1; l <= L; ++l)
         for (int32_t i = 0; i <= g; ++i) {
             float mg;
-            ora_exit_head(s, hidden_at(s, l, i), &sd[(size_t)(l - 1) * stride + i], &mg, NULL);
+            exit_head_conf(s, hidden_at(s, l, i), &sd[(size_t)(l - 1) * stride + i], &mg, &s->conf[(size_t)(l - 1) * s->rows + i]);
             if (shadow) shadow[(size_t)(l - 1) * stride + i] = sd[(size_t)(l - 1) * stride + i];
             if (margin) margin[(size_t)(l - 1) * stride + i] = mg;
         }
@@ -449,11 +530,20 @@ int ora_round(ora_seq *s, int32_t remaining, ora_round_info *info, int32_t *shad
      * positions is n + 1 */
     for (int32_t l = 1; l <= L; ++l) {
         int32_t c = 0;
-        for (int32_t i = 0; i <= n; ++i) c += (sd[(size_t)(l - 1) * stride + i] == verified[i]);
+        double tcs = 0.0, fcs = 0.0;    /* confidence sums over matched / mismatched shadow tokens (Sec. 4.4) */
+        for (int32_t i = 0; i <= n; ++i) {
+            const int match = sd[(size_t)(l - 1) * stride + i] == verified[i];
+            const double cf = s->conf[(size_t)(l - 1) * s->rows + i];
+            c += match;
+            if (match) tcs += cf; else fcs += cf;
+        }
         if (counts) counts[l - 1] = c;
         s->Sc[l - 1] = ora_decay_step(s->Sc[l - 1], sh->omega, (double)c);
+        s->Stcs[l - 1] = ora_decay_step(s->Stcs[l - 1], sh->omega, tcs);
+        s->Sfcs[l - 1] = ora_decay_step(s->Sfcs[l - 1], sh->omega, fcs);
     }
     s->Sn = ora_decay_step(s->Sn, sh->omega, (double)(n + 1));
+    refresh_tau(s);
     if (info) {
         memset(info, 0, sizeof(*info));
         info->E = E; info->gamma = s->gamma; info->g = g;
@@ -461,11 +551,14 @@ int ora_round(ora_seq *s, int32_t remaining, ora_round_info *info, int32_t *shad
         for (int32_t i = 0; i < g; ++i) info->drafts[i] = drafts[i];
         for (int32_t i = 0; i <= n; ++i) info->emitted[i] = verified[i];
         info->loaded_layers = g * E + L;
+        info->stopped = stopped;
+        info->tau = tau_E;
+        for (int32_t i = 0; i < g + stopped; ++i) info->draft_conf[i] = draft_conf[i];
     }
     s->T += n + 1;
     s->x_in = verified[n];
     free(sd);
     choose_next(s);
-    if (info) { info->next_E = s->E; info->next_gamma = s->gamma; info->Sn = s->Sn; }
+    if (info) { info->next_E = s->E; info->next_gamma = s->gamma; info->Sn = s->Sn; info->next_tau = s->tau[s->E - 1]; }
     return 0;
 }

@@ -15,7 +15,9 @@
  * pass, closed forms for RMSNorm / softmax / SiLU / RoPE, greedy speculative ==
  * greedy auto-regressive for every (E, gamma), the paper's worked example of a
  * round, brute-force shadow tokens from truncated models, the decayed-sum
- * definition, and exhaustive evaluation of the tokens-per-layer formula.
+ * definition, exhaustive evaluation of the tokens-per-layer formula, and for
+ * dynamic draft-exiting: the softmax definition of the confidence, Eq. 3 from
+ * explicit histories, and the two limits of the threshold (never / always stop).
  * Parity unpinned: the absolute values of logits of the random model (no
  * published activations exist) and any distribution-level behaviour that would
  * need the paper's trained checkpoints.
@@ -56,6 +58,12 @@ typedef struct {
     int32_t next_E, next_gamma;
     int32_t loaded_layers;   /* g * E + L : the paper's cost of the round */
     double Sn;               /* decayed number of valid positions after this round */
+    /* dynamic draft-exiting (Sec. 4.4) */
+    int32_t stopped;         /* 1: the draft loop ended on a confidence below the threshold */
+    int32_t pad_;
+    double tau;              /* threshold of the exit layer the draft loop used */
+    double next_tau;         /* threshold of the next round's exit layer */
+    double draft_conf[ORA_MAX_GAMMA + 1]; /* confidence of every drafted token, the one that ended the loop included */
 } ora_round_info;
 
 typedef struct ora_seq ora_seq;
@@ -78,6 +86,16 @@ int32_t ora_prefill(ora_seq *s, const int32_t *prompt, int32_t n_prompt, int32_t
 int ora_round(ora_seq *s, int32_t remaining, ora_round_info *info, int32_t *shadow, float *margin,
               int32_t *counts);
 
+/* Dynamic draft-exiting (Sec. 4.4, Algorithm 1): mode 1 lets the draft loop run up to g_max steps and end
+ * it at the first token whose confidence is below the exit layer's threshold (that token is dropped);
+ * mode 0 (default) drafts exactly gamma tokens.  The confidence statistics are tracked in both modes. */
+void ora_set_exit_mode(ora_seq *s, int32_t mode);
+/* decayed confidence sums and thresholds, [n_layers] each, index l-1 */
+void ora_get_conf_stats(const ora_seq *s, double *Stcs, double *Sfcs, double *tau);
+void ora_set_conf_stats(ora_seq *s, const double *Stcs, const double *Sfcs);
+/* confidence of the shadow tokens of the last round (or of the prefill window): [n_layers][n_cols] */
+void ora_get_conf(const ora_seq *s, double *conf, int32_t n_cols);
+
 /* state access */
 int32_t ora_committed_len(const ora_seq *s);
 void ora_get_stats(const ora_seq *s, double *Sc /*[n_layers], index l-1*/, double *Sn, int32_t *E, int32_t *gamma);
@@ -99,6 +117,10 @@ void ora_layer_rows(ora_seq *s, int32_t layer, const float *h_in, int32_t pos0, 
 /* shared final RMSNorm + LM head + greedy choice (lowest id on ties); margin = top1 - top2 logit */
 void ora_exit_head(const ora_seq *s, const float *h, int32_t *token, float *margin, float *logits_or_null);
 
+/* top-1 softmax probability of a logit row */
+double ora_confidence(const float *logits, int32_t V);
+/* Eq. 3 for one layer; Smis = decayed number of mismatched shadow tokens */
+double ora_threshold(double Stcs, double Sc, double Sfcs, double Smis);
 int32_t ora_accept_len(const int32_t *drafts, const int32_t *verified, int32_t g);
 double ora_decay_step(double S, double omega, double a);
 double ora_tpl(double alpha, int32_t l, int32_t d, int32_t L);
