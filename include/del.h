@@ -10,7 +10,9 @@
  *   Sec. 4.2: run the LM head over every layer's cached hidden states of the round ("shadow tokens"),
  *          count matches with the target's tokens inside the valid context, keep decayed sums;
  *   Sec. 4.1 (Eq. 1) and Sec. 4.3: pick the next (E, gamma) maximising expected tokens per loaded layer;
- *   Algorithm 1: the loop (without its confidence-threshold early break).
+ *   Sec. 4.4 and Eq. 3: confidence of a token = its softmax probability; decayed confidence sums over
+ *          matched and mismatched shadow tokens give each layer a threshold;
+ *   Algorithm 1: the loop, with its confidence break when a sequence is in exit mode (del_set_exit_mode).
  *
  * Conventions
  *   - Plain C ABI.  Every pointer is either HOST or DEVICE memory as stated per field/argument.
@@ -103,6 +105,9 @@ typedef struct {
     int32_t tokens[DEL_MAX_GAMMA + 1];   /* the n_emitted tokens committed by the round */
     int32_t next_E, next_gamma;   /* choice for the next round */
     int32_t status;               /* 0, or a DEL_E* code reported by a kernel */
+    int32_t stopped;              /* 1: the draft loop ended on a confidence below tau (that token was dropped) */
+    double tau;                   /* threshold of layer E the draft loop compared with (exit mode), else 0 */
+    double next_tau;              /* Eq. 3 for layer next_E from the updated statistics */
 } del_round_out;
 
 /* Bytes of DEVICE workspace del_init needs for this shape (256-byte aligned base expected). */
@@ -158,6 +163,26 @@ int del_round(del_ctx *ctx, del_round_out *out);
 /* Fix the policy of a sequence: del_round uses (E, gamma) as given instead of the selection
  * (gamma = 0: plain auto-regressive decoding).  E <= 0 restores the dynamic choice. */
 int del_set_policy(del_ctx *ctx, int seq, int E, int gamma);
+
+/* Dynamic draft-exiting (Sec. 4.4, Algorithm 1) for a sequence: mode 1 lets the draft loop run for up to
+ * g_max tokens (del_round) or the given gamma (del_draft) and ends it at the first token whose
+ * confidence (top-1 softmax probability of the exit head, fp32) is below the threshold of layer E from
+ * Eq. 3; that token is not appended, and its pass through layers 1..E is reused by the verify phase.
+ * The host checks the confidence after every draft step, so a round then costs one synchronisation
+ * per drafted token instead of one per round.  mode 0 (default) drafts exactly gamma tokens.  The
+ * confidence statistics and thresholds are maintained in both modes. */
+int del_set_exit_mode(del_ctx *ctx, int seq, int mode);
+
+/* Confidence statistics (Sec. 4.4).  HOST double [n_layers] each, entry l-1 for layer l: decayed sums of
+ * the confidences of matched / mismatched shadow tokens, and the thresholds of Eq. 3 (a mean over no
+ * tokens counts as 1 for matched and 0 for mismatched ones).  Any pointer of the getter may be NULL.
+ * Synchronise. */
+int del_get_conf_stats(del_ctx *ctx, int seq, double *Stcs, double *Sfcs, double *tau);
+int del_set_conf_stats(del_ctx *ctx, int seq, const double *Stcs, const double *Sfcs);
+/* Confidences of the last round: shadow_conf fp32 [n_layers][g_max + 1] (shadow tokens of
+ * del_layer_accept), draft_conf fp32 [g_max + 1] (draft i at entry i, the dropped one included).
+ * HOST, either may be NULL.  Synchronises. */
+int del_get_conf(del_ctx *ctx, int seq, float *shadow_conf, float *draft_conf);
 
 /* Acceptance statistics, for resuming and for tests.  Sc: HOST double [n_layers], entry l-1 is the
  * decayed match count of layer l; Sn: decayed number of valid positions.  Synchronise. */

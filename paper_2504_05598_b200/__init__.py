@@ -27,7 +27,8 @@ KERNEL_CLASSES = ["qkv_rope", "attention", "o_proj", "gate_up", "down", "lm_head
 EXPORTS = ["del_workspace_bytes", "del_init", "del_prefill", "del_draft", "del_verify", "del_layer_accept",
            "del_select", "del_round", "del_set_policy", "del_get_stats", "del_set_stats", "del_get_shadow",
            "del_get_drafts", "del_force_token", "del_get_hidden", "del_debug_logits", "del_get_kv", "del_committed_len", "del_release",
-           "del_launch_count", "del_get_traffic", "del_set_flags", "del_get_kernel_times", "del_head_argmax_static", "del_strerror", "del_last_cuda_error", "del_destroy"]
+           "del_launch_count", "del_get_traffic", "del_set_flags", "del_get_kernel_times", "del_head_argmax_static",
+           "del_set_exit_mode", "del_get_conf_stats", "del_set_conf_stats", "del_get_conf", "del_strerror", "del_last_cuda_error", "del_destroy"]
 
 
 class Shape(C.Structure):
@@ -52,7 +53,8 @@ class KvC(C.Structure):
 class RoundOut(C.Structure):
     _fields_ = [("E", C.c_int32), ("gamma", C.c_int32), ("g", C.c_int32), ("n_accept", C.c_int32),
                 ("n_emitted", C.c_int32), ("tokens", C.c_int32 * (MAX_GAMMA + 1)), ("next_E", C.c_int32),
-                ("next_gamma", C.c_int32), ("status", C.c_int32)]
+                ("next_gamma", C.c_int32), ("status", C.c_int32), ("stopped", C.c_int32),
+                ("tau", C.c_double), ("next_tau", C.c_double)]
 
     def emitted(self) -> List[int]:
         return [int(self.tokens[i]) for i in range(self.n_emitted)]
@@ -94,6 +96,14 @@ def load_library(build_if_missing: bool = True):
     L.del_get_stats.argtypes = [vp, ci, vp, C.POINTER(C.c_double), C.POINTER(i32), C.POINTER(i32)]
     L.del_set_stats.restype = ci
     L.del_set_stats.argtypes = [vp, ci, vp, C.c_double, i32, i32]
+    L.del_set_exit_mode.restype = ci
+    L.del_set_exit_mode.argtypes = [vp, ci, ci]
+    L.del_get_conf_stats.restype = ci
+    L.del_get_conf_stats.argtypes = [vp, ci, vp, vp, vp]
+    L.del_set_conf_stats.restype = ci
+    L.del_set_conf_stats.argtypes = [vp, ci, vp, vp]
+    L.del_get_conf.restype = ci
+    L.del_get_conf.argtypes = [vp, ci, vp, vp]
     L.del_get_shadow.restype = ci
     L.del_get_shadow.argtypes = [vp, ci, vp, vp]
     L.del_get_drafts.restype = ci
@@ -262,6 +272,30 @@ class DelContext:
     def set_stats(self, seq: int, Sc, Sn: float, E: int, gamma: int):
         Sc = np.ascontiguousarray(Sc, dtype=np.float64)
         self._ck(self.lib.del_set_stats(self._h, seq, Sc.ctypes.data, float(Sn), int(E), int(gamma)), "del_set_stats")
+
+    def set_exit_mode(self, seq: int, on: bool):
+        """Dynamic draft-exiting: the draft loop stops at the first token whose confidence is below the threshold."""
+        self._ck(self.lib.del_set_exit_mode(self._h, seq, 1 if on else 0), "del_set_exit_mode")
+
+    def get_conf_stats(self, seq: int):
+        L = self.shape.n_layers
+        Stcs, Sfcs, tau = (np.zeros(L, dtype=np.float64) for _ in range(3))
+        self._ck(self.lib.del_get_conf_stats(self._h, seq, Stcs.ctypes.data, Sfcs.ctypes.data, tau.ctypes.data),
+                 "del_get_conf_stats")
+        return Stcs, Sfcs, tau
+
+    def set_conf_stats(self, seq: int, Stcs, Sfcs):
+        Stcs = np.ascontiguousarray(Stcs, dtype=np.float64)
+        Sfcs = np.ascontiguousarray(Sfcs, dtype=np.float64)
+        self._ck(self.lib.del_set_conf_stats(self._h, seq, Stcs.ctypes.data, Sfcs.ctypes.data), "del_set_conf_stats")
+
+    def get_conf(self, seq: int):
+        """(shadow confidences [n_layers][g_max + 1], draft confidences [g_max + 1]) of the last round."""
+        L, G = self.shape.n_layers, self.shape.g_max + 1
+        sc = np.zeros((L, G), dtype=np.float32)
+        dc = np.zeros(G, dtype=np.float32)
+        self._ck(self.lib.del_get_conf(self._h, seq, sc.ctypes.data, dc.ctypes.data), "del_get_conf")
+        return sc, dc
 
     def get_shadow(self, seq: int):
         L, G = self.shape.n_layers, self.shape.g_max + 1

@@ -64,8 +64,16 @@ struct Buffers {
     int32_t *ACNT;               // [DEL_SEQ_MAX][nkv] arrival counters of the split combine
     float *LPV;                  // streaming LM head: arg-max partial values [ctas][ROWS]
     int32_t *LPI;                // ... and indices
+    float *LPS;                  // ... and sums of exp(scaled logit - scaled partial maximum)
+    float *RK;                   // [ROWS] log2(e) / rms of the rows of the last streaming LM-head launch
     float *TPV;                  // tensor-core LM head: partial values [R_max][vocab tiles]
     int32_t *TPI;
+    float *TPS;                  // ... and partial exp sums
+    float *RS;                   // [R_max] log2(e) / rms of the stacked rows
+    float *SSE;                  // [B][S][n_sst] partial sums of squares of h at the exit layer (beside XE)
+    float *DCONF;                // [B][S+1] confidence of draft i at [1 + i] (indexed like TOK)
+    float *SCONF;                // [B][L][S] confidence (top-1 probability) of the shadow tokens
+    double *STCS, *SFCS, *TAU;   // [B][L] decayed confidence sums over matched / mismatched shadow tokens, thresholds
     int32_t *PROMPT_ALL;         // [max_seq] prompt tokens of the sequence being prefilled
     bf16 *XN;                    // [R_max][d] normalised rows for the batched LM head
     int32_t *SHADOW;             // [B][L][S] shadow tokens

@@ -73,6 +73,29 @@ __device__ __forceinline__ void block_argmax(float &v, int &idx) {
     }
 }
 
+// block-wide sum in a fixed order; result valid in thread 0
+__device__ __forceinline__ float block_sum(float v) {
+    __shared__ float ssum[CTL_THREADS / 32];
+    v = warp_sum(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) ssum[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float t = 0.f;
+    if (threadIdx.x == 0)
+        for (int w = 0; w < CTL_THREADS / 32; ++w) t += ssum[w];
+    return t;
+}
+
+// Confidence score (Sec. 4.4: probability of the top-1 token) from partial (maximum, exp sum) pairs:
+// 1 / sum_p s_p * exp2(k * (v_p - M)), M the overall maximum, k = log2(e) / rms of the row.
+__device__ __forceinline__ float merged_confidence(const float *pv, const float *ps, int n_part, size_t pstride, float M, float k) {
+    float acc = 0.f;
+    for (int p = threadIdx.x; p < n_part; p += CTL_THREADS)
+        acc += ldg_cg_f32(ps + (size_t)p * pstride) * exp2f(k * (ldg_cg_f32(pv + (size_t)p * pstride) - M));
+    const float total = block_sum(acc);
+    return 1.f / total;
+}
+
 // Draft head, last step: reduce the per-CTA arg-max partials of the streaming LM head into the draft
 // token, store it, and write the embedding of that token as the next row of the sequence.
 __global__ void __launch_bounds__(CTL_THREADS) draft_finalize_embed_kernel(const __grid_constant__ CtlArgs a, int embed_next) {
@@ -88,12 +111,16 @@ __global__ void __launch_bounds__(CTL_THREADS) draft_finalize_embed_kernel(const
         const int i2 = a.B.LPI[(size_t)p * DEL_ROWS_MAX + c];
         if (v2 > v || (v2 == v && i2 < idx)) { v = v2; idx = i2; }
     }
+    __shared__ float s_max;
     block_argmax(v, idx);
     if (threadIdx.x == 0) {
         s_tok = idx;
+        s_max = v;
         a.B.TOK[rd.seq * (a.D.S + 1) + rd.slot + 1] = idx;
     }
     __syncthreads();
+    const float conf = merged_confidence(a.B.LPV + c, a.B.LPS + c, a.n_part, DEL_ROWS_MAX, s_max, ldg_cg_f32(a.B.RK + c));
+    if (threadIdx.x == 0) a.B.DCONF[rd.seq * (a.D.S + 1) + rd.slot + 1] = conf;
     if (embed_next) write_embedding(a, s_tok, rd.seq, rd.slot + 1);
 }
 
@@ -112,7 +139,8 @@ __device__ __forceinline__ bool locate_row(const UpdatePlan *up, int L, int mode
 }
 
 // Stacked LM head input: row (seq, layer, slot) of the hidden stack times the final norm's gain, as
-// bf16.  The norm's 1/rms is a positive per-row scalar and cannot change the arg-max, so it is left out.
+// bf16.  The norm's 1/rms is a positive per-row scalar and cannot change the arg-max, so it is left out
+// of the product; it is stored (times log2 e) for the confidence score, which does depend on it.
 __global__ void __launch_bounds__(CTL_THREADS) prep_rows_kernel(const CtlArgs a, const UpdatePlan *up) {
     pdl_launch();
     pdl_wait();
@@ -121,13 +149,21 @@ __global__ void __launch_bounds__(CTL_THREADS) prep_rows_kernel(const CtlArgs a,
     const int d = a.D.d;
     const float *h = a.B.H + stack_row(a.D, layer, seq, slot) * d;
     bf16 *x = a.B.XN + (size_t)blockIdx.x * d;
-    for (int o = threadIdx.x; o < d; o += CTL_THREADS) x[o] = __float2bfloat16_rn(ldg_cg_f32(h + o) * bf16_to_f(a.final_gain[o]));
+    float sq = 0.f;
+    for (int o = threadIdx.x; o < d; o += CTL_THREADS) {
+        const float hv = ldg_cg_f32(h + o);
+        x[o] = __float2bfloat16_rn(hv * bf16_to_f(a.final_gain[o]));
+        sq += hv * hv;
+    }
+    const float total = block_sum(sq);
+    if (threadIdx.x == 0) a.B.RS[blockIdx.x] = rsqrtf(total / (float)d + a.D.eps) * 1.4426950408889634f;
 }
 
 // Reduce the vocabulary-tile partials of one stacked row into its shadow token.
 __global__ void __launch_bounds__(CTL_THREADS) shadow_reduce_kernel(const CtlArgs a, const UpdatePlan *up, const float *pv,
-                                                                    const int32_t *pi, int n_part, int pstride, int cstride,
-                                                                    int row_base) {
+                                                                    const int32_t *pi, const float *ps, int n_part, int pstride,
+                                                                    int cstride, int row_base) {
+    __shared__ float s_max;
     pdl_launch();
     pdl_wait();
     const int c = blockIdx.x;
@@ -139,11 +175,33 @@ __global__ void __launch_bounds__(CTL_THREADS) shadow_reduce_kernel(const CtlArg
         if (v2 > v || (v2 == v && i2 < idx)) { v = v2; idx = i2; }
     }
     block_argmax(v, idx);
+    if (threadIdx.x == 0) s_max = v;
+    __syncthreads();
+    const float conf = merged_confidence(pv + (size_t)c * cstride, ps + (size_t)c * cstride, n_part, pstride, s_max,
+                                         ldg_cg_f32(a.B.RS + row_base + c));
     if (threadIdx.x == 0) {
         int seq, layer, slot;
-        if (locate_row(up, a.D.L, a.mode, row_base + c, seq, layer, slot))
+        if (locate_row(up, a.D.L, a.mode, row_base + c, seq, layer, slot)) {
             a.B.SHADOW[((size_t)seq * a.D.L + (layer - 1)) * a.D.S + slot] = idx;
+            a.B.SCONF[((size_t)seq * a.D.L + (layer - 1)) * a.D.S + slot] = conf;
+        }
     }
+}
+
+// Eq. 3 for one layer: midpoint of the decayed mean confidences of matched and mismatched shadow tokens
+// (a mean over no tokens counts as 1 for the matched and as 0 for the mismatched ones).
+__device__ __forceinline__ double threshold(double Stcs, double Sc, double Sfcs, double Sn) {
+    const double Smis = __dsub_rn(Sn, Sc);
+    const double mean_true = Sc > 0.0 ? __ddiv_rn(Stcs, Sc) : 1.0;
+    const double mean_false = Smis > 0.0 ? __ddiv_rn(Sfcs, Smis) : 0.0;
+    return __dmul_rn(0.5, __dadd_rn(mean_true, mean_false));
+}
+
+// Thresholds of every layer from the statistics as they stand (after the statistics were set from outside).
+__global__ void refresh_tau_kernel(const CtlArgs a, int seq) {
+    const int L = a.D.L;
+    for (int l = threadIdx.x; l < L; l += blockDim.x)
+        a.B.TAU[seq * L + l] = threshold(a.B.STCS[seq * L + l], a.B.SC[seq * L + l], a.B.SFCS[seq * L + l], a.B.ST[seq].Sn);
 }
 
 // Prefix acceptance, per-layer match counts over the valid context and decayed statistics
@@ -156,15 +214,25 @@ __global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const Upda
     const int seq = up->s[u].seq, g = up->s[u].g, L = a.D.L, S = a.D.S;
     const int32_t *sh = a.B.SHADOW + (size_t)seq * L * S;
     const int32_t *verified = sh + (size_t)(L - 1) * S;
+    const float *cf = a.B.SCONF + (size_t)seq * L * S;
     int32_t *tok = a.B.TOK + seq * (S + 1);
     del_round_out *o = out + seq;
     if (a.mode == 1) {
         const int W = up->s[u].n_valid_init;
         for (int l = threadIdx.x; l < L; l += blockDim.x) {
             int c = 0;
-            for (int j = 0; j < W; ++j) c += (sh[(size_t)l * S + j] == verified[j]);
+            double tcs = 0.0, fcs = 0.0;
+            for (int j = 0; j < W; ++j) {
+                const bool match = sh[(size_t)l * S + j] == verified[j];
+                c += match;
+                if (match) tcs = __dadd_rn(tcs, (double)cf[(size_t)l * S + j]);
+                else fcs = __dadd_rn(fcs, (double)cf[(size_t)l * S + j]);
+            }
             a.B.COUNTS[seq * L + l] = c;
             a.B.SC[seq * L + l] = (double)c;
+            a.B.STCS[seq * L + l] = tcs;
+            a.B.SFCS[seq * L + l] = fcs;
+            a.B.TAU[seq * L + l] = threshold(tcs, (double)c, fcs, (double)W);
         }
         if (threadIdx.x == 0) {
             a.B.ST[seq].Sn = (double)W;
@@ -186,11 +254,24 @@ __global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const Upda
     }
     __syncthreads();
     const int n = s_n;
+    const double Sn_new = a.B.ST[seq].Sn;            // written by thread 0 before the barrier
     for (int l = threadIdx.x; l < L; l += blockDim.x) {
         int c = 0;
-        for (int i = 0; i <= n; ++i) c += (sh[(size_t)l * S + i] == verified[i]);
+        double tcs = 0.0, fcs = 0.0;                 // confidence sums over matched / mismatched shadow tokens (Sec. 4.4)
+        for (int i = 0; i <= n; ++i) {
+            const bool match = sh[(size_t)l * S + i] == verified[i];
+            c += match;
+            if (match) tcs = __dadd_rn(tcs, (double)cf[(size_t)l * S + i]);
+            else fcs = __dadd_rn(fcs, (double)cf[(size_t)l * S + i]);
+        }
         a.B.COUNTS[seq * L + l] = c;
-        a.B.SC[seq * L + l] = __dadd_rn(__dmul_rn(a.omega, a.B.SC[seq * L + l]), (double)c);
+        const double Sc = __dadd_rn(__dmul_rn(a.omega, a.B.SC[seq * L + l]), (double)c);
+        const double St = __dadd_rn(__dmul_rn(a.omega, a.B.STCS[seq * L + l]), tcs);
+        const double Sf = __dadd_rn(__dmul_rn(a.omega, a.B.SFCS[seq * L + l]), fcs);
+        a.B.SC[seq * L + l] = Sc;
+        a.B.STCS[seq * L + l] = St;
+        a.B.SFCS[seq * L + l] = Sf;
+        a.B.TAU[seq * L + l] = threshold(St, Sc, Sf, Sn_new);
     }
     __syncthreads();
     if (threadIdx.x == 0) tok[0] = verified[n];      // next round's input token
@@ -241,6 +322,7 @@ __global__ void __launch_bounds__(64) select_kernel(const CtlArgs a, const Updat
         st->gamma = G;
         out[seq].next_E = E;
         out[seq].next_gamma = G;
+        out[seq].next_tau = a.B.TAU[seq * L + E - 1];
     }
 }
 
@@ -310,9 +392,12 @@ cudaError_t launch_draft_finalize_embed(const CtlArgs &a, int m, bool embed_next
 cudaError_t launch_prep_rows(const CtlArgs &a, const UpdatePlan *up, int n_rows, cudaStream_t st, bool pdl) {
     return launch(prep_rows_kernel, n_rows, CTL_THREADS, st, pdl, a, up);
 }
-cudaError_t launch_shadow_reduce(const CtlArgs &a, const UpdatePlan *up, const float *pv, const int32_t *pi, int n_part,
-                                 int pstride, int cstride, int row_base, int n_rows, cudaStream_t st, bool pdl) {
-    return launch(shadow_reduce_kernel, n_rows, CTL_THREADS, st, pdl, a, up, pv, pi, n_part, pstride, cstride, row_base);
+cudaError_t launch_shadow_reduce(const CtlArgs &a, const UpdatePlan *up, const float *pv, const int32_t *pi, const float *ps,
+                                 int n_part, int pstride, int cstride, int row_base, int n_rows, cudaStream_t st, bool pdl) {
+    return launch(shadow_reduce_kernel, n_rows, CTL_THREADS, st, pdl, a, up, pv, pi, ps, n_part, pstride, cstride, row_base);
+}
+cudaError_t launch_refresh_tau(const CtlArgs &a, int seq, cudaStream_t st) {
+    return launch(refresh_tau_kernel, 1, 128, st, false, a, seq);
 }
 cudaError_t launch_update(const CtlArgs &a, const UpdatePlan *up, void *out_dev, int n_seq, cudaStream_t st, bool pdl) {
     return launch(update_kernel, n_seq, 128, st, pdl, a, up, (del_round_out *)out_dev);

@@ -25,6 +25,10 @@ struct SeqHost {
     int fixed_E = 0, fixed_gamma = 0;
     int phase = 0;           // 0 idle, 1 drafted, 2 verified
     int cur_E = 0, cur_g = 0, cur_gamma = 0;
+    int exit_mode = 0;       // 1: the draft loop stops on a low confidence (checked by the host per step)
+    int cur_stopped = 0;
+    double tau = 0.0;        // Eq. 3 threshold of the exit layer the next round uses
+    double cur_tau = 0.0;
     std::vector<int> pages;
 };
 
@@ -105,8 +109,18 @@ size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max
     B.ACNT = c.take<int32_t>(base, (size_t)DEL_SEQ_MAX * D.nkv);
     B.LPV = c.take<float>(base, (size_t)1024 * DEL_ROWS_MAX);
     B.LPI = c.take<int32_t>(base, (size_t)1024 * DEL_ROWS_MAX);
+    B.LPS = c.take<float>(base, (size_t)1024 * DEL_ROWS_MAX);
+    B.RK = c.take<float>(base, (size_t)DEL_ROWS_MAX);
     B.TPV = c.take<float>(base, (size_t)(R_max + 128) * n_vtiles);
     B.TPI = c.take<int32_t>(base, (size_t)(R_max + 128) * n_vtiles);
+    B.TPS = c.take<float>(base, (size_t)(R_max + 128) * n_vtiles);
+    B.RS = c.take<float>(base, (size_t)(R_max + 128));
+    B.SSE = c.take<float>(base, BS * D.n_sst);
+    B.DCONF = c.take<float>(base, (size_t)D.B * (D.S + 1));
+    B.SCONF = c.take<float>(base, (size_t)D.B * D.L * D.S);
+    B.STCS = c.take<double>(base, (size_t)D.B * D.L);
+    B.SFCS = c.take<double>(base, (size_t)D.B * D.L);
+    B.TAU = c.take<double>(base, (size_t)D.B * D.L);
     B.PROMPT_ALL = c.take<int32_t>(base, (size_t)D.max_seq);
     B.XN = c.take<bf16>(base, (size_t)(R_max + 128) * D.d);
     B.SHADOW = c.take<int32_t>(base, (size_t)D.B * D.L * D.S);
@@ -380,13 +394,71 @@ int run_layer(del_ctx *c, const PassInfo &pi, int l, bool write_exit) {
 }
 
 // sequences of a call with their round parameters
-struct Job { int seq, E, g; };
+struct Job { int seq, E, g; int stopped = 0; };
 
 // ---- draft (a1-a3): g tokens per sequence, layers 1..E, exit head, arg-max, next embedding
 int plans_needed_draft(const std::vector<Job> &jobs) {
     int gmax = 0;
     for (const Job &j : jobs) gmax = std::max(gmax, j.g);
     return gmax * ((int)jobs.size() + 1);
+}
+
+// plans of one draft step: all drafting rows, and per distinct exit layer the rows that go on beyond it
+struct DraftStep { int full_idx = -1; std::vector<int> sub_idx; };
+
+std::vector<int> exit_layers(const std::vector<Job> &jobs) {
+    // distinct exit layers, ascending: the rows of a pass thin out as sequences reach their exit
+    std::vector<int> Es;
+    for (const Job &j : jobs) Es.push_back(j.E);
+    std::sort(Es.begin(), Es.end());
+    Es.erase(std::unique(Es.begin(), Es.end()), Es.end());
+    return Es;
+}
+
+// `act`: the sequences that draft token i
+void plan_draft_step(del_ctx *c, PlanBatch &pb, const std::vector<Job> &act, const std::vector<int> &Es, int i, DraftStep &st) {
+    std::vector<RowSpec> full;
+    for (const Job &j : act) full.push_back(RowSpec{j.seq, i, 1});
+    fill_plan(c, pb.add(&st.full_idx), full, false);
+    for (size_t e = 0; e < Es.size(); ++e) {
+        if (e == 0) { st.sub_idx.push_back(st.full_idx); continue; }
+        std::vector<RowSpec> sub;
+        for (const Job &j : act)
+            if (j.E >= Es[e]) sub.push_back(RowSpec{j.seq, i, 1});
+        int idx = -1;
+        if (!sub.empty()) fill_plan(c, pb.add(&idx), sub, false);
+        st.sub_idx.push_back(idx);
+    }
+}
+
+// layers 1..E of every drafting row, the exit head in one pass over W_lm, arg-max + confidence, next embedding
+int launch_draft_step(del_ctx *c, const DraftStep &st, const std::vector<int> &Es, int i) {
+    const bool P = pdl(c);
+    const PassInfo full = pass_info(c, st.full_idx);
+    if (i == 0) {
+        CtlArgs ca = ctl_base(c, full.plan_idx);
+        LAUNCH(launch_embed(ca, full.m, c->st, P));
+    }
+    int l = 1;
+    for (size_t e = 0; e < Es.size(); ++e) {
+        if (st.sub_idx[e] < 0) break;
+        const PassInfo pi = pass_info(c, st.sub_idx[e]);
+        for (; l <= Es[e]; ++l) {
+            int rc = run_layer(c, pi, l, l == Es[e]);
+            if (rc) return rc;
+        }
+    }
+    GemmArgs a = gemm_base(c, full.plan_idx, 0);
+    a.K = c->D.d;
+    a.n_items = c->D.V / 16;
+    a.X = c->B.XE;
+    a.W0 = c->lm_head;
+    TAG(CLS_LMHEAD, 2.0 * c->D.V * c->D.d);
+    LAUNCH(launch_rowgemm(EPI_LMHEAD, a, full.m, c->n_sms, c->st, P));
+    CtlArgs ca = ctl_base(c, full.plan_idx);
+    ca.n_part = rowgemm_lmhead_grid(a.n_items, full.m, c->n_sms);
+    LAUNCH(launch_draft_finalize_embed(ca, full.m, true, c->st, P));
+    return DEL_OK;
 }
 
 int enqueue_draft(del_ctx *c, const std::vector<Job> &jobs) {
@@ -396,57 +468,67 @@ int enqueue_draft(del_ctx *c, const std::vector<Job> &jobs) {
     int rc = plan_begin(c, plans_needed_draft(jobs));
     if (rc) return rc;
     PlanBatch pb(c);
-    // distinct exit layers, ascending: the rows of a pass thin out as sequences reach their exit
-    std::vector<int> Es;
-    for (const Job &j : jobs) Es.push_back(j.E);
-    std::sort(Es.begin(), Es.end());
-    Es.erase(std::unique(Es.begin(), Es.end()), Es.end());
-    struct Step { int full_idx; std::vector<int> sub_idx; };
-    std::vector<Step> steps(gmax);
+    const std::vector<int> Es = exit_layers(jobs);
+    std::vector<DraftStep> steps(gmax);
     for (int i = 0; i < gmax; ++i) {
-        std::vector<RowSpec> full;
+        std::vector<Job> act;
         for (const Job &j : jobs)
-            if (i < j.g) full.push_back(RowSpec{j.seq, i, 1});
-        fill_plan(c, pb.add(&steps[i].full_idx), full, false);
-        for (size_t e = 0; e < Es.size(); ++e) {
-            if (e == 0) { steps[i].sub_idx.push_back(steps[i].full_idx); continue; }
-            std::vector<RowSpec> sub;
-            for (const Job &j : jobs)
-                if (i < j.g && j.E >= Es[e]) sub.push_back(RowSpec{j.seq, i, 1});
-            int idx = -1;
-            if (!sub.empty()) fill_plan(c, pb.add(&idx), sub, false);
-            steps[i].sub_idx.push_back(idx);
-        }
+            if (i < j.g) act.push_back(j);
+        plan_draft_step(c, pb, act, Es, i, steps[i]);
     }
     rc = plan_commit(c, pb);
     if (rc) return rc;
-    const bool P = pdl(c);
     for (int i = 0; i < gmax; ++i) {
-        const PassInfo full = pass_info(c, steps[i].full_idx);
-        if (i == 0) {
-            CtlArgs ca = ctl_base(c, full.plan_idx);
-            LAUNCH(launch_embed(ca, full.m, c->st, P));
-        }
-        int l = 1;
-        for (size_t e = 0; e < Es.size(); ++e) {
-            if (steps[i].sub_idx[e] < 0) break;
-            const PassInfo pi = pass_info(c, steps[i].sub_idx[e]);
-            for (; l <= Es[e]; ++l) {
-                rc = run_layer(c, pi, l, l == Es[e]);
-                if (rc) return rc;
+        rc = launch_draft_step(c, steps[i], Es, i);
+        if (rc) return rc;
+    }
+    return DEL_OK;
+}
+
+// Draft loop of Algorithm 1 with its confidence break.  On entry job.g is the most tokens the sequence
+// may draft; on return it is the number it kept, and job.stopped tells whether a low confidence ended
+// the loop (the dropped token's pass through layers 1..E then serves as the verify phase's last row).
+// The host reads each new token's confidence, so there is one synchronisation per step.
+int draft_with_exit(del_ctx *c, std::vector<Job> &jobs) {
+    std::vector<int> cap(jobs.size());
+    int gmax = 0;
+    for (size_t k = 0; k < jobs.size(); ++k) {
+        cap[k] = jobs[k].g;
+        jobs[k].g = 0;
+        jobs[k].stopped = 0;
+        gmax = std::max(gmax, cap[k]);
+    }
+    const std::vector<int> Es = exit_layers(jobs);
+    float *conf_host = reinterpret_cast<float *>(c->stage_host) + 2048;
+    for (int i = 0; i < gmax; ++i) {
+        std::vector<Job> act;
+        std::vector<size_t> who;
+        for (size_t k = 0; k < jobs.size(); ++k)
+            if (!jobs[k].stopped && i < cap[k]) { act.push_back(jobs[k]); who.push_back(k); }
+        if (act.empty()) break;
+        int rc = plan_begin(c, (int)Es.size() + 1);
+        if (rc) return rc;
+        PlanBatch pb(c);
+        DraftStep st;
+        plan_draft_step(c, pb, act, Es, i, st);
+        rc = plan_commit(c, pb);
+        if (rc) return rc;
+        rc = launch_draft_step(c, st, Es, i);
+        if (rc) return rc;
+        bool any = false;
+        for (size_t k : who)
+            if (c->seq[jobs[k].seq].exit_mode) {
+                CK(cudaMemcpyAsync(conf_host + k, c->B.DCONF + (size_t)jobs[k].seq * (c->D.S + 1) + i + 1, sizeof(float),
+                                   cudaMemcpyDeviceToHost, c->st));
+                c->d2h_bytes += sizeof(float);
+                any = true;
             }
+        if (any) CK(cudaStreamSynchronize(c->st));
+        for (size_t k : who) {
+            const SeqHost &s = c->seq[jobs[k].seq];
+            if (s.exit_mode && (double)conf_host[k] < s.cur_tau) jobs[k].stopped = 1;   // Algorithm 1: break, token dropped
+            else jobs[k].g = i + 1;
         }
-        // exit head of every drafting sequence in one pass over W_lm, then arg-max and next embedding
-        GemmArgs a = gemm_base(c, full.plan_idx, 0);
-        a.K = c->D.d;
-        a.n_items = c->D.V / 16;
-        a.X = c->B.XE;
-        a.W0 = c->lm_head;
-        TAG(CLS_LMHEAD, 2.0 * c->D.V * c->D.d);
-        LAUNCH(launch_rowgemm(EPI_LMHEAD, a, full.m, c->n_sms, c->st, P));
-        CtlArgs ca = ctl_base(c, full.plan_idx);
-        ca.n_part = rowgemm_lmhead_grid(a.n_items, full.m, c->n_sms);
-        LAUNCH(launch_draft_finalize_embed(ca, full.m, true, c->st, P));
     }
     return DEL_OK;
 }
@@ -467,17 +549,19 @@ int enqueue_verify(del_ctx *c, const std::vector<Job> &jobs) {
         const int l_first = k == 0 ? 1 : Es[k - 1] + 1;
         std::vector<RowSpec> specs;
         for (const Job &j : jobs) {
-            if (l_first <= j.E) specs.push_back(RowSpec{j.seq, j.g, 1});
+            // a sequence whose draft loop stopped on a low confidence already has row g through layer E
+            if (l_first <= j.E) { if (!j.stopped) specs.push_back(RowSpec{j.seq, j.g, 1}); }
             else specs.push_back(RowSpec{j.seq, 0, j.g + 1});
         }
-        fill_plan(c, pb.add(&idx[k]), specs, false);
+        idx[k] = -1;
+        if (!specs.empty()) fill_plan(c, pb.add(&idx[k]), specs, false);
     }
     // sequences that drafted nothing still need their input token embedded
     int embed_idx = -1;
     {
         std::vector<RowSpec> specs;
         for (const Job &j : jobs)
-            if (j.g == 0) specs.push_back(RowSpec{j.seq, 0, 1});
+            if (j.g == 0 && !j.stopped) specs.push_back(RowSpec{j.seq, 0, 1});
         if (!specs.empty()) fill_plan(c, pb.add(&embed_idx), specs, false);
     }
     rc = plan_commit(c, pb);
@@ -489,6 +573,7 @@ int enqueue_verify(del_ctx *c, const std::vector<Job> &jobs) {
     int l = 1;
     for (size_t k = 0; k <= Es.size(); ++k) {
         const int l_last = k < Es.size() ? Es[k] : c->D.L;
+        if (idx[k] < 0) { l = l_last + 1; continue; }
         const PassInfo pi = pass_info(c, idx[k]);
         for (; l <= l_last; ++l) {
             rc = run_layer(c, pi, l, false);
@@ -521,8 +606,9 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
         // one pass over W_lm on the tensor cores, arg-max fused; partials [row][vocabulary tile]
         const int nvt = lmhead_tc_vtiles(c->D.V);
         TAG(CLS_LMSTACK, 2.0 * c->D.V * c->D.d);
-        LAUNCH(launch_lmhead_tc(c->map_x, c->map_w, c->B.TPV, c->B.TPI, rows, c->D.V, c->D.d, c->B.ERR, c->n_sms, c->st, P));
-        LAUNCH(launch_shadow_reduce(ca, c->up_dev, c->B.TPV, c->B.TPI, nvt, 1, nvt, 0, rows, c->st, P));
+        LAUNCH(launch_lmhead_tc(c->map_x, c->map_w, c->B.TPV, c->B.TPI, c->B.TPS, c->B.RS, rows, c->D.V, c->D.d, c->B.ERR,
+                                c->n_sms, c->st, P));
+        LAUNCH(launch_shadow_reduce(ca, c->up_dev, c->B.TPV, c->B.TPI, c->B.TPS, nvt, 1, nvt, 0, rows, c->st, P));
         LAUNCH(launch_update(ca, c->up_dev, c->out_dev, up->n_seq, c->st, P));
         if (do_select) LAUNCH(launch_select(ca, c->up_dev, c->out_dev, up->n_seq, c->st, P));
         return DEL_OK;
@@ -548,10 +634,12 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
         a.X = c->B.XN + (size_t)k * DEL_ROWS_MAX * c->D.d;
         a.W0 = c->lm_head;
         a.x_by_row = 1;
+        a.row_scale = c->B.RS + (size_t)k * DEL_ROWS_MAX;
         TAG(CLS_LMSTACK, 2.0 * c->D.V * c->D.d);
         LAUNCH(launch_rowgemm(EPI_LMHEAD, a, m, c->n_sms, c->st, P));
         const int n_part = rowgemm_lmhead_grid(a.n_items, m, c->n_sms);
-        LAUNCH(launch_shadow_reduce(ca, c->up_dev, c->B.LPV, c->B.LPI, n_part, DEL_ROWS_MAX, 1, k * DEL_ROWS_MAX, m, c->st, P));
+        LAUNCH(launch_shadow_reduce(ca, c->up_dev, c->B.LPV, c->B.LPI, c->B.LPS, n_part, DEL_ROWS_MAX, 1, k * DEL_ROWS_MAX, m,
+                                    c->st, P));
     }
     LAUNCH(launch_update(ca, c->up_dev, c->out_dev, up->n_seq, c->st, P));
     if (do_select) LAUNCH(launch_select(ca, c->up_dev, c->out_dev, up->n_seq, c->st, P));
@@ -572,6 +660,29 @@ int read_out(del_ctx *c) {
         return DEL_ETIMEOUT;
     }
     return DEL_OK;
+}
+
+// thresholds of a sequence recomputed on the device from its statistics; the host copy of the
+// threshold of the current exit layer follows
+int refresh_tau(del_ctx *c, int sq) {
+    CtlArgs ca = ctl_base(c, -1);
+    cudaError_t e = launch_refresh_tau(ca, sq, c->st);
+    if (e != cudaSuccess) return fail(c, e);
+    CK(cudaStreamSynchronize(c->st));
+    if (c->seq[sq].E >= 1) {
+        double t = 0.0;
+        CK(cudaMemcpy(&t, c->B.TAU + (size_t)sq * c->D.L + (c->seq[sq].E - 1), sizeof(double), cudaMemcpyDeviceToHost));
+        c->seq[sq].tau = t;
+    }
+    return DEL_OK;
+}
+
+// threshold of an arbitrary layer (the caller fixed E itself); synchronises
+double exit_threshold(del_ctx *c, int sq, int E) {
+    double t = 0.0;
+    if (cudaStreamSynchronize(c->st) != cudaSuccess) return 0.0;
+    if (cudaMemcpy(&t, c->B.TAU + (size_t)sq * c->D.L + (E - 1), sizeof(double), cudaMemcpyDeviceToHost) != cudaSuccess) return 0.0;
+    return t;
 }
 
 int clip_gamma(const SeqHost &s, int gamma) { return std::max(0, std::min(gamma, s.remaining - 1)); }
@@ -716,12 +827,14 @@ int del_prefill(del_ctx *c, int sq, const int32_t *prompt, int n_prompt, int max
     s.remaining -= 1;
     s.E = o.next_E;
     s.gamma = o.next_gamma;
+    s.tau = o.next_tau;
     if (first_out) {
         memset(first_out, 0, sizeof(*first_out));
         first_out->n_emitted = 1;
         first_out->tokens[0] = o.tokens[0];
         first_out->next_E = o.next_E;
         first_out->next_gamma = o.next_gamma;
+        first_out->next_tau = o.next_tau;
     }
     return DEL_OK;
 }
@@ -734,9 +847,12 @@ int del_draft(del_ctx *c, int sq, int E, int gamma) {
     const int g = clip_gamma(s, gamma);
     int rc = ensure_pages(c, sq, s.T + g + 1);
     if (rc) return rc;
-    rc = enqueue_draft(c, {Job{sq, E, g}});
+    std::vector<Job> jobs{Job{sq, E, g}};
+    s.cur_tau = s.exit_mode ? exit_threshold(c, sq, E) : 0.0;
+    if (s.exit_mode) rc = draft_with_exit(c, jobs);
+    else rc = enqueue_draft(c, jobs);
     if (rc) return rc;
-    s.cur_E = E; s.cur_g = g; s.cur_gamma = gamma; s.phase = 1;
+    s.cur_E = E; s.cur_g = jobs[0].g; s.cur_stopped = jobs[0].stopped; s.cur_gamma = gamma; s.phase = 1;
     return DEL_OK;
 }
 
@@ -744,7 +860,7 @@ int del_verify(del_ctx *c, int sq) {
     if (!seq_ok(c, sq)) return DEL_EINVAL;
     SeqHost &s = c->seq[sq];
     if (!s.active || s.phase != 1) return DEL_ESTATE;
-    int rc = enqueue_verify(c, {Job{sq, s.cur_E, s.cur_g}});
+    int rc = enqueue_verify(c, {Job{sq, s.cur_E, s.cur_g, s.cur_stopped}});
     if (rc) return rc;
     s.phase = 2;
     return DEL_OK;
@@ -756,12 +872,14 @@ static void finish_round(del_ctx *c, int sq, del_round_out *dst, bool with_next)
     s.T += o.n_emitted;
     s.remaining -= o.n_emitted;
     s.phase = 0;
-    if (with_next) { s.E = o.next_E; s.gamma = o.next_gamma; }
+    if (with_next) { s.E = o.next_E; s.gamma = o.next_gamma; s.tau = o.next_tau; }
     if (dst) {
         *dst = o;
         dst->E = s.cur_E; dst->gamma = s.cur_gamma; dst->g = s.cur_g;
         dst->status = 0;
-        if (!with_next) { dst->next_E = 0; dst->next_gamma = 0; }
+        dst->stopped = s.cur_stopped;
+        dst->tau = s.cur_tau;
+        if (!with_next) { dst->next_E = 0; dst->next_gamma = 0; dst->next_tau = 0.0; }
     }
 }
 
@@ -792,6 +910,7 @@ int del_select(del_ctx *c, int sq, int32_t *E, int32_t *gamma) {
     if (rc) return rc;
     s.E = c->out_host[sq].next_E;
     s.gamma = c->out_host[sq].next_gamma;
+    s.tau = c->out_host[sq].next_tau;
     if (E) *E = s.E;
     if (gamma) *gamma = s.gamma;
     return DEL_OK;
@@ -800,6 +919,7 @@ int del_select(del_ctx *c, int sq, int32_t *E, int32_t *gamma) {
 int del_round(del_ctx *c, del_round_out *out) {
     if (!c || !out) return DEL_EINVAL;
     std::vector<Job> jobs;
+    bool any_exit = false;
     for (int sq = 0; sq < c->D.B; ++sq) {
         SeqHost &s = c->seq[sq];
         memset(&out[sq], 0, sizeof(out[sq]));
@@ -807,15 +927,19 @@ int del_round(del_ctx *c, del_round_out *out) {
         if (s.phase != 0) return DEL_ESTATE;
         const int E = s.fixed_E > 0 ? s.fixed_E : s.E;
         const int gamma = s.fixed_E > 0 ? s.fixed_gamma : s.gamma;
-        const int g = clip_gamma(s, gamma);
+        // Algorithm 1: with draft-exiting the loop may run up to d_max tokens, otherwise gamma tokens
+        const int g = clip_gamma(s, s.exit_mode ? c->sh.g_max : gamma);
         int rc = ensure_pages(c, sq, s.T + g + 1);
         if (rc) return rc;
-        s.cur_E = E; s.cur_g = g; s.cur_gamma = gamma;
+        s.cur_E = E; s.cur_g = g; s.cur_gamma = gamma; s.cur_stopped = 0;
+        s.cur_tau = s.exit_mode ? (s.fixed_E > 0 ? exit_threshold(c, sq, E) : s.tau) : 0.0;
+        any_exit = any_exit || s.exit_mode;
         jobs.push_back(Job{sq, E, g});
     }
     if (jobs.empty()) return DEL_ESTATE;
-    int rc = enqueue_draft(c, jobs);
+    int rc = any_exit ? draft_with_exit(c, jobs) : enqueue_draft(c, jobs);
     if (rc) return rc;
+    for (const Job &j : jobs) { c->seq[j.seq].cur_g = j.g; c->seq[j.seq].cur_stopped = j.stopped; }
     rc = enqueue_verify(c, jobs);
     if (rc) return rc;
     rc = enqueue_update(c, jobs, 0, 0, true);
@@ -863,6 +987,46 @@ int del_set_stats(del_ctx *c, int sq, const double *Sc, double Sn, int32_t E, in
     CK(cudaMemcpy(c->B.ST + sq, &st, sizeof(st), cudaMemcpyHostToDevice));
     c->seq[sq].E = E;
     c->seq[sq].gamma = gamma;
+    return refresh_tau(c, sq);
+}
+
+int del_set_exit_mode(del_ctx *c, int sq, int mode) {
+    if (!seq_ok(c, sq)) return DEL_EINVAL;
+    c->seq[sq].exit_mode = mode ? 1 : 0;
+    return DEL_OK;
+}
+
+int del_get_conf_stats(del_ctx *c, int sq, double *Stcs, double *Sfcs, double *tau) {
+    if (!seq_ok(c, sq)) return DEL_EINVAL;
+    CK(cudaStreamSynchronize(c->st));
+    const size_t off = (size_t)sq * c->D.L, nb = sizeof(double) * c->D.L;
+    if (Stcs) CK(cudaMemcpy(Stcs, c->B.STCS + off, nb, cudaMemcpyDeviceToHost));
+    if (Sfcs) CK(cudaMemcpy(Sfcs, c->B.SFCS + off, nb, cudaMemcpyDeviceToHost));
+    if (tau) CK(cudaMemcpy(tau, c->B.TAU + off, nb, cudaMemcpyDeviceToHost));
+    return DEL_OK;
+}
+
+int del_set_conf_stats(del_ctx *c, int sq, const double *Stcs, const double *Sfcs) {
+    if (!seq_ok(c, sq) || !Stcs || !Sfcs) return DEL_EINVAL;
+    CK(cudaStreamSynchronize(c->st));
+    const size_t off = (size_t)sq * c->D.L, nb = sizeof(double) * c->D.L;
+    CK(cudaMemcpy(c->B.STCS + off, Stcs, nb, cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(c->B.SFCS + off, Sfcs, nb, cudaMemcpyHostToDevice));
+    return refresh_tau(c, sq);
+}
+
+int del_get_conf(del_ctx *c, int sq, float *shadow_conf, float *draft_conf) {
+    if (!seq_ok(c, sq)) return DEL_EINVAL;
+    CK(cudaStreamSynchronize(c->st));
+    const int L = c->D.L, S = c->D.S, G = c->sh.g_max + 1;
+    if (shadow_conf) {
+        std::vector<float> tmp((size_t)L * S);
+        CK(cudaMemcpy(tmp.data(), c->B.SCONF + (size_t)sq * L * S, sizeof(float) * L * S, cudaMemcpyDeviceToHost));
+        for (int l = 0; l < L; ++l)
+            for (int i = 0; i < G; ++i) shadow_conf[l * G + i] = tmp[(size_t)l * S + i];
+    }
+    if (draft_conf)
+        CK(cudaMemcpy(draft_conf, c->B.DCONF + (size_t)sq * (S + 1) + 1, sizeof(float) * G, cudaMemcpyDeviceToHost));
     return DEL_OK;
 }
 

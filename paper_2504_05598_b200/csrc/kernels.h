@@ -17,6 +17,7 @@ struct GemmArgs {
     const bf16 *gain_a, *gain_b;
     int32_t *tile_ctr;         // per-launch zeroed counter for dynamic tile claims (nullptr: static round-robin)
     int32_t x_by_row;          // LMHEAD: activations are X[c] (stacked rows) instead of XE[seq][slot]
+    const float *row_scale;    // LMHEAD with x_by_row: log2(e) / rms per row (nullptr: taken from B.SSE)
 };
 
 cudaError_t launch_rowgemm(int epi, const GemmArgs &a, int m, int n_sms, cudaStream_t st, bool pdl);
@@ -64,8 +65,9 @@ struct UpdatePlan {
 cudaError_t launch_embed(const CtlArgs &a, int m, cudaStream_t st, bool pdl);
 cudaError_t launch_draft_finalize_embed(const CtlArgs &a, int m, bool embed_next, cudaStream_t st, bool pdl);
 cudaError_t launch_prep_rows(const CtlArgs &a, const UpdatePlan *up, int n_rows, cudaStream_t st, bool pdl);
-cudaError_t launch_shadow_reduce(const CtlArgs &a, const UpdatePlan *up, const float *pv, const int32_t *pi, int n_part,
-                                 int pstride, int cstride, int row_base, int n_rows, cudaStream_t st, bool pdl);
+cudaError_t launch_shadow_reduce(const CtlArgs &a, const UpdatePlan *up, const float *pv, const int32_t *pi, const float *ps,
+                                 int n_part, int pstride, int cstride, int row_base, int n_rows, cudaStream_t st, bool pdl);
+cudaError_t launch_refresh_tau(const CtlArgs &a, int seq, cudaStream_t st);
 cudaError_t launch_update(const CtlArgs &a, const UpdatePlan *up, void *out_dev, int n_seq, cudaStream_t st, bool pdl);
 cudaError_t launch_select(const CtlArgs &a, const UpdatePlan *up, void *out_dev, int n_seq, cudaStream_t st, bool pdl);
 cudaError_t launch_debug_logits(const CtlArgs &a, int layer, int seq, int slot, float *out_dev, cudaStream_t st);
@@ -75,5 +77,5 @@ cudaError_t launch_gather_kv(const CtlArgs &a, int layer, int seq, int pos, floa
 // opaque blobs (CUtensorMap) kept by the host context.
 int lmhead_tc_make_map(void *map_out, const void *base, uint64_t rows, uint64_t d, uint32_t box_rows);
 int lmhead_tc_vtiles(int V);
-cudaError_t launch_lmhead_tc(const void *map_x, const void *map_w, float *part_v, int32_t *part_i, int n_rows, int V, int d,
-                             int32_t *err, int n_sms, cudaStream_t st, bool pdl);
+cudaError_t launch_lmhead_tc(const void *map_x, const void *map_w, float *part_v, int32_t *part_i, float *part_s,
+                             const float *row_scale, int n_rows, int V, int d, int32_t *err, int n_sms, cudaStream_t st, bool pdl);

@@ -27,6 +27,8 @@ constexpr uint32_t WAIT_LIMIT = 1u << 26;
 struct TcParams {
     float *part_v;
     int32_t *part_i;
+    float *part_s;               // exp sums relative to part_v (for the confidence score)
+    const float *row_scale;      // [rows] log2(e) / rms: the logit behind accumulator v is v / rms
     int32_t n_rows, V, d, n_mtiles, n_vtiles, n_tiles;
     int32_t *err;
 };
@@ -165,17 +167,24 @@ lmhead_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int row = mt * BM + q * 32 + lane;
             const int v0 = vt * BN;
-            float best = -INFINITY;
+            const float k = row < p.n_rows ? p.row_scale[row] : 0.f;
+            float best = -INFINITY, esum = 0.f;
             int bidx = 0x7fffffff;
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), r);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                const float before = best;
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     const float v = __uint_as_float(r[j]);
                     if (v0 + c0 + j < p.V && v > best) { best = v; bidx = v0 + c0 + j; }
                 }
+                // exp sum relative to the running maximum (rescaled when this chunk raised it)
+                if (best > before) esum *= exp2f(k * (before - best));
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (v0 + c0 + j < p.V) esum += exp2f(k * (__uint_as_float(r[j]) - best));
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
@@ -183,6 +192,7 @@ lmhead_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             if (row < p.n_rows) {
                 p.part_v[(size_t)row * p.n_vtiles + vt] = best;
                 p.part_i[(size_t)row * p.n_vtiles + vt] = bidx;
+                p.part_s[(size_t)row * p.n_vtiles + vt] = esum;
             }
         }
     }
@@ -229,10 +239,10 @@ int lmhead_tc_make_map(void *map_out, const void *base, uint64_t rows, uint64_t 
 
 int lmhead_tc_vtiles(int V) { return (V + BN - 1) / BN; }
 
-cudaError_t launch_lmhead_tc(const void *map_x, const void *map_w, float *part_v, int32_t *part_i, int n_rows, int V, int d,
-                             int32_t *err, int n_sms, cudaStream_t st, bool pdl) {
+cudaError_t launch_lmhead_tc(const void *map_x, const void *map_w, float *part_v, int32_t *part_i, float *part_s,
+                             const float *row_scale, int n_rows, int V, int d, int32_t *err, int n_sms, cudaStream_t st, bool pdl) {
     TcParams p;
-    p.part_v = part_v; p.part_i = part_i; p.n_rows = n_rows; p.V = V; p.d = d;
+    p.part_v = part_v; p.part_i = part_i; p.part_s = part_s; p.row_scale = row_scale; p.n_rows = n_rows; p.V = V; p.d = d;
     p.n_mtiles = (n_rows + BM - 1) / BM;
     p.n_vtiles = (V + BN - 1) / BN;
     p.n_tiles = p.n_mtiles * p.n_vtiles;

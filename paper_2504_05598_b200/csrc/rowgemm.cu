@@ -35,7 +35,7 @@ namespace {
 
 // bytes of the reduction buffer, result tile, row scales and arg-max state (16-byte multiple)
 __host__ __device__ constexpr size_t small_smem_bytes(int nt) {
-    return (sizeof(float4) * 8 * nt * 32 + sizeof(float) * (nt * 8 * 16 + 3 * nt * 8) + 15) & ~(size_t)15;
+    return (sizeof(float4) * 8 * nt * 32 + sizeof(float) * (nt * 8 * 16 + 4 * nt * 8) + 15) & ~(size_t)15;
 }
 
 // The 16 weight rows of a tile are two groups of 8 (MMA rows g and g+8), which need not be adjacent:
@@ -78,6 +78,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     float *rscale = res + NC * 16;                                      // [NC]
     float *best_v = rscale + NC;                                              // [NC]
     int *best_i = reinterpret_cast<int *>(best_v + NC);                       // [NC]
+    float *best_s = best_v + 2 * NC;                                          // [NC] exp sums relative to best_v
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int K = a.K;
@@ -169,7 +170,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
         }
     }
     if (EPI == EPI_LMHEAD) {
-        for (int c = tid; c < NC; c += DEL_GEMM_THREADS) { best_v[c] = -INFINITY; best_i[c] = 0x7fffffff; }
+        for (int c = tid; c < NC; c += DEL_GEMM_THREADS) { best_v[c] = -INFINITY; best_i[c] = 0x7fffffff; best_s[c] = 0.f; }
     }
     // no barrier here: rscale / best_* are first read in an epilogue, after the two barriers of tile_end
 
@@ -265,7 +266,10 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
                 ss += __shfl_xor_sync(0xffffffffu, ss, 1);
                 if (valid && i == 0) {
                     if (EPI == EPI_OPROJ) a.B.SSM[(size_t)c * a.D.n_sst + item] = ss;
-                    else a.B.SS[stack_row(a.D, a.layer, rd.seq, rd.slot) * a.D.n_sst + item] = ss;
+                    else {
+                        a.B.SS[stack_row(a.D, a.layer, rd.seq, rd.slot) * a.D.n_sst + item] = ss;
+                        if (a.gain_b) a.B.SSE[((size_t)rd.seq * a.D.S + rd.slot) * a.D.n_sst + item] = ss;
+                    }
                 }
             } else if (EPI == EPI_LMHEAD) {
                 float v = valid ? ra : -INFINITY;      // the row's 1/rms is positive: it cannot change the arg-max
@@ -276,7 +280,23 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
                     const int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
                     if (v2 > v || (v2 == v && i2 < idx)) { v = v2; idx = i2; }
                 }
-                if (valid && i == 0 && (v > best_v[c] || (v == best_v[c] && idx < best_i[c]))) { best_v[c] = v; best_i[c] = idx; }
+                // running sum of exp over the vocabulary for the confidence score (top-1 probability): the
+                // normalised logit is raw / rms, kept as exp2(k * (raw - running maximum)) with k = log2(e) / rms
+                const float k = rscale[c];
+                float es = valid ? exp2f(k * (ra - v)) : 0.f;
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) es += __shfl_xor_sync(0xffffffffu, es, o);
+                if (valid && i == 0) {
+                    const float bv = best_v[c];
+                    if (v > bv) {
+                        best_s[c] = best_s[c] * exp2f(k * (bv - v)) + es;
+                        best_v[c] = v;
+                        best_i[c] = idx;
+                    } else {
+                        best_s[c] += es * exp2f(k * (v - bv));
+                        if (v == bv && idx < best_i[c]) best_i[c] = idx;
+                    }
+                }
             }
         }
         // `res` and `best_*` are next written after the following tile's first barrier
@@ -308,6 +328,26 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
             }
             s = warp_sum(s);
             if (lane == 0) rscale[c] = rsqrtf(s / (float)a.D.d + a.D.eps);
+        }
+    }
+    if (EPI == EPI_LMHEAD) {
+        for (int c = warp; c < NC; c += DEL_GEMM_WARPS) {
+            float k = 0.f;
+            if (c < m) {
+                if (a.row_scale) {
+                    k = a.row_scale[c];
+                } else if (a.B.SSE != nullptr) {    // (callers that want no confidences pass neither: k = 0)
+                    const float *ss = a.B.SSE + ((size_t)plan->rows[c].seq * a.D.S + plan->rows[c].slot) * a.D.n_sst;
+                    float sq = 0.f;
+                    for (int i = lane; i < a.D.n_sst; i += 32) sq += ldg_cg_f32(ss + i);
+                    sq = warp_sum(sq);
+                    k = rsqrtf(sq / (float)a.D.d + a.D.eps) * 1.4426950408889634f;
+                }
+            }
+            if (lane == 0) {
+                rscale[c] = k;
+                if (blockIdx.x == 0 && c < m && a.B.RK != nullptr) a.B.RK[c] = k;
+            }
         }
     }
     int u0 = U;
@@ -342,6 +382,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
         for (int c = tid; c < m; c += DEL_GEMM_THREADS) {
             a.B.LPV[(size_t)blockIdx.x * DEL_ROWS_MAX + c] = best_v[c];
             a.B.LPI[(size_t)blockIdx.x * DEL_ROWS_MAX + c] = best_i[c];
+            if (a.B.LPS) a.B.LPS[(size_t)blockIdx.x * DEL_ROWS_MAX + c] = best_s[c];
         }
     }
 }

@@ -6,15 +6,24 @@ MARGIN.  A difference at a smaller margin is a tolerated flip: it is counted, an
 re-synchronised to the oracle (re-prefill on the oracle's tokens, forced next token, statistics
 restored) so that later rounds stay comparable.  The acceptance statistics are doubles computed with the
 same operation order on both sides, so after identical integer inputs they must agree bit for bit.
+
+Confidence scores (top-1 softmax probabilities) are floating point on both sides: fp32 from bf16
+activations in the library, fp64 in the oracle.  With logits within EPS_LOGIT of each other the sum of
+exponentials changes by at most a factor exp(2 * EPS_LOGIT), so confidences, their decayed sums and the
+thresholds are compared with the relative tolerance CONF_RTOL = exp(2 * EPS_LOGIT) - 1.  The draft
+loop's decision "confidence < threshold" must be the same wherever the oracle's two numbers are further
+apart than that tolerance allows; a decision inside the band is a tolerated flip (counted, re-synchronised).
 """
 from __future__ import annotations
 
 from dataclasses import dataclass, field
-from typing import List
+from typing import List, Optional
 
 import numpy as np
 
 MARGIN = 0.05
+EPS_LOGIT = 3e-2
+CONF_RTOL = float(np.exp(2 * EPS_LOGIT) - 1.0)
 
 
 @dataclass
@@ -32,6 +41,14 @@ class RoundRef:
     next_gamma: int
     Sc: np.ndarray
     Sn: float
+    # dynamic draft-exiting (None / defaults when the reference trace does not carry them)
+    conf: Optional[np.ndarray] = None       # [L][g+1] confidence of the shadow tokens
+    draft_conf: Optional[List[float]] = None  # confidence of each drafted token, the dropped one included
+    stopped: bool = False
+    tau: float = 0.0
+    next_tau: float = 0.0
+    Stcs: Optional[np.ndarray] = None
+    Sfcs: Optional[np.ndarray] = None
 
 
 @dataclass
@@ -46,6 +63,11 @@ class SeqRef:
     init_gamma: int
     rounds: List[RoundRef]
     tokens: List[int]
+    init_conf: Optional[np.ndarray] = None
+    init_Stcs: Optional[np.ndarray] = None
+    init_Sfcs: Optional[np.ndarray] = None
+    init_tau: float = 0.0
+    exit_mode: bool = False
 
 
 @dataclass
@@ -54,27 +76,36 @@ class Report:
     flips: int = 0
     resyncs: int = 0
     compared: int = 0
+    conf_compared: int = 0
+    conf_max_rel: float = 0.0
+    decisions: int = 0
+    decision_flips: int = 0
     failures: List[str] = field(default_factory=list)
 
     def ok(self) -> bool:
         return not self.failures
 
 
-def ref_from_oracle(cfg, weights, prompt, gen_len=None, policy=None) -> SeqRef:
+def ref_from_oracle(cfg, weights, prompt, gen_len=None, policy=None, exit_mode=False) -> SeqRef:
     """Runs the oracle now (small models)."""
     import oracle
     o = oracle.OracleSeq(cfg, weights)
     if policy:
         o.set_policy(*policy)
+    o.set_exit_mode(exit_mode)
     n_tok = gen_len or cfg.gen_len
     tok, init = o.prefill(prompt)
     Sc, Sn, E, g = o.get_stats()
-    ref = SeqRef(np.asarray(prompt, dtype=np.int32), tok, init.shadow, init.margin, Sc, Sn, E, g, [], [tok])
+    Stcs, Sfcs, _ = o.get_conf_stats()
+    ref = SeqRef(np.asarray(prompt, dtype=np.int32), tok, init.shadow, init.margin, Sc, Sn, E, g, [], [tok],
+                 init_conf=init.conf, init_Stcs=Stcs, init_Sfcs=Sfcs, init_tau=init.next_tau, exit_mode=exit_mode)
     while len(ref.tokens) < n_tok:
         r = o.round(n_tok - len(ref.tokens))
         Sc, Sn, _, _ = o.get_stats()
+        Stcs, Sfcs, _ = o.get_conf_stats()
         ref.rounds.append(RoundRef(r.E, r.gamma, r.g, r.n_accept, r.drafts, r.emitted, r.shadow, r.margin, r.counts,
-                                   r.next_E, r.next_gamma, Sc, Sn))
+                                   r.next_E, r.next_gamma, Sc, Sn, conf=r.conf, draft_conf=r.draft_conf,
+                                   stopped=r.stopped, tau=r.tau, next_tau=r.next_tau, Stcs=Stcs, Sfcs=Sfcs))
         ref.tokens.extend(r.emitted)
     o.close()
     return ref
@@ -96,12 +127,29 @@ def ref_from_golden(doc, seq_index, prompt) -> SeqRef:
     return ref
 
 
-def _resync(ctx, seq, ref: SeqRef, n_done_tokens: int, Sc, Sn, E, gamma, total_tokens: int):
+def _resync(ctx, seq, ref: SeqRef, n_done_tokens: int, Sc, Sn, E, gamma, total_tokens: int, Stcs=None, Sfcs=None):
     """Puts the library into the oracle's state after `n_done_tokens` emitted tokens."""
     ctx_tokens = list(ref.prompt) + ref.tokens[:n_done_tokens - 1]
     ctx.prefill(seq, ctx_tokens, total_tokens - n_done_tokens + 1)
     ctx.force_token(seq, ref.tokens[n_done_tokens - 1])
+    if Stcs is not None:
+        ctx.set_conf_stats(seq, Stcs, Sfcs)
     ctx.set_stats(seq, Sc, Sn, E, gamma)
+    if ref.exit_mode:
+        ctx.set_exit_mode(seq, True)
+
+
+def _compare_conf(rep: Report, what: str, got, want):
+    """Element-wise relative comparison of confidence-like numbers."""
+    got, want = np.asarray(got, dtype=np.float64), np.asarray(want, dtype=np.float64)
+    rel = np.abs(got - want) / np.maximum(np.abs(want), 1e-6)
+    rel = np.where(np.abs(got - want) < 1e-6, 0.0, rel)
+    rep.conf_compared += rel.size
+    if rel.size:
+        rep.conf_max_rel = max(rep.conf_max_rel, float(rel.max()))
+        if rel.max() > CONF_RTOL:
+            k = int(np.argmax(rel))
+            rep.failures.append(f"{what}: element {k} gpu {got.flat[k]:.6f} oracle {want.flat[k]:.6f}")
 
 
 def compare_init(ctx, seq, ref: SeqRef, total_tokens: int, rep: Report, policy=None) -> None:
@@ -123,6 +171,13 @@ def compare_init(ctx, seq, ref: SeqRef, total_tokens: int, rep: Report, policy=N
                                         f"margin {ref.init_margin[l, j]:.3f}")
                 flips += 1
     Sc, Sn, E, g = ctx.get_stats(seq)
+    if flips == 0 and ref.init_conf is not None:
+        sc, _ = ctx.get_conf(seq)
+        _compare_conf(rep, "init confidences", sc[:, :ncol], ref.init_conf[:, :ncol])
+        Stcs, Sfcs, tau = ctx.get_conf_stats(seq)
+        if ncol == W:       # the sums run over the whole window
+            _compare_conf(rep, "init Stcs", Stcs, ref.init_Stcs)
+            _compare_conf(rep, "init Sfcs", Sfcs, ref.init_Sfcs)
     same = (out.tokens[0] == ref.first_token and np.array_equal(Sc, ref.init_Sc) and Sn == ref.init_Sn
             and (policy or (E, g) == (ref.init_E, ref.init_gamma)))
     if not same:
@@ -136,15 +191,44 @@ def compare_init(ctx, seq, ref: SeqRef, total_tokens: int, rep: Report, policy=N
         rep.flips += flips
         rep.resyncs += 1
         ctx.force_token(seq, ref.first_token)
+        if ref.init_Stcs is not None:
+            ctx.set_conf_stats(seq, ref.init_Stcs, ref.init_Sfcs)
         ctx.set_stats(seq, ref.init_Sc, ref.init_Sn, ref.init_E, ref.init_gamma)
+    if ref.exit_mode:
+        ctx.set_exit_mode(seq, True)
 
 
 def compare_round(ctx, seq, out, r: RoundRef, rep: Report, check_choice=True) -> bool:
     """Compares one finished round; returns True if the library must be re-synchronised."""
     L = r.shadow.shape[0]
     rep.rounds += 1
-    if (out.E, out.gamma, out.g) != (r.E, r.gamma, r.g):
-        rep.failures.append(f"round {rep.rounds}: ran with (E,gamma,g)={(out.E, out.gamma, out.g)}, oracle {(r.E, r.gamma, r.g)}")
+    if r.draft_conf is not None and r.tau > 0.0 and out.tau > 0.0:
+        # dynamic draft-exiting: the loop's decisions, wherever the oracle's numbers are clearly apart
+        _, dc = ctx.get_conf(seq)
+        n_dec = min(len(r.draft_conf), out.g + int(out.stopped))
+        rep.decisions += n_dec
+        _compare_conf(rep, f"round {rep.rounds}: tau", [out.tau], [r.tau])
+        for i in range(n_dec):
+            want_stop, got_stop = r.draft_conf[i] < r.tau, float(dc[i]) < out.tau
+            if want_stop != got_stop:
+                band = CONF_RTOL * (r.draft_conf[i] + r.tau)
+                if abs(r.draft_conf[i] - r.tau) > band:
+                    rep.failures.append(f"round {rep.rounds}: draft {i} confidence {dc[i]:.5f} vs tau {out.tau:.5f}, oracle "
+                                        f"{r.draft_conf[i]:.5f} vs {r.tau:.5f}")
+                rep.decision_flips += 1
+                rep.flips += 1
+                return True
+            if want_stop:
+                break
+    if (out.E, out.gamma, out.g) != (r.E, r.gamma, r.g) or bool(out.stopped) != bool(r.stopped):
+        # a draft token that differs at a low margin changes the confidences that follow
+        drafts = ctx.get_drafts(seq)
+        k = next((i for i in range(min(out.g, r.g)) if drafts[i] != r.drafts[i]), None)
+        if k is not None and r.margin[r.E - 1, k] <= MARGIN:
+            rep.flips += 1
+            return True
+        rep.failures.append(f"round {rep.rounds}: ran with (E,gamma,g,stopped)={(out.E, out.gamma, out.g, bool(out.stopped))}, "
+                            f"oracle {(r.E, r.gamma, r.g, bool(r.stopped))}")
         return True
     sh, counts = ctx.get_shadow(seq)
     drafts = ctx.get_drafts(seq)[:r.g]
@@ -167,6 +251,15 @@ def compare_round(ctx, seq, out, r: RoundRef, rep: Report, check_choice=True) ->
                     rep.failures.append(f"round {rep.rounds}: shadow l={l + 1} i={i} gpu {sh[l, i]} oracle {r.shadow[l, i]} "
                                         f"margin {r.margin[l, i]:.3f}")
                 flips += 1
+    if flips == 0 and r.conf is not None:
+        sc, dc = ctx.get_conf(seq)
+        _compare_conf(rep, f"round {rep.rounds}: shadow confidences", sc[:, :r.g + 1], r.conf)
+        if r.draft_conf:
+            _compare_conf(rep, f"round {rep.rounds}: draft confidences", dc[:len(r.draft_conf)], r.draft_conf)
+        Stcs, Sfcs, tau = ctx.get_conf_stats(seq)
+        _compare_conf(rep, f"round {rep.rounds}: Stcs", Stcs, r.Stcs)
+        _compare_conf(rep, f"round {rep.rounds}: Sfcs", Sfcs, r.Sfcs)
+        _compare_conf(rep, f"round {rep.rounds}: next tau", [out.next_tau], [r.next_tau])
     if flips == 0:
         Sc, Sn, E, g = ctx.get_stats(seq)
         if out.n_accept != r.n or out.emitted() != list(r.emitted):
@@ -196,9 +289,10 @@ def run_sequence(ctx, seq, ref: SeqRef, total_tokens: int, policy=None, max_roun
         done += r.n + 1
         if need and k + 1 < len(ref.rounds):
             rep.resyncs += 1
-            _resync(ctx, seq, ref, done, r.Sc, r.Sn, r.next_E, r.next_gamma, total_tokens)
+            _resync(ctx, seq, ref, done, r.Sc, r.Sn, r.next_E, r.next_gamma, total_tokens, r.Stcs, r.Sfcs)
             if policy:
                 ctx.set_policy(seq, *policy)
+
         if len(rep.failures) > 20:
             break
     return rep
@@ -226,7 +320,7 @@ def run_batch(ctx, refs: List[SeqRef], total_tokens: int, max_rounds=None) -> Li
             k[s] += 1
             if need and k[s] < len(refs[s].rounds):
                 reps[s].resyncs += 1
-                _resync(ctx, s, refs[s], done[s], r.Sc, r.Sn, r.next_E, r.next_gamma, total_tokens)
+                _resync(ctx, s, refs[s], done[s], r.Sc, r.Sn, r.next_E, r.next_gamma, total_tokens, r.Stcs, r.Sfcs)
         if sum(len(rp.failures) for rp in reps) > 20:
             break
     return reps

@@ -222,6 +222,38 @@ def test_streaming_lm_head_against_oracle(small):
     assert rep.rounds == len(ref.rounds)
 
 
+def test_dynamic_draft_exiting_against_oracle(small):
+    """Sec. 4.4 / Algorithm 1 with the confidence break: the draft loop runs up to g_max tokens and stops at
+    the first token whose confidence is below the exit layer's threshold; same streams, same g, same
+    stop decisions (outside the tolerance band), confidences and thresholds within tolerance."""
+    cfg, w, ctx = small
+    ref = ref_from_oracle(cfg, w, synth.make_prompt(cfg), exit_mode=True)
+    rep = run_sequence(ctx, 0, ref, cfg.gen_len)
+    ctx.set_exit_mode(0, False)
+    stops = sum(r.stopped for r in ref.rounds)
+    print(f"{cfg.name} (draft-exiting): rounds {rep.rounds} stops {stops} decisions {rep.decisions} decision flips "
+          f"{rep.decision_flips} conf compared {rep.conf_compared} max rel err {rep.conf_max_rel:.2e} flips {rep.flips}")
+    assert rep.ok(), rep.failures[:5]
+    assert rep.rounds == len(ref.rounds)
+    assert rep.decisions > 0 and rep.decision_flips <= max(1, rep.decisions // 10)
+
+
+def test_confidences_in_fixed_gamma_rounds(small):
+    """The confidence statistics are maintained in every mode; here with the streaming LM head as well."""
+    import paper_2504_05598_b200 as dl
+    cfg, w, ctx = small
+    ref = ref_from_oracle(cfg, w, synth.make_prompt(cfg))
+    for flags in (dl.FLAG_PDL | dl.FLAG_TC, dl.FLAG_PDL):
+        old = ctx.set_flags(flags)
+        try:
+            rep = run_sequence(ctx, 0, ref, cfg.gen_len)
+        finally:
+            ctx.set_flags(old)
+        print(f"{cfg.name} flags {flags}: conf compared {rep.conf_compared} max rel err {rep.conf_max_rel:.2e}")
+        assert rep.ok(), rep.failures[:5]
+        assert rep.conf_compared > 0 and rep.conf_max_rel <= 0.02     # far inside the derived bound in practice
+
+
 def test_streaming_lm_head_full_size():
     import paper_2504_05598_b200 as dl
     name = "llama2_7b"
