@@ -86,14 +86,40 @@ __device__ __forceinline__ float block_sum(float v) {
     return t;
 }
 
-// Confidence score (Sec. 4.4: probability of the top-1 token) from partial (maximum, exp sum) pairs:
-// 1 / sum_p s_p * exp2(k * (v_p - M)), M the overall maximum, k = log2(e) / rms of the row.
-__device__ __forceinline__ float merged_confidence(const float *pv, const float *ps, int n_part, size_t pstride, float M, float k) {
+// Partials (maximum, index, exp sum) of one row reduced to the token and its confidence score (Sec. 4.4:
+// the probability of the top-1 token) = 1 / sum_p s_p * exp2(k * (v_p - M)), M the overall maximum,
+// k = log2(e) / rms of the row.  All partials are loaded once (up to PMAX per thread stay in registers).
+// Results valid in thread 0.
+constexpr int PMAX = 4;                              // CTL_THREADS * PMAX = 1024 partials
+__device__ __forceinline__ void reduce_partials(const float *pv, const int32_t *pi, const float *ps, int n_part, size_t pstride,
+                                                const float *kp, int &token, float &conf) {
+    __shared__ float s_max;
+    float vv[PMAX], sv[PMAX];
+    int iv[PMAX];
+#pragma unroll
+    for (int q = 0; q < PMAX; ++q) {
+        const int p = threadIdx.x + q * CTL_THREADS;
+        const bool ok = p < n_part;
+        vv[q] = ok ? ldg_cg_f32(pv + (size_t)p * pstride) : -INFINITY;
+        sv[q] = ok ? ldg_cg_f32(ps + (size_t)p * pstride) : 0.f;
+        iv[q] = ok ? pi[(size_t)p * pstride] : 0x7fffffff;
+    }
+    const float k = ldg_cg_f32(kp);
+    float v = -INFINITY;
+    int idx = 0x7fffffff;
+#pragma unroll
+    for (int q = 0; q < PMAX; ++q)
+        if (vv[q] > v || (vv[q] == v && iv[q] < idx)) { v = vv[q]; idx = iv[q]; }
+    block_argmax(v, idx);
+    if (threadIdx.x == 0) s_max = v;
+    __syncthreads();
+    const float M = s_max;
     float acc = 0.f;
-    for (int p = threadIdx.x; p < n_part; p += CTL_THREADS)
-        acc += ldg_cg_f32(ps + (size_t)p * pstride) * exp2f(k * (ldg_cg_f32(pv + (size_t)p * pstride) - M));
+#pragma unroll
+    for (int q = 0; q < PMAX; ++q) acc += sv[q] * exp2f(k * (vv[q] - M));
     const float total = block_sum(acc);
-    return 1.f / total;
+    token = idx;
+    conf = 1.f / total;
 }
 
 // Draft head, last step: reduce the per-CTA arg-max partials of the streaming LM head into the draft
@@ -104,23 +130,15 @@ __global__ void __launch_bounds__(CTL_THREADS) draft_finalize_embed_kernel(const
     pdl_wait();
     const int c = blockIdx.x;
     const RowDesc rd = a.plan.rows[c];
-    float v = -INFINITY;
-    int idx = 0x7fffffff;
-    for (int p = threadIdx.x; p < a.n_part; p += CTL_THREADS) {
-        const float v2 = ldg_cg_f32(a.B.LPV + (size_t)p * DEL_ROWS_MAX + c);
-        const int i2 = a.B.LPI[(size_t)p * DEL_ROWS_MAX + c];
-        if (v2 > v || (v2 == v && i2 < idx)) { v = v2; idx = i2; }
-    }
-    __shared__ float s_max;
-    block_argmax(v, idx);
+    int idx;
+    float conf;
+    reduce_partials(a.B.LPV + c, a.B.LPI + c, a.B.LPS + c, a.n_part, DEL_ROWS_MAX, a.B.RK + c, idx, conf);
     if (threadIdx.x == 0) {
         s_tok = idx;
-        s_max = v;
         a.B.TOK[rd.seq * (a.D.S + 1) + rd.slot + 1] = idx;
+        a.B.DCONF[rd.seq * (a.D.S + 1) + rd.slot + 1] = conf;
     }
     __syncthreads();
-    const float conf = merged_confidence(a.B.LPV + c, a.B.LPS + c, a.n_part, DEL_ROWS_MAX, s_max, ldg_cg_f32(a.B.RK + c));
-    if (threadIdx.x == 0) a.B.DCONF[rd.seq * (a.D.S + 1) + rd.slot + 1] = conf;
     if (embed_next) write_embedding(a, s_tok, rd.seq, rd.slot + 1);
 }
 
@@ -163,22 +181,13 @@ __global__ void __launch_bounds__(CTL_THREADS) prep_rows_kernel(const CtlArgs a,
 __global__ void __launch_bounds__(CTL_THREADS) shadow_reduce_kernel(const CtlArgs a, const UpdatePlan *up, const float *pv,
                                                                     const int32_t *pi, const float *ps, int n_part, int pstride,
                                                                     int cstride, int row_base) {
-    __shared__ float s_max;
     pdl_launch();
     pdl_wait();
     const int c = blockIdx.x;
-    float v = -INFINITY;
-    int idx = 0x7fffffff;
-    for (int p = threadIdx.x; p < n_part; p += CTL_THREADS) {
-        const float v2 = ldg_cg_f32(pv + (size_t)p * pstride + (size_t)c * cstride);
-        const int i2 = pi[(size_t)p * pstride + (size_t)c * cstride];
-        if (v2 > v || (v2 == v && i2 < idx)) { v = v2; idx = i2; }
-    }
-    block_argmax(v, idx);
-    if (threadIdx.x == 0) s_max = v;
-    __syncthreads();
-    const float conf = merged_confidence(pv + (size_t)c * cstride, ps + (size_t)c * cstride, n_part, pstride, s_max,
-                                         ldg_cg_f32(a.B.RS + row_base + c));
+    int idx;
+    float conf;
+    reduce_partials(pv + (size_t)c * cstride, pi + (size_t)c * cstride, ps + (size_t)c * cstride, n_part, pstride,
+                    a.B.RS + row_base + c, idx, conf);
     if (threadIdx.x == 0) {
         int seq, layer, slot;
         if (locate_row(up, a.D.L, a.mode, row_base + c, seq, layer, slot)) {

@@ -750,7 +750,7 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
         del_destroy(c);
         return DEL_ECUDA;
     }
-    c->tc_ok = (shape->d_model % 64 == 0) &&
+    c->tc_ok = (shape->d_model % 64 == 0) && lmhead_tc_vtiles(shape->vocab) <= 1024 &&   // partials one block reduces
                lmhead_tc_make_map(c->map_x, c->B.XN, (uint64_t)c->R_max + 128, (uint64_t)shape->d_model, 128) == 0 &&
                lmhead_tc_make_map(c->map_w, c->lm_head, (uint64_t)shape->vocab, (uint64_t)shape->d_model, 256) == 0;
     c->pt_host.assign((size_t)c->D.B * c->D.pages_per_seq, 0);

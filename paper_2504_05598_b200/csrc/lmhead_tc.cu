@@ -182,9 +182,12 @@ lmhead_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 }
                 // exp sum relative to the running maximum (rescaled when this chunk raised it)
                 if (best > before) esum *= exp2f(k * (before - best));
+                float part[4] = {0.f, 0.f, 0.f, 0.f};          // four chains instead of one 32-long dependent sum
+                const float kb = k * best;
 #pragma unroll
                 for (int j = 0; j < 32; ++j)
-                    if (v0 + c0 + j < p.V) esum += exp2f(k * (__uint_as_float(r[j]) - best));
+                    if (v0 + c0 + j < p.V) part[j & 3] += exp2f(fmaf(k, __uint_as_float(r[j]), -kb));
+                esum += (part[0] + part[1]) + (part[2] + part[3]);
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();

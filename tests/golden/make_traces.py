@@ -4,11 +4,14 @@ Calls only ``synth`` (seeded inputs) and ``oracle`` (the CPU oracle); nothing fr
 
     python tests/golden/make_traces.py tiny
     python tests/golden/make_traces.py llama2_7b [--gen-len N] [--seqs K]
+    python tests/golden/make_traces.py llama2_7b --exit-mode --gen-len 128     (-> trace_llama2_7b_exit.json)
 
 Output: tests/golden/trace_<config>.json.  Per sequence: the prompt recipe's identifiers, the token
 emitted by the prefill, the initial window's shadow tokens / margins / statistics, and for every round
 E, gamma, g (drafts made), the drafts, every layer's shadow tokens with the top-1 minus top-2 logit
 margin (in 1/1000, capped at 9999), the accepted count, per-layer match counts and the next (E, gamma).
+With --exit-mode (dynamic draft-exiting) also: every shadow token's confidence (in 1e-7), the drafted
+tokens' confidences and the thresholds as full doubles, the stop flag and the decayed confidence sums.
 """
 from __future__ import annotations
 
@@ -31,8 +34,13 @@ def _q(m: np.ndarray):
     return np.minimum(np.floor(m.astype(np.float64) * 1000.0), 9999).astype(int).tolist()
 
 
-def trace_sequence(cfg, weights, seq: int, gen_len: int):
+def _c(conf: np.ndarray):
+    return np.rint(conf * 1e7).astype(np.int64).tolist()
+
+
+def trace_sequence(cfg, weights, seq: int, gen_len: int, exit_mode: bool = False):
     o = oracle.OracleSeq(cfg, weights)
+    o.set_exit_mode(exit_mode)
     prompt = synth.make_prompt(cfg, seq)
     t0 = time.time()
     tok, init = o.prefill(prompt)
@@ -44,6 +52,9 @@ def trace_sequence(cfg, weights, seq: int, gen_len: int):
                  "E": E, "gamma": g},
         "rounds": [],
     }
+    if exit_mode:
+        Stcs, Sfcs, _ = o.get_conf_stats()
+        rec["init"].update({"conf_e7": _c(init.conf), "Stcs": Stcs.tolist(), "Sfcs": Sfcs.tolist(), "tau": init.next_tau})
     out = [int(tok)]
     t0 = time.time()
     while len(out) < gen_len:
@@ -54,6 +65,10 @@ def trace_sequence(cfg, weights, seq: int, gen_len: int):
             "shadow": r.shadow.tolist(), "margin_milli": _q(r.margin), "counts": r.counts.tolist(),
             "next_E": r.next_E, "next_gamma": r.next_gamma, "Sc": Sc.tolist(), "Sn": Sn,
         })
+        if exit_mode:
+            Stcs, Sfcs, _ = o.get_conf_stats()
+            rec["rounds"][-1].update({"conf_e7": _c(r.conf), "draft_conf": r.draft_conf, "stopped": int(r.stopped),
+                                      "tau": r.tau, "next_tau": r.next_tau, "Stcs": Stcs.tolist(), "Sfcs": Sfcs.tolist()})
         out.extend(r.emitted)
         print(f"  seq {seq} round {len(rec['rounds'])}: E={r.E} g={r.g} n={r.n_accept} -> {len(out)}/{gen_len} "
               f"({time.time() - t0:.1f}s)", flush=True)
@@ -69,6 +84,7 @@ def main():
     ap.add_argument("--gen-len", type=int, default=None)
     ap.add_argument("--seqs", type=int, default=None)
     ap.add_argument("--out", default=None)
+    ap.add_argument("--exit-mode", action="store_true")
     a = ap.parse_args()
     cfg = synth.CONFIGS[a.config]
     gen_len = a.gen_len or cfg.gen_len
@@ -80,8 +96,10 @@ def main():
     doc = {"config": cfg.name, "seed": cfg.seed, "prompt_len": cfg.prompt_len, "gen_len": gen_len,
            "e_range": [cfg.e_min, cfg.e_max], "g_range": [cfg.g_min, cfg.g_max], "omega": cfg.omega,
            "oracle_threads": oracle.num_threads(),
-           "sequences": [trace_sequence(cfg, weights, s, gen_len) for s in range(n_seq)]}
-    out = a.out or os.path.join(os.path.dirname(os.path.abspath(__file__)), f"trace_{cfg.name}.json")
+           "exit_mode": bool(a.exit_mode),
+           "sequences": [trace_sequence(cfg, weights, s, gen_len, a.exit_mode) for s in range(n_seq)]}
+    out = a.out or os.path.join(os.path.dirname(os.path.abspath(__file__)),
+                                f"trace_{cfg.name}{'_exit' if a.exit_mode else ''}.json")
     with open(out, "w") as f:
         json.dump(doc, f, separators=(",", ":"))
     print("wrote", out, os.path.getsize(out), "bytes")

@@ -118,12 +118,21 @@ def ref_from_golden(doc, seq_index, prompt) -> SeqRef:
     ref = SeqRef(np.asarray(prompt, dtype=np.int32), s["first_token"], np.array(init["shadow"], dtype=np.int32),
                  np.array(init["margin_milli"], dtype=np.float64) / 1000.0, np.array(init["Sc"]), init["Sn"], init["E"],
                  init["gamma"], [], list(s["tokens"]))
+    exit_mode = bool(doc.get("exit_mode", False))
+    if exit_mode:
+        ref.exit_mode = True
+        ref.init_conf = np.array(init["conf_e7"], dtype=np.float64) / 1e7
+        ref.init_Stcs, ref.init_Sfcs, ref.init_tau = np.array(init["Stcs"]), np.array(init["Sfcs"]), init["tau"]
     for r in s["rounds"]:
-        ref.rounds.append(RoundRef(r["E"], r["gamma"], r["g"], r["n"], r["drafts"], r["emitted"],
-                                   np.array(r["shadow"], dtype=np.int32).reshape(len(r["shadow"]), -1),
-                                   np.array(r["margin_milli"], dtype=np.float64).reshape(len(r["shadow"]), -1) / 1000.0,
-                                   np.array(r["counts"], dtype=np.int32), r["next_E"], r["next_gamma"], np.array(r["Sc"]),
-                                   r["Sn"]))
+        rr = RoundRef(r["E"], r["gamma"], r["g"], r["n"], r["drafts"], r["emitted"],
+                      np.array(r["shadow"], dtype=np.int32).reshape(len(r["shadow"]), -1),
+                      np.array(r["margin_milli"], dtype=np.float64).reshape(len(r["shadow"]), -1) / 1000.0,
+                      np.array(r["counts"], dtype=np.int32), r["next_E"], r["next_gamma"], np.array(r["Sc"]), r["Sn"])
+        if exit_mode:
+            rr.conf = np.array(r["conf_e7"], dtype=np.float64).reshape(len(r["shadow"]), -1) / 1e7
+            rr.draft_conf, rr.stopped, rr.tau, rr.next_tau = list(r["draft_conf"]), bool(r["stopped"]), r["tau"], r["next_tau"]
+            rr.Stcs, rr.Sfcs = np.array(r["Stcs"]), np.array(r["Sfcs"])
+        ref.rounds.append(rr)
     return ref
 
 

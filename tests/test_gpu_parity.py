@@ -254,6 +254,24 @@ def test_confidences_in_fixed_gamma_rounds(small):
         assert rep.conf_compared > 0 and rep.conf_max_rel <= 0.02     # far inside the derived bound in practice
 
 
+def test_dynamic_draft_exiting_full_size():
+    """Llama-2-7B shape with the confidence break, against the stored oracle trace."""
+    name = "llama2_7b"
+    doc = json.load(open(os.path.join(GOLDEN, f"trace_{name}_exit.json")))
+    cfg = synth.CONFIGS[name]
+    w = synth.make_weights(cfg)
+    ctx = make_ctx(cfg, w)
+    ref = ref_from_golden(doc, 0, synth.make_prompt(cfg, 0))
+    assert ref.exit_mode
+    rep = run_sequence(ctx, 0, ref, doc["gen_len"])
+    stops = sum(r.stopped for r in ref.rounds)
+    print(f"{name} (draft-exiting): rounds {rep.rounds} stops {stops} decisions {rep.decisions} decision flips "
+          f"{rep.decision_flips} conf compared {rep.conf_compared} max rel err {rep.conf_max_rel:.2e} flips {rep.flips} "
+          f"resyncs {rep.resyncs}")
+    assert rep.ok(), rep.failures[:8]
+    assert rep.decisions > 0 and rep.decision_flips <= max(2, rep.decisions // 10)
+
+
 def test_streaming_lm_head_full_size():
     import paper_2504_05598_b200 as dl
     name = "llama2_7b"
