@@ -164,6 +164,12 @@ int del_round(del_ctx *ctx, del_round_out *out);
  * (gamma = 0: plain auto-regressive decoding).  E <= 0 restores the dynamic choice. */
 int del_set_policy(del_ctx *ctx, int seq, int E, int gamma);
 
+/* The paper's baseline FS(E-gamma) on the same round (Sec. 5.1): fixed exit layer E, the speculation length
+ * starts at gamma0 (>= 1) and moves by +1 after a round whose drafts were all accepted and by -1 after a
+ * round with a rejection, within [max(1, g_min), g_max].  (The baseline LS(E-gamma) is del_set_policy.)
+ * del_set_policy with E <= 0 ends it. */
+int del_set_policy_fs(del_ctx *ctx, int seq, int E, int gamma0);
+
 /* Dynamic draft-exiting (Sec. 4.4, Algorithm 1) for a sequence: mode 1 lets the draft loop run for up to
  * g_max tokens (del_round) or the given gamma (del_draft) and ends it at the first token whose
  * confidence (top-1 softmax probability of the exit head, fp32) is below the threshold of layer E from

@@ -92,6 +92,9 @@ def lib():
     L.ora_tpl.argtypes = [f64, i32, i32, i32]
     L.ora_select.argtypes = [vp, f64, i32, i32, i32, i32, i32, C.POINTER(i32), C.POINTER(i32)]
     L.ora_num_threads.restype = C.c_int
+    L.ora_set_policy_fs.argtypes = [vp, i32, i32]
+    L.ora_fs_next_gamma.restype = i32
+    L.ora_fs_next_gamma.argtypes = [i32, i32, i32, i32, i32]
     L.ora_set_exit_mode.argtypes = [vp, i32]
     L.ora_get_conf_stats.argtypes = [vp, vp, vp, vp]
     L.ora_set_conf_stats.argtypes = [vp, vp, vp]
@@ -164,6 +167,10 @@ class OracleSeq:
     # ---- policy / state
     def set_policy(self, E: int, gamma: int):
         lib().ora_set_policy(self._h, E, gamma)
+
+    def set_policy_fs(self, E: int, gamma0: int):
+        """Baseline FS(E-gamma): fixed exit layer, speculation length moved by +-1 per round."""
+        lib().ora_set_policy_fs(self._h, E, gamma0)
 
     @property
     def T(self) -> int:
@@ -299,6 +306,10 @@ def confidence(logits: np.ndarray) -> float:
 
 def threshold(Stcs: float, Sc: float, Sfcs: float, Smis: float) -> float:
     return lib().ora_threshold(Stcs, Sc, Sfcs, Smis)
+
+
+def fs_next_gamma(gamma: int, g: int, n: int, g_min: int, g_max: int) -> int:
+    return lib().ora_fs_next_gamma(gamma, g, n, g_min, g_max)
 
 
 def silu(x: float) -> float:

@@ -32,6 +32,7 @@ struct ora_seq {
     int32_t x_in;       /* token to be fed at position T */
     int32_t E, gamma;   /* choice for the next round */
     int32_t fixed_E, fixed_gamma;
+    int32_t fs_mode;    /* 1: fixed exit layer, speculation length steered by the +-1 controller (baseline FS) */
     double *Sc;         /* [L], index l-1; Sc[L-1] (layer L) tracked too: it must equal Sn */
     double Sn;
     double *Stcs, *Sfcs; /* [L] decayed confidence sums over matched / mismatched shadow tokens (Sec. 4.4) */
@@ -198,7 +199,23 @@ void ora_seq_destroy(ora_seq *s) {
 void ora_set_policy(ora_seq *s, int32_t fixed_E, int32_t fixed_gamma) {
     s->fixed_E = fixed_E;
     s->fixed_gamma = fixed_gamma;
+    s->fs_mode = 0;
     if (fixed_E > 0) { s->E = fixed_E; s->gamma = fixed_gamma; }
+}
+
+void ora_set_policy_fs(ora_seq *s, int32_t fixed_E, int32_t gamma0) {
+    ora_set_policy(s, fixed_E, gamma0);
+    s->fs_mode = 1;
+}
+
+/* The FS baseline of Sec. 5.1: one more draft next time if every draft of this round was accepted, one
+ * fewer if any was rejected.  The paper gives no bounds; here the length stays within [max(1, g_min),
+ * g_max] (at 0 nothing could ever be accepted again) and a round without drafts changes nothing. */
+int32_t ora_fs_next_gamma(int32_t gamma, int32_t g, int32_t n, int32_t g_min, int32_t g_max) {
+    const int32_t lo = g_min > 1 ? g_min : 1;
+    if (g < 1) return gamma;
+    if (n == g) return gamma + 1 > g_max ? g_max : gamma + 1;
+    return gamma - 1 < lo ? lo : gamma - 1;
 }
 
 int32_t ora_committed_len(const ora_seq *s) { return s->T; }
@@ -424,8 +441,13 @@ void ora_select(const double *Sc, double Sn, int32_t L, int32_t e_min, int32_t e
     *gamma = bg;
 }
 
-static void choose_next(ora_seq *s) {
+static void choose_next(ora_seq *s, int32_t g, int32_t n) {
     const ora_shape *sh = &s->sh;
+    if (s->fixed_E > 0 && s->fs_mode) {
+        s->E = s->fixed_E;
+        s->gamma = ora_fs_next_gamma(s->gamma, g, n, sh->g_min, sh->g_max);
+        return;
+    }
     if (s->fixed_E > 0) { s->E = s->fixed_E; s->gamma = s->fixed_gamma; return; }
     ora_select(s->Sc, s->Sn, sh->n_layers, sh->e_min, sh->e_max, sh->g_min, sh->g_max, &s->E, &s->gamma);
 }
@@ -472,7 +494,7 @@ int32_t ora_prefill(ora_seq *s, const int32_t *prompt, int32_t P, int32_t *shado
     s->T = P;
     s->x_in = sd[(size_t)(L - 1) * W + (W - 1)];
     free(sd);
-    choose_next(s);
+    choose_next(s, 0, 0);
     if (info) {
         memset(info, 0, sizeof(*info));
         info->n_emitted = 1;
@@ -558,7 +580,7 @@ int ora_round(ora_seq *s, int32_t remaining, ora_round_info *info, int32_t *shad
     s->T += n + 1;
     s->x_in = verified[n];
     free(sd);
-    choose_next(s);
+    choose_next(s, g, n);
     if (info) { info->next_E = s->E; info->next_gamma = s->gamma; info->Sn = s->Sn; info->next_tau = s->tau[s->E - 1]; }
     return 0;
 }

@@ -75,6 +75,11 @@ void ora_seq_destroy(ora_seq *s);
  * E <= 0 restores the dynamic selection. */
 void ora_set_policy(ora_seq *s, int32_t fixed_E, int32_t fixed_gamma);
 
+/* Baseline FS(E-gamma) of Sec. 5.1: fixed exit layer, the speculation length starts at gamma0 and moves by
+ * +1 after a round whose drafts were all accepted, by -1 after a round with a rejection. */
+void ora_set_policy_fs(ora_seq *s, int32_t fixed_E, int32_t gamma0);
+int32_t ora_fs_next_gamma(int32_t gamma, int32_t g, int32_t n, int32_t g_min, int32_t g_max);
+
 /* Prefill over the prompt, initial statistics from the last init_window positions, first token and
  * first (E, gamma).  shadow/margin (may be NULL): [n_layers][init_window] row-major, layer 1 first,
  * only the first W = min(init_window, n_prompt) columns are written.  Returns the first token. */

@@ -28,7 +28,7 @@ EXPORTS = ["del_workspace_bytes", "del_init", "del_prefill", "del_draft", "del_v
            "del_select", "del_round", "del_set_policy", "del_get_stats", "del_set_stats", "del_get_shadow",
            "del_get_drafts", "del_force_token", "del_get_hidden", "del_debug_logits", "del_get_kv", "del_committed_len", "del_release",
            "del_launch_count", "del_get_traffic", "del_set_flags", "del_get_kernel_times", "del_head_argmax_static",
-           "del_set_exit_mode", "del_get_conf_stats", "del_set_conf_stats", "del_get_conf", "del_strerror", "del_last_cuda_error", "del_destroy"]
+           "del_set_policy_fs", "del_set_exit_mode", "del_get_conf_stats", "del_set_conf_stats", "del_get_conf", "del_strerror", "del_last_cuda_error", "del_destroy"]
 
 
 class Shape(C.Structure):
@@ -96,6 +96,8 @@ def load_library(build_if_missing: bool = True):
     L.del_get_stats.argtypes = [vp, ci, vp, C.POINTER(C.c_double), C.POINTER(i32), C.POINTER(i32)]
     L.del_set_stats.restype = ci
     L.del_set_stats.argtypes = [vp, ci, vp, C.c_double, i32, i32]
+    L.del_set_policy_fs.restype = ci
+    L.del_set_policy_fs.argtypes = [vp, ci, ci, ci]
     L.del_set_exit_mode.restype = ci
     L.del_set_exit_mode.argtypes = [vp, ci, ci]
     L.del_get_conf_stats.restype = ci
@@ -272,6 +274,10 @@ class DelContext:
     def set_stats(self, seq: int, Sc, Sn: float, E: int, gamma: int):
         Sc = np.ascontiguousarray(Sc, dtype=np.float64)
         self._ck(self.lib.del_set_stats(self._h, seq, Sc.ctypes.data, float(Sn), int(E), int(gamma)), "del_set_stats")
+
+    def set_policy_fs(self, seq: int, E: int, gamma0: int):
+        """Baseline FS(E-gamma): fixed exit layer, speculation length moved by +-1 per round."""
+        self._ck(self.lib.del_set_policy_fs(self._h, seq, E, gamma0), "del_set_policy_fs")
 
     def set_exit_mode(self, seq: int, on: bool):
         """Dynamic draft-exiting: the draft loop stops at the first token whose confidence is below the threshold."""

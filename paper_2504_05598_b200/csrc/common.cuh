@@ -36,7 +36,8 @@ struct SeqState {
     double Sn;
     int32_t E, gamma;            // choice for the next round
     int32_t fixed_E, fixed_gamma;
-    int32_t pad[2];
+    int32_t fs_mode;             // 1: fixed E, gamma moved by the +-1 controller
+    int32_t pad;
 };
 
 // Device view of the model shape and of the workspace carve-up (passed by value to kernels).

@@ -295,7 +295,15 @@ __global__ void __launch_bounds__(64) select_kernel(const CtlArgs a, const Updat
     const int seq = up->s[blockIdx.x].seq, L = a.D.L;
     SeqState *st = a.B.ST + seq;
     int E = a.e_min, G = a.g_min;
-    if (st->fixed_E > 0) {
+    if (st->fixed_E > 0 && st->fs_mode) {
+        // baseline FS (Sec. 5.1): one more draft after a round whose drafts were all accepted, one fewer after
+        // a rejection, within [max(1, g_min), g_max]; a round without drafts changes nothing
+        E = st->fixed_E;
+        G = st->gamma;
+        const int g = up->s[blockIdx.x].g, n = out[seq].n_accept;
+        const int lo = a.g_min > 1 ? a.g_min : 1;
+        if (a.mode == 0 && g >= 1) G = (n == g) ? min(G + 1, a.g_max) : max(G - 1, lo);
+    } else if (st->fixed_E > 0) {
         E = st->fixed_E;
         G = st->fixed_gamma;
     } else {

@@ -23,6 +23,7 @@ struct SeqHost {
     int remaining = 0;       // tokens still to emit
     int E = 0, gamma = 0;    // choice for the next round
     int fixed_E = 0, fixed_gamma = 0;
+    int fs_mode = 0;         // fixed E with the +-1 speculation-length controller
     int phase = 0;           // 0 idle, 1 drafted, 2 verified
     int cur_E = 0, cur_g = 0, cur_gamma = 0;
     int exit_mode = 0;       // 1: the draft loop stops on a low confidence (checked by the host per step)
@@ -903,6 +904,7 @@ int del_select(del_ctx *c, int sq, int32_t *E, int32_t *gamma) {
     memset(up, 0, sizeof(*up));
     up->n_seq = 1;
     up->s[0].seq = sq;
+    up->s[0].g = s.cur_g;            // the +-1 controller looks at the round just accepted
     CK(cudaMemcpyAsync(c->up_dev + 1, up, sizeof(UpdatePlan), cudaMemcpyHostToDevice, c->st));
     CtlArgs ca = ctl_base(c, -1);
     LAUNCH(launch_select(ca, c->up_dev + 1, c->out_dev, 1, c->st, pdl(c)));
@@ -926,7 +928,7 @@ int del_round(del_ctx *c, del_round_out *out) {
         if (!s.active || s.remaining < 1) continue;
         if (s.phase != 0) return DEL_ESTATE;
         const int E = s.fixed_E > 0 ? s.fixed_E : s.E;
-        const int gamma = s.fixed_E > 0 ? s.fixed_gamma : s.gamma;
+        const int gamma = (s.fixed_E > 0 && !s.fs_mode) ? s.fixed_gamma : s.gamma;
         // Algorithm 1: with draft-exiting the loop may run up to d_max tokens, otherwise gamma tokens
         const int g = clip_gamma(s, s.exit_mode ? c->sh.g_max : gamma);
         int rc = ensure_pages(c, sq, s.T + g + 1);
@@ -950,20 +952,28 @@ int del_round(del_ctx *c, del_round_out *out) {
     return DEL_OK;
 }
 
-int del_set_policy(del_ctx *c, int sq, int E, int gamma) {
+static int set_policy(del_ctx *c, int sq, int E, int gamma, int fs) {
     if (!seq_ok(c, sq)) return DEL_EINVAL;
     if (E > 0 && (E >= c->D.L || gamma < 0 || gamma > c->sh.g_max)) return DEL_EINVAL;
+    if (fs && (E < 1 || gamma < 1)) return DEL_EINVAL;
     SeqHost &s = c->seq[sq];
     s.fixed_E = E > 0 ? E : 0;
     s.fixed_gamma = E > 0 ? gamma : 0;
+    s.fs_mode = fs;
+    if (fs) s.gamma = gamma;
     CK(cudaStreamSynchronize(c->st));
     SeqState st;
     CK(cudaMemcpy(&st, c->B.ST + sq, sizeof(st), cudaMemcpyDeviceToHost));
     st.fixed_E = s.fixed_E;
     st.fixed_gamma = s.fixed_gamma;
+    st.fs_mode = fs;
+    if (fs) st.gamma = gamma;
     CK(cudaMemcpy(c->B.ST + sq, &st, sizeof(st), cudaMemcpyHostToDevice));
     return DEL_OK;
 }
+
+int del_set_policy(del_ctx *c, int sq, int E, int gamma) { return set_policy(c, sq, E, gamma, 0); }
+int del_set_policy_fs(del_ctx *c, int sq, int E, int gamma0) { return set_policy(c, sq, E, gamma0, 1); }
 
 int del_get_stats(del_ctx *c, int sq, double *Sc, double *Sn, int32_t *E, int32_t *gamma) {
     if (!seq_ok(c, sq)) return DEL_EINVAL;

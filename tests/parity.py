@@ -86,7 +86,7 @@ class Report:
         return not self.failures
 
 
-def ref_from_oracle(cfg, weights, prompt, gen_len=None, policy=None, exit_mode=False) -> SeqRef:
+def ref_from_oracle(cfg, weights, prompt, gen_len=None, policy=None, exit_mode=False, policy_fs=None) -> SeqRef:
     """Runs the oracle now (small models)."""
     import oracle
     o = oracle.OracleSeq(cfg, weights)
@@ -95,6 +95,8 @@ def ref_from_oracle(cfg, weights, prompt, gen_len=None, policy=None, exit_mode=F
     o.set_exit_mode(exit_mode)
     n_tok = gen_len or cfg.gen_len
     tok, init = o.prefill(prompt)
+    if policy_fs:
+        o.set_policy_fs(*policy_fs)
     Sc, Sn, E, g = o.get_stats()
     Stcs, Sfcs, _ = o.get_conf_stats()
     ref = SeqRef(np.asarray(prompt, dtype=np.int32), tok, init.shadow, init.margin, Sc, Sn, E, g, [], [tok],
@@ -285,10 +287,13 @@ def compare_round(ctx, seq, out, r: RoundRef, rep: Report, check_choice=True) ->
     return True
 
 
-def run_sequence(ctx, seq, ref: SeqRef, total_tokens: int, policy=None, max_rounds=None) -> Report:
-    """Prefill + rounds of one sequence through del_round, compared with the oracle's trace."""
+def run_sequence(ctx, seq, ref: SeqRef, total_tokens: int, policy=None, max_rounds=None, policy_fs=None) -> Report:
+    """Prefill + rounds of one sequence through del_round, compared with the oracle's trace.
+    policy = (E, gamma) fixes both; policy_fs = (E, gamma0) fixes E and lets the +-1 controller move gamma."""
     rep = Report()
     compare_init(ctx, seq, ref, total_tokens, rep, policy)
+    if policy_fs:
+        ctx.set_policy_fs(seq, *policy_fs)
     done = 1
     for k, r in enumerate(ref.rounds):
         if max_rounds is not None and k >= max_rounds:
@@ -301,7 +306,8 @@ def run_sequence(ctx, seq, ref: SeqRef, total_tokens: int, policy=None, max_roun
             _resync(ctx, seq, ref, done, r.Sc, r.Sn, r.next_E, r.next_gamma, total_tokens, r.Stcs, r.Sfcs)
             if policy:
                 ctx.set_policy(seq, *policy)
-
+            if policy_fs:
+                ctx.set_policy_fs(seq, policy_fs[0], r.next_gamma)
         if len(rep.failures) > 20:
             break
     return rep

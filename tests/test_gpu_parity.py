@@ -238,6 +238,18 @@ def test_dynamic_draft_exiting_against_oracle(small):
     assert rep.decisions > 0 and rep.decision_flips <= max(1, rep.decisions // 10)
 
 
+def test_fs_baseline_policy_against_oracle(small):
+    """Baseline FS(E-gamma) of Sec. 5.1 on the same kernels: fixed exit layer, gamma moved by +-1 on the device."""
+    cfg, w, ctx = small
+    fs = (cfg.e_min, 3)
+    ref = ref_from_oracle(cfg, w, synth.make_prompt(cfg), policy_fs=fs)
+    rep = run_sequence(ctx, 0, ref, cfg.gen_len, policy_fs=fs)
+    gammas = [r.gamma for r in ref.rounds]
+    print(f"{cfg.name} (FS): rounds {rep.rounds} gamma trajectory {gammas[:12]} flips {rep.flips}")
+    assert rep.ok(), rep.failures[:5]
+    assert rep.rounds == len(ref.rounds) and len(set(gammas)) > 1
+
+
 def test_confidences_in_fixed_gamma_rounds(small):
     """The confidence statistics are maintained in every mode; here with the streaming LM head as well."""
     import paper_2504_05598_b200 as dl

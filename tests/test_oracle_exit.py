@@ -179,3 +179,34 @@ def test_exit_mode_off_is_the_fixed_gamma_round(case):
     r = o.round(cfg.gen_len - 1)
     assert r.g == g and not r.stopped
     o.close()
+
+
+# ---------------------------------------------------------------- baseline policies on the same round (Sec. 5.1)
+def test_fs_controller_rule():
+    # +1 after a round whose drafts were all accepted, -1 after a rejection, inside [max(1, g_min), g_max]
+    assert oracle.fs_next_gamma(4, 4, 4, 1, 12) == 5
+    assert oracle.fs_next_gamma(4, 4, 3, 1, 12) == 3
+    assert oracle.fs_next_gamma(4, 4, 0, 1, 12) == 3
+    assert oracle.fs_next_gamma(12, 12, 12, 1, 12) == 12
+    assert oracle.fs_next_gamma(1, 1, 0, 0, 12) == 1          # never down to 0: nothing could be accepted again
+    assert oracle.fs_next_gamma(2, 2, 1, 2, 12) == 2
+    assert oracle.fs_next_gamma(6, 3, 3, 1, 12) == 7          # clipped round (g < gamma), all accepted
+    assert oracle.fs_next_gamma(6, 0, 0, 1, 12) == 6          # no drafts: unchanged
+
+
+def test_fs_policy_stream_and_trajectory(case):
+    cfg, w, prompt = case
+    want = _greedy_stream(cfg, w, prompt, cfg.gen_len)
+    o = oracle.OracleSeq(cfg, w)
+    o.prefill(prompt)
+    E, g0 = cfg.e_min, 3
+    o.set_policy_fs(E, g0)
+    out, gamma = want[:1], g0
+    while len(out) < cfg.gen_len:
+        r = o.round(cfg.gen_len - len(out))
+        assert (r.E, r.gamma) == (E, gamma)
+        gamma = oracle.fs_next_gamma(gamma, r.g, r.n_accept, cfg.g_min, cfg.g_max)
+        assert (r.next_E, r.next_gamma) == (E, gamma)
+        out.extend(r.emitted)
+    assert out == want
+    o.close()
