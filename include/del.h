@@ -222,7 +222,8 @@ int64_t del_launch_count(const del_ctx *ctx);
 int del_get_traffic(const del_ctx *ctx, int64_t *h2d_bytes, int64_t *d2h_bytes);
 /* Switches of the launch machinery (bit 0: programmatic dependent launch, bit 1: CUDA graphs for
  * single-sequence rounds, bit 2: tcgen05 LM head instead of the streaming one, bit 3: record CUDA
- * events around every launch).  Returns the previous flags. */
+ * events around every launch, bit 4: one weight-streaming CTA per SM, bit 5: prefill every prompt
+ * position through the decode kernels instead of the tensor-core GEMMs).  Returns the previous flags. */
 int del_set_flags(del_ctx *ctx, int flags);
 
 /* With flag bit 3 set, per kernel class (0 QKV, 1 attention, 2 O-proj, 3 gate/up, 4 down, 5 draft LM

@@ -14,7 +14,7 @@ namespace {
 
 constexpr int PLAN_RING = 192;
 constexpr int CTR_RING = 4096;
-constexpr int FLAG_PDL = 1, FLAG_GRAPH = 2, FLAG_TC = 4, FLAG_TIMING = 8, FLAG_ONECTA = 16;
+constexpr int FLAG_PDL = 1, FLAG_GRAPH = 2, FLAG_TC = 4, FLAG_TIMING = 8, FLAG_ONECTA = 16, FLAG_NO_BULK_PREFILL = 32;
 enum { CLS_QKV = 0, CLS_ATTN, CLS_OPROJ, CLS_GATEUP, CLS_DOWN, CLS_LMHEAD, CLS_LMSTACK, CLS_OTHER, CLS_N };
 
 struct SeqHost {
@@ -67,6 +67,12 @@ struct del_ctx {
     void *stage_host = nullptr;                            // small pinned scratch
     float *dbg_dev = nullptr;                              // [V] debug logits / kv rows
     alignas(64) unsigned char map_x[128], map_w[128];     // tensor maps of the stacked rows and of W_lm
+    // bulk prefill on the tensor cores: chunk buffers in the workspace, tensor maps of them and of every layer's weights
+    struct TMap { alignas(64) unsigned char b[128]; };
+    PfArgs pf;                                            // buffer pointers (the per-launch fields are filled in later)
+    TMap pf_xs, pf_att, pf_xm, pf_act;
+    std::vector<TMap> pf_wq, pf_wk, pf_wv, pf_wo, pf_wg, pf_wu, pf_wd;
+    bool pf_ok = false;
     bool tc_ok = false;
     int64_t launches = 0, h2d_bytes = 0, d2h_bytes = 0;
     // optional per-launch timing (FLAG_TIMING): events around every launch, summed per kernel class
@@ -84,10 +90,12 @@ struct del_ctx {
 namespace {
 
 size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max, int &n_vtiles,
-                 UpdatePlan **up_dev, del_round_out **out_dev, float **dbg_dev) {
+                 UpdatePlan **up_dev, del_round_out **out_dev, float **dbg_dev, PfArgs *pf) {
     D.L = s.n_layers; D.d = s.d_model; D.nh = s.n_heads; D.nkv = s.n_kv_heads; D.hd = s.head_dim; D.F = s.d_ffn; D.V = s.vocab;
     D.B = s.max_batch;
-    D.S = std::max(s.g_max + 1, s.init_window);
+    // slots of the hidden stack per sequence: what a round needs (g_max + 1 rows, the prefill window), raised to
+    // a full pass so that the prefill streams the weights once per DEL_ROWS_MAX prompt positions
+    D.S = std::max(std::max(s.g_max + 1, s.init_window), DEL_ROWS_MAX);
     D.max_seq = s.max_seq; D.page_size = s.page_size; D.pages_per_seq = s.max_seq / s.page_size;
     D.n_sst = s.d_model / 16;
     D.eps = s.rms_eps;
@@ -134,6 +142,19 @@ size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max
     *up_dev = c.take<UpdatePlan>(base, 2);
     *out_dev = c.take<del_round_out>(base, (size_t)D.B);
     *dbg_dev = c.take<float>(base, (size_t)std::max(D.V, 2 * D.nkv * D.hd));
+    // chunk buffers of the bulk prefill (PF_ROWS prompt positions)
+    PfArgs pfa;
+    memset(&pfa, 0, sizeof(pfa));
+    pfa.n_ssp = (D.d + 255) / 256;
+    pfa.H = c.take<float>(base, (size_t)PF_ROWS * D.d);
+    pfa.XS = c.take<bf16>(base, (size_t)PF_ROWS * D.d);
+    pfa.SSP = c.take<float>(base, (size_t)PF_ROWS * pfa.n_ssp);
+    pfa.Q = c.take<bf16>(base, (size_t)PF_ROWS * qd);
+    pfa.ATT = c.take<bf16>(base, (size_t)PF_ROWS * qd);
+    pfa.XM = c.take<bf16>(base, (size_t)PF_ROWS * D.d);
+    pfa.SSPM = c.take<float>(base, (size_t)PF_ROWS * pfa.n_ssp);
+    pfa.ACT = c.take<bf16>(base, (size_t)PF_ROWS * D.F);
+    if (pf) *pf = pfa;
     return (c.off + 255) & ~(size_t)255;
 }
 
@@ -534,6 +555,59 @@ int draft_with_exit(del_ctx *c, std::vector<Job> &jobs) {
     return DEL_OK;
 }
 
+// ---- bulk of a prompt (positions 0 .. n_pos-1 of sequence sq) through the tensor-core GEMMs: only the KV
+// cache is produced; chunks of PF_ROWS positions, attention in passes of DEL_ROWS_MAX query rows
+int prefill_bulk(del_ctx *c, int sq, int n_pos) {
+    const Dims &D = c->D;
+    const bool P = pdl(c);
+    for (int p0 = 0; p0 < n_pos; p0 += PF_ROWS) {
+        PfArgs a = c->pf;
+        a.M = std::min(PF_ROWS, n_pos - p0);
+        a.seq = sq;
+        a.pos0 = p0;
+        cudaError_t e = launch_prefill_embed(a, c->tok_emb, c->B.PROMPT_ALL, c->attn_norm[0], c->st);
+        if (e != cudaSuccess) return fail(c, e);
+        ++c->launches;
+        for (int l = 1; l <= D.L; ++l) {
+            a.layer = l;
+            a.K = D.d;
+            a.n_ntiles = prefill_tc_ntiles(PF_QKV, D);
+            LAUNCH(launch_prefill_gemm(PF_QKV, c->pf_xs.b, c->pf_wq[l - 1].b, c->pf_wk[l - 1].b, c->pf_wv[l - 1].b, a, c->n_sms, c->st, P));
+            if (l == D.L) break;             // the last layer's keys and values are all that is needed of it
+            for (int r0 = 0; r0 < a.M; r0 += DEL_ROWS_MAX) {
+                AttnArgs at;
+                memset(&at, 0, sizeof(at));
+                at.D = D;
+                at.B = c->B;
+                at.B.Q = a.Q + (size_t)r0 * D.nh * D.hd;
+                at.B.ATT = a.ATT + (size_t)r0 * D.nh * D.hd;
+                const int nr = std::min(DEL_ROWS_MAX, a.M - r0);
+                at.plan.m = nr;
+                at.plan.n_seg = 1;
+                at.plan.seg[0] = Segment{sq, 0, nr, p0 + r0};
+                at.layer = l;
+                const int pages = (p0 + r0 + nr + 15) / 16;
+                const int R = nr * (D.nh / D.nkv), n_mt = (R + 15) / 16;
+                at.n_splits = attention_splits(pages, D.nkv, n_mt >= 3 ? 4 : n_mt, c->n_sms);
+                at.max_rows = nr;
+                LAUNCH(launch_attention(at, 1, c->st, P));
+            }
+            a.K = D.nh * D.hd;
+            a.n_ntiles = prefill_tc_ntiles(PF_OPROJ, D);
+            a.gain = c->ffn_norm[l - 1];
+            LAUNCH(launch_prefill_gemm(PF_OPROJ, c->pf_att.b, c->pf_wo[l - 1].b, nullptr, nullptr, a, c->n_sms, c->st, P));
+            a.K = D.d;
+            a.n_ntiles = prefill_tc_ntiles(PF_GATEUP, D);
+            LAUNCH(launch_prefill_gemm(PF_GATEUP, c->pf_xm.b, c->pf_wg[l - 1].b, c->pf_wu[l - 1].b, nullptr, a, c->n_sms, c->st, P));
+            a.K = D.F;
+            a.n_ntiles = prefill_tc_ntiles(PF_DOWN, D);
+            a.gain = c->attn_norm[l];        // the next layer's attention norm (l < L here)
+            LAUNCH(launch_prefill_gemm(PF_DOWN, c->pf_act.b, c->pf_wd[l - 1].b, nullptr, nullptr, a, c->n_sms, c->st, P));
+        }
+    }
+    return DEL_OK;
+}
+
 // ---- verify (a4-a5)
 int enqueue_verify(del_ctx *c, const std::vector<Job> &jobs) {
     int rc = plan_begin(c, (int)jobs.size() + 2);
@@ -698,7 +772,7 @@ extern "C" {
 size_t del_workspace_bytes(const del_shape *shape) {
     if (validate(shape) != DEL_OK) return 0;
     Dims D; Buffers B; int R, nv; UpdatePlan *u; del_round_out *o; float *dbg;
-    return carve_all(*shape, nullptr, D, B, R, nv, &u, &o, &dbg);
+    return carve_all(*shape, nullptr, D, B, R, nv, &u, &o, &dbg, nullptr);
 }
 
 int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const del_kv *kv, void *workspace,
@@ -714,7 +788,7 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
     del_ctx *c = new (std::nothrow) del_ctx();
     if (!c) return DEL_ENOSPC;
     c->sh = *shape;
-    carve_all(*shape, workspace, c->D, c->B, c->R_max, c->n_vtiles, &c->up_dev, &c->out_dev, &c->dbg_dev);
+    carve_all(*shape, workspace, c->D, c->B, c->R_max, c->n_vtiles, &c->up_dev, &c->out_dev, &c->dbg_dev, &c->pf);
     c->B.KP = (bf16 *)kv->k_pages; c->B.VP = (bf16 *)kv->v_pages; c->B.PT = kv->page_table;
     c->B.rope_cos = w->rope_cos; c->B.rope_sin = w->rope_sin;
     c->tok_emb = (const bf16 *)w->tok_emb; c->final_norm = (const bf16 *)w->final_norm; c->lm_head = (const bf16 *)w->lm_head;
@@ -754,6 +828,31 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
     c->tc_ok = (shape->d_model % 64 == 0) && lmhead_tc_vtiles(shape->vocab) <= 1024 &&   // partials one block reduces
                lmhead_tc_make_map(c->map_x, c->B.XN, (uint64_t)c->R_max + 128, (uint64_t)shape->d_model, 128) == 0 &&
                lmhead_tc_make_map(c->map_w, c->lm_head, (uint64_t)shape->vocab, (uint64_t)shape->d_model, 256) == 0;
+    {
+        // tensor maps of the bulk prefill: activations in boxes of 128 rows, weights of 256 (gate / up: 128)
+        const uint64_t d = shape->d_model, qd = (uint64_t)shape->n_heads * shape->head_dim,
+                       kvd = (uint64_t)shape->n_kv_heads * shape->head_dim, F = shape->d_ffn;
+        bool ok = lmhead_tc_make_map(c->pf_xs.b, c->pf.XS, PF_ROWS, d, 128) == 0 &&
+                  lmhead_tc_make_map(c->pf_att.b, c->pf.ATT, PF_ROWS, qd, 128) == 0 &&
+                  lmhead_tc_make_map(c->pf_xm.b, c->pf.XM, PF_ROWS, d, 128) == 0 &&
+                  lmhead_tc_make_map(c->pf_act.b, c->pf.ACT, PF_ROWS, F, 128) == 0;
+        auto maps = [&](std::vector<del_ctx::TMap> &dst, const std::vector<const bf16 *> &w, uint64_t rows, uint64_t cols, uint32_t box) {
+            dst.resize(L);
+            for (int l = 0; l < L && ok; ++l) ok = lmhead_tc_make_map(dst[l].b, w[l], rows, cols, box) == 0;
+        };
+        maps(c->pf_wq, c->wq, qd, d, 256);
+        maps(c->pf_wk, c->wk, kvd, d, 256);
+        maps(c->pf_wv, c->wv, kvd, d, 256);
+        maps(c->pf_wo, c->wo, d, qd, 256);
+        maps(c->pf_wg, c->w_gate, F, d, 128);
+        maps(c->pf_wu, c->w_up, F, d, 128);
+        maps(c->pf_wd, c->w_down, d, F, 256);
+        c->pf_ok = ok;
+        c->pf.D = c->D;
+        c->pf.KP = c->B.KP; c->pf.VP = c->B.VP; c->pf.PT = c->B.PT;
+        c->pf.rope_cos = c->B.rope_cos; c->pf.rope_sin = c->B.rope_sin;
+        c->pf.err = c->B.ERR;
+    }
     c->pt_host.assign((size_t)c->D.B * c->D.pages_per_seq, 0);
     for (int p = shape->n_pages - 1; p >= 0; --p) c->free_pages.push_back(p);
     *out = c;
@@ -795,7 +894,13 @@ int del_prefill(del_ctx *c, int sq, const int32_t *prompt, int n_prompt, int max
     // chunks of <= S positions; the last chunk is exactly the window so that its hidden states stay
     // in slots 0..W-1 of the stack
     std::vector<std::pair<int, int>> chunks;
-    for (int p0 = 0; p0 < n_prompt - W; p0 += S) chunks.push_back({p0, std::min(S, n_prompt - W - p0)});
+    int p_bulk = 0;                          // positions [0, p_bulk) go through the tensor-core prefill
+    if (c->pf_ok && !(c->flags & FLAG_NO_BULK_PREFILL) && n_prompt - W >= 64) {
+        p_bulk = n_prompt - W;
+        rc = prefill_bulk(c, sq, p_bulk);
+        if (rc) return rc;
+    }
+    for (int p0 = p_bulk; p0 < n_prompt - W; p0 += S) chunks.push_back({p0, std::min(S, n_prompt - W - p0)});
     chunks.push_back({n_prompt - W, W});
     s.T = 0;
     for (auto ch : chunks) {

@@ -79,3 +79,31 @@ int lmhead_tc_make_map(void *map_out, const void *base, uint64_t rows, uint64_t 
 int lmhead_tc_vtiles(int V);
 cudaError_t launch_lmhead_tc(const void *map_x, const void *map_w, float *part_v, int32_t *part_i, float *part_s,
                              const float *row_scale, int n_rows, int V, int d, int32_t *err, int n_sms, cudaStream_t st, bool pdl);
+
+// Prompt prefill on tcgen05 (prefill_tc.cu): tiled GEMMs over up to PF_ROWS prompt positions of one sequence
+// with the layer's element-wise work fused into the epilogues.  All buffers hold PF_ROWS rows.
+#define PF_ROWS 512
+enum { PF_QKV = 0, PF_OPROJ = 1, PF_GATEUP = 2, PF_DOWN = 3 };
+struct PfArgs {
+    Dims D;
+    int32_t M, K;              // valid rows of the chunk, in-features of this GEMM
+    int32_t n_ntiles;          // output tiles of this GEMM (prefill_tc_ntiles)
+    int32_t n_ssp;             // partial sums of squares per row (= output tiles of a d-wide GEMM)
+    int32_t layer, seq, pos0;  // 1-based layer; the rows are positions pos0 .. pos0 + M - 1 of sequence seq
+    float *H;                  // [PF_ROWS][d] residual stream, updated in place
+    bf16 *XS;                  // [PF_ROWS][d] bf16(h * attention-norm gain): input of QKV, written by DOWN
+    float *SSP;                // [PF_ROWS][n_ssp] sums of squares of h per output tile (QKV's 1/rms)
+    bf16 *Q, *ATT;             // [PF_ROWS][nh * hd]
+    bf16 *XM;                  // [PF_ROWS][d] bf16(h_mid * ffn-norm gain), written by OPROJ
+    float *SSPM;               // [PF_ROWS][n_ssp]
+    bf16 *ACT;                 // [PF_ROWS][F]
+    const bf16 *gain;          // OPROJ: ffn-norm gain; DOWN: the next layer's attention-norm gain
+    bf16 *KP, *VP;             // paged cache
+    const int32_t *PT;
+    const float *rope_cos, *rope_sin;
+    int32_t *err;
+};
+int prefill_tc_ntiles(int epi, const Dims &D);
+cudaError_t launch_prefill_gemm(int epi, const void *map_a, const void *map_b0, const void *map_b1, const void *map_b2,
+                                const PfArgs &p, int n_sms, cudaStream_t st, bool pdl);
+cudaError_t launch_prefill_embed(const PfArgs &p, const bf16 *tok_emb, const int32_t *prompt, const bf16 *gain0, cudaStream_t st);

@@ -7,4 +7,7 @@ TINY_GQA = synth.small_variant(TINY, name="tiny_gqa", n_layers=6, n_kv_heads=2, 
                                residual_scaling="decay", e_min=1, e_max=5, g_max=5, emb_scale=10.0,
                                prompt_len=40, gen_len=48, seed=77)
 # ragged shapes: prompt shorter than the initialisation window, odd generation length
+# long prompts: the bulk of the prompt goes through the tensor-core prefill (ragged last row tile)
+TINY_LONG = synth.small_variant(TINY, name="tiny_long", prompt_len=300, gen_len=24, emb_scale=10.0, seed=11)
+TINY_GQA_LONG = synth.small_variant(TINY_GQA, name="tiny_gqa_long", prompt_len=200, gen_len=24, seed=78)
 TINY_SHORT = synth.small_variant(TINY, name="tiny_short", prompt_len=7, gen_len=21, emb_scale=10.0, seed=5)

@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 
 import synth
-from cases import TINY, TINY_GQA, TINY_SHORT
+from cases import TINY, TINY_GQA, TINY_GQA_LONG, TINY_LONG, TINY_SHORT
 from parity import MARGIN, ref_from_golden, ref_from_oracle, run_batch, run_sequence
 
 pytestmark = pytest.mark.gpu
@@ -55,6 +55,41 @@ def test_prefill_hidden_kv_and_logits(small):
         assert np.abs(got - ref).max() <= 3e-2, (l, np.abs(got - ref).max())
         if np.sort(ref)[-1] - np.sort(ref)[-2] > MARGIN:
             assert int(np.argmax(got)) == int(np.argmax(ref))
+
+
+@pytest.mark.parametrize("cfg", [TINY_LONG, TINY_GQA_LONG], ids=lambda c: c.name)
+def test_tensor_core_prefill_against_oracle(cfg):
+    """Prompts longer than the initialisation window: their bulk is prefilled by the tcgen05 GEMMs (only the KV
+    cache comes out of it).  Cached K/V of bulk positions in every layer, the window's hidden states (which
+    attend to those keys), and the rounds that follow must match the oracle; the same through the decode kernels."""
+    import oracle
+    import paper_2504_05598_b200 as dl
+    w = synth.make_weights(cfg)
+    ctx = make_ctx(cfg, w)
+    prompt = synth.make_prompt(cfg)
+    o = oracle.OracleSeq(cfg, w)
+    o.prefill(prompt)
+    P, W = len(prompt), min(cfg.init_window, len(prompt))
+    ref = ref_from_oracle(cfg, w, prompt)
+    for flags in (dl.FLAG_PDL | dl.FLAG_TC, dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_NO_BULK_PREFILL):
+        ctx.set_flags(flags)
+        launches0 = ctx.launch_count()
+        ctx.prefill(0, prompt, cfg.gen_len)
+        n_launch = ctx.launch_count() - launches0
+        for l in range(1, cfg.n_layers + 1):
+            for pos in (0, 1, 15, 16, 127, 128, P - W - 1, P - W, P - 1):
+                k, v = ctx.get_kv(0, l, pos)
+                kr, vr = o.k_row(l, pos), o.v_row(l, pos)
+                assert np.abs(k - kr).max() <= 2e-2 * np.abs(kr).max() + 1e-6, ("k", flags, l, pos)
+                assert np.abs(v - vr).max() <= 2e-2 * np.abs(vr).max() + 1e-6, ("v", flags, l, pos)
+        for l in range(cfg.n_layers + 1):
+            for j in (0, W - 1):
+                r, got = o.hidden(l, j), ctx.get_hidden(0, l, j)
+                assert np.abs(got - r).max() <= 2e-2 * np.abs(r).max() + 1e-6, ("h", flags, l, j)
+        rep = run_sequence(ctx, 0, ref, cfg.gen_len)
+        print(f"{cfg.name} flags {flags}: prefill launches {n_launch}, rounds {rep.rounds} flips {rep.flips}")
+        assert rep.ok(), rep.failures[:5]
+    o.close()
 
 
 def test_dynamic_rounds_match_oracle(small):
