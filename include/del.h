@@ -220,8 +220,8 @@ int64_t del_launch_count(const del_ctx *ctx);
 /* Bytes the library itself copied host->device (plans, page-table entries, prompts) and
  * device->host (round results) since del_init. */
 int del_get_traffic(const del_ctx *ctx, int64_t *h2d_bytes, int64_t *d2h_bytes);
-/* Switches of the launch machinery (bit 0: programmatic dependent launch, bit 1: CUDA graphs for
- * single-sequence rounds, bit 2: tcgen05 LM head instead of the streaming one, bit 3: record CUDA
+/* Switches of the launch machinery (bit 0: programmatic dependent launch, bit 1: reserved,
+ * bit 2: tcgen05 LM head instead of the streaming one, bit 3: record CUDA
  * events around every launch, bit 4: one weight-streaming CTA per SM, bit 5: prefill every prompt
  * position through the decode kernels instead of the tensor-core GEMMs).  Returns the previous flags. */
 int del_set_flags(del_ctx *ctx, int flags);

@@ -35,6 +35,13 @@ struct TcParams {
     int32_t *err;
 };
 
+// 2^x on the special-function unit (one instruction; the confidence score tolerates its 2-ulp error)
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __global__ void __launch_bounds__(TC_THREADS, 1)
 lmhead_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const TcParams p) {
     extern __shared__ unsigned char smem_dyn[];
@@ -126,18 +133,24 @@ lmhead_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), r);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 const float before = best;
+                const int nv = min(32, p.V - (v0 + c0));     // columns of this chunk inside the vocabulary (whole chunk: 32)
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     const float v = __uint_as_float(r[j]);
-                    if (v0 + c0 + j < p.V && v > best) { best = v; bidx = v0 + c0 + j; }
+                    if (j < nv && v > best) { best = v; bidx = v0 + c0 + j; }
                 }
                 // exp sum relative to the running maximum (rescaled when this chunk raised it)
-                if (best > before) esum *= exp2f(k * (before - best));
+                if (best > before) esum *= ex2(k * (before - best));
                 float part[4] = {0.f, 0.f, 0.f, 0.f};          // four chains instead of one 32-long dependent sum
                 const float kb = k * best;
+                if (nv >= 32) {
 #pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    if (v0 + c0 + j < p.V) part[j & 3] += exp2f(fmaf(k, __uint_as_float(r[j]), -kb));
+                    for (int j = 0; j < 32; ++j) part[j & 3] += ex2(fmaf(k, __uint_as_float(r[j]), -kb));
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (j < nv) part[j & 3] += ex2(fmaf(k, __uint_as_float(r[j]), -kb));
+                }
                 esum += (part[0] + part[1]) + (part[2] + part[3]);
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
