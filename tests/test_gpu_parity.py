@@ -273,6 +273,47 @@ def test_dynamic_draft_exiting_against_oracle(small):
     assert rep.decisions > 0 and rep.decision_flips <= max(1, rep.decisions // 10)
 
 
+def test_draft_exiting_step_calls_equal_round_call(small):
+    """del_draft in exit mode runs the same confidence-checked loop as del_round."""
+    cfg, w, ctx = small
+    prompt = synth.make_prompt(cfg)
+    first = ctx.prefill(0, prompt, 24)
+    ctx.set_exit_mode(0, True)
+    a_tokens, E, trace = [first.tokens[0]], first.next_E, []
+    while len(a_tokens) < 24:
+        ctx.draft(0, E, cfg.g_max)
+        ctx.verify(0)
+        out = ctx.layer_accept(0)
+        E, _ = ctx.select(0)
+        a_tokens += out.emitted()
+        trace.append((out.E, out.g, out.stopped, out.n_accept, E))
+    first = ctx.prefill(0, prompt, 24)
+    ctx.set_exit_mode(0, True)
+    b_tokens, k = [first.tokens[0]], 0
+    while len(b_tokens) < 24:
+        out = ctx.round()[0]
+        b_tokens += out.emitted()
+        assert (out.E, out.g, out.stopped, out.n_accept, out.next_E) == trace[k], k
+        k += 1
+    assert a_tokens == b_tokens and len(a_tokens) == 24
+    assert any(t[2] for t in trace)                     # the break did fire
+    ctx.set_exit_mode(0, False)
+
+
+def test_batch_with_mixed_exit_modes():
+    """Three sequences share the layer passes; two of them draft with the confidence break, one does not."""
+    cfg = synth.small_variant(TINY_GQA, batch=3)
+    w = synth.make_weights(cfg)
+    ctx = make_ctx(cfg, w)
+    refs = [ref_from_oracle(cfg, w, synth.make_prompt(cfg, s), gen_len=24, exit_mode=(s != 1)) for s in range(3)]
+    reps = run_batch(ctx, refs, 24)
+    for s, rep in enumerate(reps):
+        print(f"seq {s} exit {refs[s].exit_mode}: rounds {rep.rounds} decisions {rep.decisions} flips {rep.flips} "
+              f"resyncs {rep.resyncs}")
+        assert rep.ok(), (s, rep.failures[:5])
+        assert rep.rounds == len(refs[s].rounds)
+
+
 def test_fs_baseline_policy_against_oracle(small):
     """Baseline FS(E-gamma) of Sec. 5.1 on the same kernels: fixed exit layer, gamma moved by +-1 on the device."""
     cfg, w, ctx = small
