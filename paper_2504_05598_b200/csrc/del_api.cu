@@ -145,7 +145,7 @@ size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max
     // chunk buffers of the bulk prefill (PF_ROWS prompt positions)
     PfArgs pfa;
     memset(&pfa, 0, sizeof(pfa));
-    pfa.n_ssp = (D.d + 255) / 256;
+    pfa.n_ssp = prefill_tc_ntiles(PF_DOWN, D);
     pfa.H = c.take<float>(base, (size_t)PF_ROWS * D.d);
     pfa.XS = c.take<bf16>(base, (size_t)PF_ROWS * D.d);
     pfa.SSP = c.take<float>(base, (size_t)PF_ROWS * pfa.n_ssp);
@@ -555,9 +555,10 @@ int draft_with_exit(del_ctx *c, std::vector<Job> &jobs) {
     return DEL_OK;
 }
 
-// ---- bulk of a prompt (positions 0 .. n_pos-1 of sequence sq) through the tensor-core GEMMs: only the KV
-// cache is produced; chunks of PF_ROWS positions, attention in passes of DEL_ROWS_MAX query rows
-int prefill_bulk(del_ctx *c, int sq, int n_pos) {
+// ---- a whole prompt (positions 0 .. n_pos-1 of sequence sq) through the tensor-core GEMMs: the KV cache of
+// every position, and every layer's hidden state of the positions from win0 on (the window that seeds the
+// statistics) into the hidden stack; chunks of PF_ROWS positions, attention in passes of DEL_ROWS_MAX query rows
+int prefill_bulk(del_ctx *c, int sq, int n_pos, int win0) {
     const Dims &D = c->D;
     const bool P = pdl(c);
     for (int p0 = 0; p0 < n_pos; p0 += PF_ROWS) {
@@ -565,6 +566,9 @@ int prefill_bulk(del_ctx *c, int sq, int n_pos) {
         a.M = std::min(PF_ROWS, n_pos - p0);
         a.seq = sq;
         a.pos0 = p0;
+        a.stackH = c->B.H;
+        a.win0 = win0;
+        const bool has_window = p0 + a.M > win0;      // then the last layer is needed in full
         cudaError_t e = launch_prefill_embed(a, c->tok_emb, c->B.PROMPT_ALL, c->attn_norm[0], c->st);
         if (e != cudaSuccess) return fail(c, e);
         ++c->launches;
@@ -573,7 +577,7 @@ int prefill_bulk(del_ctx *c, int sq, int n_pos) {
             a.K = D.d;
             a.n_ntiles = prefill_tc_ntiles(PF_QKV, D);
             LAUNCH(launch_prefill_gemm(PF_QKV, c->pf_xs.b, c->pf_wq[l - 1].b, c->pf_wk[l - 1].b, c->pf_wv[l - 1].b, a, c->n_sms, c->st, P));
-            if (l == D.L) break;             // the last layer's keys and values are all that is needed of it
+            if (l == D.L && !has_window) break;       // of the last layer only the keys and values are needed
             for (int r0 = 0; r0 < a.M; r0 += DEL_ROWS_MAX) {
                 AttnArgs at;
                 memset(&at, 0, sizeof(at));
@@ -601,7 +605,7 @@ int prefill_bulk(del_ctx *c, int sq, int n_pos) {
             LAUNCH(launch_prefill_gemm(PF_GATEUP, c->pf_xm.b, c->pf_wg[l - 1].b, c->pf_wu[l - 1].b, nullptr, a, c->n_sms, c->st, P));
             a.K = D.F;
             a.n_ntiles = prefill_tc_ntiles(PF_DOWN, D);
-            a.gain = c->attn_norm[l];        // the next layer's attention norm (l < L here)
+            a.gain = l < D.L ? c->attn_norm[l] : nullptr;      // the next layer's attention norm
             LAUNCH(launch_prefill_gemm(PF_DOWN, c->pf_act.b, c->pf_wd[l - 1].b, nullptr, nullptr, a, c->n_sms, c->st, P));
         }
     }
@@ -843,10 +847,10 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
         maps(c->pf_wq, c->wq, qd, d, 256);
         maps(c->pf_wk, c->wk, kvd, d, 256);
         maps(c->pf_wv, c->wv, kvd, d, 256);
-        maps(c->pf_wo, c->wo, d, qd, 256);
+        maps(c->pf_wo, c->wo, d, qd, 128);
         maps(c->pf_wg, c->w_gate, F, d, 128);
         maps(c->pf_wu, c->w_up, F, d, 128);
-        maps(c->pf_wd, c->w_down, d, F, 256);
+        maps(c->pf_wd, c->w_down, d, F, 128);
         c->pf_ok = ok;
         c->pf.D = c->D;
         c->pf.KP = c->B.KP; c->pf.VP = c->B.VP; c->pf.PT = c->B.PT;
@@ -894,14 +898,14 @@ int del_prefill(del_ctx *c, int sq, const int32_t *prompt, int n_prompt, int max
     // chunks of <= S positions; the last chunk is exactly the window so that its hidden states stay
     // in slots 0..W-1 of the stack
     std::vector<std::pair<int, int>> chunks;
-    int p_bulk = 0;                          // positions [0, p_bulk) go through the tensor-core prefill
+    // long prompts go through the tensor-core prefill as a whole; short ones through the decode kernels
     if (c->pf_ok && !(c->flags & FLAG_NO_BULK_PREFILL) && n_prompt - W >= 64) {
-        p_bulk = n_prompt - W;
-        rc = prefill_bulk(c, sq, p_bulk);
+        rc = prefill_bulk(c, sq, n_prompt, n_prompt - W);
         if (rc) return rc;
+    } else {
+        for (int p0 = 0; p0 < n_prompt - W; p0 += S) chunks.push_back({p0, std::min(S, n_prompt - W - p0)});
+        chunks.push_back({n_prompt - W, W});
     }
-    for (int p0 = p_bulk; p0 < n_prompt - W; p0 += S) chunks.push_back({p0, std::min(S, n_prompt - W - p0)});
-    chunks.push_back({n_prompt - W, W});
     s.T = 0;
     for (auto ch : chunks) {
         rc = plan_begin(c, 1);

@@ -92,7 +92,7 @@ struct PfArgs {
     int32_t layer, seq, pos0;  // 1-based layer; the rows are positions pos0 .. pos0 + M - 1 of sequence seq
     float *H;                  // [PF_ROWS][d] residual stream, updated in place
     bf16 *XS;                  // [PF_ROWS][d] bf16(h * attention-norm gain): input of QKV, written by DOWN
-    float *SSP;                // [PF_ROWS][n_ssp] sums of squares of h per output tile (QKV's 1/rms)
+    float *SSP;                // [PF_ROWS][n_ssp] sums of squares of h per output tile of DOWN (QKV's 1/rms)
     bf16 *Q, *ATT;             // [PF_ROWS][nh * hd]
     bf16 *XM;                  // [PF_ROWS][d] bf16(h_mid * ffn-norm gain), written by OPROJ
     float *SSPM;               // [PF_ROWS][n_ssp]
@@ -102,6 +102,10 @@ struct PfArgs {
     const int32_t *PT;
     const float *rope_cos, *rope_sin;
     int32_t *err;
+    // rows at positions >= win0 belong to the window that seeds the acceptance statistics: their hidden state
+    // after every layer is also stored in the hidden stack (slot = position - win0)
+    float *stackH;
+    int32_t win0;
 };
 int prefill_tc_ntiles(int epi, const Dims &D);
 cudaError_t launch_prefill_gemm(int epi, const void *map_a, const void *map_b0, const void *map_b1, const void *map_b2,

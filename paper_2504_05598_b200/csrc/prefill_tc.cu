@@ -8,11 +8,12 @@
 //   OPROJ   + residual (in place), ffn-norm input, per-tile sums of squares
 //   GATEUP  1/rms, SiLU(gate) * up -> activation buffer (the tile holds 128 gate and the same 128 up rows)
 //   DOWN    + residual (in place), next layer's attention-norm input, per-tile sums of squares
-// Only the KV cache of the prompt's bulk is needed later (the last window of positions goes through the
-// ordinary kernels, which also keep every layer's hidden states for the initialisation of the
-// acceptance statistics), so nothing else leaves these buffers.
+// Of most prompt positions only the KV cache is needed later.  The last window of positions also seeds
+// the acceptance statistics: the hidden state of those rows after every layer (and their embedding) is
+// copied into the hidden stack, where the stacked LM head finds it.
 //
-// CTA tile 128 rows x 256 output features, K blocks of 64 (one 128-byte swizzle span), same roles as
+// CTA tile 128 rows x 256 output features (128 for the two d-wide projections, whose 256-wide tiles would
+// fill less than half of the SMs), K blocks of 64 (one 128-byte swizzle span), same roles as
 // the stacked LM head: warp 0 issues TMA loads into a 4-stage shared-memory ring, warp 1 issues
 // tcgen05.mma into one of two 256-column accumulators in tensor memory, warps 2-5 read their own row
 // with tcgen05.ld and run the epilogue while the next tile's MMAs proceed.  Ragged shapes (rows, N, K)
@@ -29,6 +30,8 @@ using namespace tc;
 constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int PF_THREADS = 192;
+constexpr int BN_NARROW = 128;     // tile width of O-proj and down (N = d_model)
+template <int EPI> __host__ __device__ constexpr int tile_n() { return (EPI == PF_OPROJ || EPI == PF_DOWN) ? BN_NARROW : BN; }
 
 struct PfMaps {
     CUtensorMap a;             // activations [PF_ROWS, K], box 64 x 128
@@ -136,11 +139,11 @@ __device__ __forceinline__ void epilogue(const PfArgs &p, uint32_t taddr, int ro
     } else {   // PF_OPROJ, PF_DOWN: residual update in place, next norm input, sums of squares of the new h
         float ss = 0.f;
         bf16 *xo = EPI == PF_OPROJ ? p.XM : p.XS;
-        for (int c0 = 0; c0 < BN; c0 += 32) {
+        for (int c0 = 0; c0 < BN_NARROW; c0 += 32) {
             __syncwarp();
             tmem_ld32(taddr + (uint32_t)c0, r0);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            const int n = nt * BN + c0;
+            const int n = nt * BN_NARROW + c0;
             if (!live || n >= D.d) continue;                     // d is a multiple of 32
             float *hp = p.H + (size_t)row * D.d + n;
             float h[32];
@@ -152,6 +155,12 @@ __device__ __forceinline__ void epilogue(const PfArgs &p, uint32_t taddr, int ro
                 h[4 * q + 2] = v.z + __uint_as_float(r0[4 * q + 2]);
                 h[4 * q + 3] = v.w + __uint_as_float(r0[4 * q + 3]);
                 *reinterpret_cast<float4 *>(hp + 4 * q) = make_float4(h[4 * q], h[4 * q + 1], h[4 * q + 2], h[4 * q + 3]);
+            }
+            if (EPI == PF_DOWN && p.pos0 + row >= p.win0) {
+                float *sp = p.stackH + stack_row(D, p.layer, p.seq, p.pos0 + row - p.win0) * D.d + n;
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    *reinterpret_cast<float4 *>(sp + 4 * q) = make_float4(h[4 * q], h[4 * q + 1], h[4 * q + 2], h[4 * q + 3]);
             }
             float x[32];
 #pragma unroll
@@ -208,7 +217,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1) prefill_gemm_kernel(const __gri
                 for (int kb = 0; kb < n_kb; ++kb, ++it) {
                     const int s = it % STAGES;
                     if (!mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1)) { s_err = 1; break; }
-                    mbar_expect_tx(&full_bar[s], STAGE_BYTES);
+                    mbar_expect_tx(&full_bar[s], A_BYTES + tile_n<EPI>() * BK * 2);
                     unsigned char *sa = tiles + (size_t)s * STAGE_BYTES;
                     tma_load_2d(sa, &maps.a, kb * BK, mt * BM, &full_bar[s]);
                     if (EPI == PF_QKV) {
@@ -220,15 +229,16 @@ __global__ void __launch_bounds__(PF_THREADS, 1) prefill_gemm_kernel(const __gri
                         tma_load_2d(sa + A_BYTES, &maps.b0, kb * BK, nt * (BN / 2), &full_bar[s]);
                         tma_load_2d(sa + A_BYTES + B_BYTES / 2, &maps.b1, kb * BK, nt * (BN / 2), &full_bar[s]);
                     } else {
-                        tma_load_2d(sa + A_BYTES, &maps.b0, kb * BK, nt * BN, &full_bar[s]);
+                        tma_load_2d(sa + A_BYTES, &maps.b0, kb * BK, nt * tile_n<EPI>(), &full_bar[s]);
                     }
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, N = 256, M = 128
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, N = tile width, M = 128
+            const uint32_t idesc =
+                (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(tile_n<EPI>() >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
             int it = 0;
             for (int i = 0; i < my_tiles && !s_err; ++i) {
                 const int buf = i & 1;
@@ -281,10 +291,12 @@ __global__ void __launch_bounds__(256) prefill_embed_kernel(const PfArgs p, cons
     pdl_wait();
     const int row = blockIdx.x, d = p.D.d;
     const bf16 *e = tok_emb + (size_t)prompt[p.pos0 + row] * d;
+    float *sp = p.pos0 + row >= p.win0 ? p.stackH + stack_row(p.D, 0, p.seq, p.pos0 + row - p.win0) * d : nullptr;
     float ss = 0.f;
     for (int o = threadIdx.x; o < d; o += 256) {
         const float h = bf16_to_f(e[o]);
         p.H[(size_t)row * d + o] = h;
+        if (sp) sp[o] = h;
         p.XS[(size_t)row * d + o] = __float2bfloat16_rn(h * bf16_to_f(gain0[o]));
         ss += h * h;
     }
@@ -329,11 +341,12 @@ int prefill_tc_ntiles(int epi, const Dims &D) {
     switch (epi) {
         case PF_QKV: return (D.nh * D.hd + BN - 1) / BN + 2 * ((D.nkv * D.hd + BN - 1) / BN);
         case PF_GATEUP: return (D.F + BN / 2 - 1) / (BN / 2);
-        default: return (D.d + BN - 1) / BN;
+        default: return (D.d + BN_NARROW - 1) / BN_NARROW;
     }
 }
 
-// map_a / map_b*: 128-byte CUtensorMap blobs made by lmhead_tc_make_map (weights: box of 256 rows, gate / up: 128)
+// map_a / map_b*: 128-byte CUtensorMap blobs made by lmhead_tc_make_map (boxes of 256 rows for Wq / Wk / Wv, of
+// 128 rows for the activations and for W_gate / W_up / W_o / W_down)
 cudaError_t launch_prefill_gemm(int epi, const void *map_a, const void *map_b0, const void *map_b1, const void *map_b2,
                                 const PfArgs &p, int n_sms, cudaStream_t st, bool pdl) {
     PfMaps maps;
