@@ -10,4 +10,7 @@ TINY_GQA = synth.small_variant(TINY, name="tiny_gqa", n_layers=6, n_kv_heads=2, 
 # long prompts: the bulk of the prompt goes through the tensor-core prefill (ragged last row tile)
 TINY_LONG = synth.small_variant(TINY, name="tiny_long", prompt_len=300, gen_len=24, emb_scale=10.0, seed=11)
 TINY_GQA_LONG = synth.small_variant(TINY_GQA, name="tiny_gqa_long", prompt_len=200, gen_len=24, seed=78)
+# two prefill passes of 512 positions; in the second variant the 32-position window straddles the pass boundary
+TINY_LONG2 = synth.small_variant(TINY, name="tiny_long2", prompt_len=600, gen_len=16, emb_scale=10.0, seed=12)
+TINY_LONG3 = synth.small_variant(TINY_GQA, name="tiny_gqa_long3", prompt_len=530, gen_len=16, seed=79)
 TINY_SHORT = synth.small_variant(TINY, name="tiny_short", prompt_len=7, gen_len=21, emb_scale=10.0, seed=5)

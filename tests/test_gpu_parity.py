@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 
 import synth
-from cases import TINY, TINY_GQA, TINY_GQA_LONG, TINY_LONG, TINY_SHORT
+from cases import TINY, TINY_GQA, TINY_GQA_LONG, TINY_LONG, TINY_LONG2, TINY_LONG3, TINY_SHORT
 from parity import MARGIN, ref_from_golden, ref_from_oracle, run_batch, run_sequence
 
 pytestmark = pytest.mark.gpu
@@ -57,7 +57,7 @@ def test_prefill_hidden_kv_and_logits(small):
             assert int(np.argmax(got)) == int(np.argmax(ref))
 
 
-@pytest.mark.parametrize("cfg", [TINY_LONG, TINY_GQA_LONG], ids=lambda c: c.name)
+@pytest.mark.parametrize("cfg", [TINY_LONG, TINY_GQA_LONG, TINY_LONG2, TINY_LONG3], ids=lambda c: c.name)
 def test_tensor_core_prefill_against_oracle(cfg):
     """Prompts longer than the initialisation window: their bulk is prefilled by the tcgen05 GEMMs (only the KV
     cache comes out of it).  Cached K/V of bulk positions in every layer, the window's hidden states (which
@@ -77,7 +77,7 @@ def test_tensor_core_prefill_against_oracle(cfg):
         ctx.prefill(0, prompt, cfg.gen_len)
         n_launch = ctx.launch_count() - launches0
         for l in range(1, cfg.n_layers + 1):
-            for pos in (0, 1, 15, 16, 127, 128, P - W - 1, P - W, P - 1):
+            for pos in sorted({0, 1, 15, 16, 127, 128, min(511, P - 1), min(512, P - 1), P - W - 1, P - W, P - 1}):
                 k, v = ctx.get_kv(0, l, pos)
                 kr, vr = o.k_row(l, pos), o.v_row(l, pos)
                 assert np.abs(k - kr).max() <= 2e-2 * np.abs(kr).max() + 1e-6, ("k", flags, l, pos)
