@@ -30,6 +30,14 @@ struct AttnView {
 
 namespace attn {
 
+// head-major row index -> (query head within the group, row of the segment); ms = rows of the segment.
+// One-row segments (plain drafting, the common case on the critical path) skip the integer division.
+__device__ __forceinline__ void split_row(int rr, int ms, int &hq, int &i) {
+    if (ms == 1) { hq = rr; i = 0; return; }
+    hq = rr / ms;
+    i = rr - hq * ms;
+}
+
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr int NW = 8;                 // warps per CTA
 constexpr int PG = 4;                 // page ids fetched ahead per warp
@@ -62,8 +70,8 @@ __device__ __forceinline__ void tile_begin(TileState<HD> &ts, const AttnView &a,
     for (int h = 0; h < 2; ++h) {
         const int rr = mt * 16 + g + 8 * h;
         ts.rv[h] = mt < n_mt && rr < R;
-        const int rh = ts.rv[h] ? rr / ms : 0;
-        const int ri = ts.rv[h] ? rr - rh * ms : 0;
+        int rh = 0, ri = 0;
+        if (ts.rv[h]) split_row(rr, ms, rh, ri);
         const bf16 *qp = a.B.Q + (size_t)(seg.row0 + ri) * qdim + (kvh * group + rh) * HD + 8 * t;
 #pragma unroll
         for (int ks = 0; ks < TileState<HD>::KS; ++ks) ts.qf[h][ks] = ldg_act16_pred(qp + 32 * ks, ts.rv[h]);
@@ -169,7 +177,8 @@ __device__ __forceinline__ void tile_end(TileState<HD> &ts, const AttnView &a, f
         for (int h = 0; h < 2; ++h) {
             const int r2 = mt2 * 16 + g + 8 * h;
             if (r2 >= R) continue;
-            const int hq = r2 / ms, i = r2 - hq * ms;
+            int hq, i;
+            split_row(r2, ms, hq, i);
             const int c = seg.row0 + i, qh = kvh * group + hq;
             if (n_slots == 1) {
                 const float inv = 1.f / Lv[h];
@@ -349,43 +358,69 @@ __device__ __forceinline__ void partial_staged(const AttnView &a, unsigned char 
 
 // Combines slots 0..n_slots-1 of every (row, head) of a (segment, kv head) in slot order and writes the
 // normalised bf16 result.  The caller has made the slots visible (fence + barrier / arrival counter).
+// NS = compile-time bound on the slots, UE = elements a thread works on at once: the loads of an iteration
+// (UE * NS partial states) are all in flight together.
+template <int HD, int NS, int UE>
+__device__ __forceinline__ void merge_slots_n(const AttnView &a, const Segment seg, int kvh, int n_slots) {
+    const int ms = seg.nrows, group = a.D.nh / a.D.nkv, R = ms * group, qdim = a.D.nh * HD;
+    const int n_el = R * (HD / 4);
+    for (int e0 = threadIdx.x; e0 < n_el; e0 += NW * 32 * UE) {
+        uint2 mlv[UE][NS];
+        uint4 ovv[UE][NS];
+        size_t out_off[UE];
+        bool live[UE];
+        // all loads first, then the arithmetic: two memory latencies per iteration in total
+#pragma unroll
+        for (int u = 0; u < UE; ++u) {
+            const int e = e0 + u * NW * 32;
+            live[u] = e < n_el;
+            const int ee = live[u] ? e : 0;
+            const int row = ee / (HD / 4), d4 = (ee - row * (HD / 4)) * 4;
+            int hq, i;
+            split_row(row, ms, hq, i);
+            const int c = seg.row0 + i, qh = kvh * group + hq;
+            const size_t pi = ((size_t)c * a.D.nh + qh) * n_slots;
+            out_off[u] = (size_t)c * qdim + qh * HD + d4;
+#pragma unroll
+            for (int s = 0; s < NS; ++s) {
+                const int se = s < n_slots ? s : n_slots - 1;       // clamped: unused slots are masked below
+                mlv[u][s] = ldg_act8(a.B.APML + (pi + se) * 2);
+                ovv[u][s] = ldg_act16(a.B.APO + (pi + se) * HD + d4);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UE; ++u) {
+            float M = -INFINITY;
+#pragma unroll
+            for (int s = 0; s < NS; ++s) {
+                if (s >= n_slots) mlv[u][s].x = 0xff800000u;        // -inf: weight 0
+                M = fmaxf(M, __uint_as_float(mlv[u][s].x));
+            }
+            float l = 0.f, o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;
+#pragma unroll
+            for (int s = 0; s < NS; ++s) {
+                const float f = exp2f(__uint_as_float(mlv[u][s].x) - M);
+                l += f * __uint_as_float(mlv[u][s].y);
+                o0 += f * __uint_as_float(ovv[u][s].x); o1 += f * __uint_as_float(ovv[u][s].y);
+                o2 += f * __uint_as_float(ovv[u][s].z); o3 += f * __uint_as_float(ovv[u][s].w);
+            }
+            const float inv = 1.f / l;
+            uint2 pk;
+            pk.x = pack_bf16(o0 * inv, o1 * inv);
+            pk.y = pack_bf16(o2 * inv, o3 * inv);
+            if (live[u]) *reinterpret_cast<uint2 *>(a.B.ATT + out_off[u]) = pk;
+        }
+    }
+}
+
 template <int HD>
 __device__ __forceinline__ void merge_slots(const AttnView &a, const Segment seg, int kvh, int n_slots) {
-    const int ms = seg.nrows, group = a.D.nh / a.D.nkv, R = ms * group, qdim = a.D.nh * HD;
-    for (int e = threadIdx.x; e < R * (HD / 4); e += NW * 32) {
-        const int row = e / (HD / 4), d4 = (e - row * (HD / 4)) * 4;
-        const int hq = row / ms, i = row - hq * ms;
-        const int c = seg.row0 + i, qh = kvh * group + hq;
-        const size_t pi = ((size_t)c * a.D.nh + qh) * n_slots;
-        // all loads first, then the arithmetic: two memory latencies in total
-        uint2 mlv[MAX_SLOTS];
-        uint4 ovv[MAX_SLOTS];
-#pragma unroll
-        for (int s = 0; s < MAX_SLOTS; ++s) {
-            const int se = s < n_slots ? s : n_slots - 1;           // clamped: unused slots are masked below
-            mlv[s] = ldg_act8(a.B.APML + (pi + se) * 2);
-            ovv[s] = ldg_act16(a.B.APO + (pi + se) * HD + d4);
-        }
-        float M = -INFINITY;
-#pragma unroll
-        for (int s = 0; s < MAX_SLOTS; ++s) {
-            if (s >= n_slots) mlv[s].x = 0xff800000u;               // -inf: weight 0
-            M = fmaxf(M, __uint_as_float(mlv[s].x));
-        }
-        float l = 0.f, o0 = 0.f, o1 = 0.f, o2 = 0.f, o3 = 0.f;
-#pragma unroll
-        for (int s = 0; s < MAX_SLOTS; ++s) {
-            const float f = exp2f(__uint_as_float(mlv[s].x) - M);
-            l += f * __uint_as_float(mlv[s].y);
-            o0 += f * __uint_as_float(ovv[s].x); o1 += f * __uint_as_float(ovv[s].y);
-            o2 += f * __uint_as_float(ovv[s].z); o3 += f * __uint_as_float(ovv[s].w);
-        }
-        const float inv = 1.f / l;
-        uint2 pk;
-        pk.x = pack_bf16(o0 * inv, o1 * inv);
-        pk.y = pack_bf16(o2 * inv, o3 * inv);
-        *reinterpret_cast<uint2 *>(a.B.ATT + (size_t)c * qdim + qh * HD + d4) = pk;
-    }
+    // a decode-sized segment has at most one element per thread: the plain form has the least index arithmetic
+    // in front of its loads; large segments (prefill passes) batch several elements per thread
+    const int n_el = seg.nrows * (a.D.nh / a.D.nkv) * (HD / 4);
+    if (n_el <= NW * 32 || n_slots > 8) merge_slots_n<HD, 16, 1>(a, seg, kvh, n_slots);
+    else if (n_slots <= 4) merge_slots_n<HD, 4, 4>(a, seg, kvh, n_slots);
+    else merge_slots_n<HD, 8, 2>(a, seg, kvh, n_slots);
 }
 
 }  // namespace attn
