@@ -130,9 +130,11 @@ int del_init(del_ctx **ctx, const del_shape *shape, const del_weights *weights, 
 int del_prefill(del_ctx *ctx, int seq, const int32_t *prompt, int n_prompt, int max_new_tokens,
                 del_round_out *first_out);
 
-/* Draft phase (Sec. 2 early-exit drafting; Algorithm 1 draft loop without the break): gamma tokens,
- * each through embedding, layers 1..E, shared final RMSNorm, LM head, argmax.  gamma is clipped like
- * in del_round.  Async.  Errors: DEL_EINVAL (E outside [1, n_layers-1], gamma outside [0, g_max]),
+/* Draft phase (Sec. 2 early-exit drafting; Algorithm 1 draft loop): gamma tokens, each through embedding,
+ * layers 1..E, shared final RMSNorm, LM head, argmax.  gamma is clipped like in del_round.  Async, except
+ * for a sequence in exit mode (del_set_exit_mode): then gamma is the most the loop may draft, the host reads
+ * each token's confidence (one synchronisation per token) and the loop ends at the first one below the
+ * threshold.  Errors: DEL_EINVAL (E outside [1, n_layers-1], gamma outside [0, g_max]),
  * DEL_ESTATE (no prefill, sequence finished, previous round not completed), DEL_ENOSPC. */
 int del_draft(del_ctx *ctx, int seq, int E, int gamma);
 

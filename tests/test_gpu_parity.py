@@ -171,6 +171,17 @@ def test_error_codes(small):
     assert lib.del_draft(h, 0, 1, 1) == dl.ESTATE                      # round in progress
     ctx.verify(0)
     ctx.layer_accept(0)
+    # policy / mode calls
+    L = cfg.n_layers
+    assert lib.del_set_policy(h, 0, L, 1) == dl.EINVAL                 # E must be < n_layers
+    assert lib.del_set_policy_fs(h, 0, 1, 0) == dl.EINVAL              # the controller needs gamma0 >= 1
+    assert lib.del_set_policy_fs(h, 0, 0, 2) == dl.EINVAL              # ... and a fixed exit layer
+    assert lib.del_set_policy_fs(h, 0, 1, cfg.g_max + 1) == dl.EINVAL
+    assert lib.del_set_exit_mode(h, 99, 1) == dl.EINVAL
+    assert lib.del_get_conf_stats(h, 99, None, None, None) == dl.EINVAL
+    assert lib.del_set_conf_stats(h, 0, None, None) == dl.EINVAL
+    assert lib.del_get_conf(h, 99, None, None) == dl.EINVAL
+    assert lib.del_get_conf(h, 0, None, None) == dl.OK                 # both outputs are optional
     # the context is still healthy
     assert ctx.round()[0].n_emitted >= 1
 
