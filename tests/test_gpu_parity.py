@@ -92,6 +92,33 @@ def test_tensor_core_prefill_against_oracle(cfg):
     o.close()
 
 
+@pytest.mark.parametrize("prompt_len", [1, 2, 95, 96, 97])
+def test_prompt_length_edges(prompt_len):
+    """One-token prompt (window of one position), and the lengths around the switch to the tensor-core
+    prefill (64 positions before the 32-position window)."""
+    import oracle
+    cfg = synth.small_variant(TINY, name=f"tiny_p{prompt_len}", prompt_len=prompt_len, gen_len=12, emb_scale=10.0,
+                              seed=300 + prompt_len)
+    w = synth.make_weights(cfg)
+    ctx = make_ctx(cfg, w)
+    prompt = synth.make_prompt(cfg)
+    o = oracle.OracleSeq(cfg, w)
+    o.prefill(prompt)
+    ctx.prefill(0, prompt, cfg.gen_len)
+    for l in (1, cfg.n_layers):
+        for pos in sorted({0, prompt_len // 2, prompt_len - 1}):
+            k, v = ctx.get_kv(0, l, pos)
+            kr, vr = o.k_row(l, pos), o.v_row(l, pos)
+            assert np.abs(k - kr).max() <= 2e-2 * np.abs(kr).max() + 1e-6, ("k", l, pos)
+            assert np.abs(v - vr).max() <= 2e-2 * np.abs(vr).max() + 1e-6, ("v", l, pos)
+    o.close()
+    ref = ref_from_oracle(cfg, w, prompt)
+    rep = run_sequence(ctx, 0, ref, cfg.gen_len)
+    assert rep.ok(), rep.failures[:5]
+    assert rep.rounds == len(ref.rounds)
+    ctx.close()
+
+
 def test_dynamic_rounds_match_oracle(small):
     cfg, w, ctx = small
     ref = ref_from_oracle(cfg, w, synth.make_prompt(cfg))
