@@ -119,6 +119,22 @@ def test_prompt_length_edges(prompt_len):
     ctx.close()
 
 
+def test_largest_speculation_length():
+    """g_max = 31 (the largest the library accepts): 32-row verify passes and a 32-row draft/verify history."""
+    cfg = synth.small_variant(TINY_GQA, name="tiny_gqa_g31", g_max=31, gen_len=80, seed=91)
+    w = synth.make_weights(cfg)
+    ctx = make_ctx(cfg, w)
+    prompt = synth.make_prompt(cfg)
+    for policy in ((2, 31), None):
+        ref = ref_from_oracle(cfg, w, prompt, policy=policy)
+        rep = run_sequence(ctx, 0, ref, cfg.gen_len, policy=policy)
+        print(f"{cfg.name} policy {policy}: rounds {rep.rounds} compared {rep.compared} flips {rep.flips}")
+        assert rep.ok(), rep.failures[:5]
+        assert rep.rounds == len(ref.rounds)
+    assert max(r.g for r in ref_from_oracle(cfg, w, prompt, policy=(2, 31)).rounds) == 31
+    ctx.close()
+
+
 def test_dynamic_rounds_match_oracle(small):
     cfg, w, ctx = small
     ref = ref_from_oracle(cfg, w, synth.make_prompt(cfg))
