@@ -229,6 +229,31 @@ def test_error_codes(small):
     assert ctx.round()[0].n_emitted >= 1
 
 
+def test_kv_pages_run_out_and_come_back():
+    """Two sequences share a page pool that holds one and a half of them: the second prefill is refused with
+    DEL_ENOSPC, the first sequence keeps decoding correctly, and after its release the second one fits."""
+    import paper_2504_05598_b200 as dl
+    cfg = synth.small_variant(TINY, batch=2, gen_len=16)
+    w = synth.make_weights(cfg)
+    # pages are handed out as positions are reached: sequence 0 holds 3 of the 7 pages after two rounds, the
+    # long prompt below needs 5 for its prefill
+    ctx = dl.DelContext(dl.make_shape(cfg, max_seq=160, n_pages=7), dl.upload_weights(w))
+    ref = ref_from_oracle(cfg, w, synth.make_prompt(cfg, 0))
+    p1 = np.ascontiguousarray(synth.make_prompt(cfg, 1), dtype=np.int32)
+    ctx.prefill(0, ref.prompt, cfg.gen_len)
+    ctx.round()
+    ctx.round()                                                                # sequence 0 now holds most of its pages
+    big = np.ascontiguousarray(np.tile(p1, 3)[:cfg.prompt_len * 2 + 8], dtype=np.int32)
+    rc = ctx.lib.del_prefill(ctx._h, 1, big.ctypes.data, len(big), 8, None)
+    assert rc == dl.ENOSPC
+    rep = run_sequence(ctx, 0, ref, cfg.gen_len)                               # sequence 0 is unharmed
+    assert rep.ok(), rep.failures[:5]
+    ctx.release(0)
+    assert ctx.lib.del_prefill(ctx._h, 1, big.ctypes.data, len(big), 8, None) == dl.OK
+    assert ctx.round()[1].n_emitted >= 1
+    ctx.close()
+
+
 def test_generation_stops_at_budget(small):
     cfg, w, ctx = small
     import paper_2504_05598_b200 as dl
