@@ -144,6 +144,49 @@ __device__ __forceinline__ void tile_end(TileState<HD> &ts, const AttnView &a, f
         ts.l_run[h] += __shfl_xor_sync(0xffffffffu, ts.l_run[h], 1);
         ts.l_run[h] += __shfl_xor_sync(0xffffffffu, ts.l_run[h], 2);
     }
+    if (R <= 8) {
+        // Few query rows (one sequence drafting or verifying a handful of tokens): only rows 0..R-1 of the tile
+        // carry data, i.e. MMA rows g < R and none of the rows g + 8.  Merge just those: [warp][row][HD] floats.
+        float *so = sm;                             // [NW][R][HD]
+        float *sml = sm + NW * 8 * HD;              // [NW][8] (max, sum)
+        if (g < R) {
+            float *dst = so + ((size_t)warp * R + g) * HD + 2 * t;
+#pragma unroll
+            for (int j = 0; j < NJ; ++j) *reinterpret_cast<float2 *>(dst + 8 * j) = make_float2(ts.O[j][0], ts.O[j][1]);
+            if (t == 0) *reinterpret_cast<float2 *>(sml + (warp * 8 + g) * 2) = make_float2(ts.m_run[0], ts.l_run[0]);
+        }
+        __syncthreads();
+        for (int e = tid; e < R * (HD / 2); e += NW * 32) {
+            const int row = e / (HD / 2), col = (e - row * (HD / 2)) * 2;
+            float M = -INFINITY;
+#pragma unroll
+            for (int w2 = 0; w2 < NW; ++w2) M = fmaxf(M, sml[(w2 * 8 + row) * 2]);
+            const float b = M == -INFINITY ? 0.f : M;
+            float L = 0.f, o0 = 0.f, o1 = 0.f;
+#pragma unroll
+            for (int w2 = 0; w2 < NW; ++w2) {
+                const float2 ml = *reinterpret_cast<const float2 *>(sml + (w2 * 8 + row) * 2);
+                const float f = exp2f(ml.x - b);
+                const float2 ov = *reinterpret_cast<const float2 *>(so + ((size_t)w2 * R + row) * HD + col);
+                L += ml.y * f;
+                o0 += ov.x * f;
+                o1 += ov.y * f;
+            }
+            int hq, i;
+            split_row(row, ms, hq, i);
+            const int c = seg.row0 + i, qh = kvh * group + hq;
+            if (n_slots == 1) {
+                const float inv = 1.f / L;
+                *reinterpret_cast<uint32_t *>(a.B.ATT + (size_t)c * qdim + qh * HD + col) = pack_bf16(o0 * inv, o1 * inv);
+            } else {
+                const size_t pi = ((size_t)c * a.D.nh + qh) * n_slots + slot;
+                *reinterpret_cast<float2 *>(a.B.APO + pi * HD + col) = make_float2(o0, o1);
+                if (col == 0) *reinterpret_cast<float2 *>(a.B.APML + pi * 2) = make_float2(M, L);
+            }
+        }
+        __syncthreads();
+        return;
+    }
     // layout [column tile][warp][lane]: consecutive lanes write consecutive 16-byte words
 #pragma unroll
     for (int j = 0; j < NJ; ++j)
