@@ -168,10 +168,20 @@ __global__ void __launch_bounds__(CTL_THREADS) prep_rows_kernel(const CtlArgs a,
     const float *h = a.B.H + stack_row(a.D, layer, seq, slot) * d;
     bf16 *x = a.B.XN + (size_t)blockIdx.x * d;
     float sq = 0.f;
-    for (int o = threadIdx.x; o < d; o += CTL_THREADS) {
-        const float hv = ldg_cg_f32(h + o);
-        x[o] = __float2bfloat16_rn(hv * bf16_to_f(a.final_gain[o]));
-        sq += hv * hv;
+    // 8 consecutive features per thread and step (d is a multiple of 32): two 16-byte loads of h, one of the gains
+    for (int o = threadIdx.x * 8; o < d; o += CTL_THREADS * 8) {
+        const uint4 h0 = ldg_act16(h + o), h1 = ldg_act16(h + o + 4);
+        const uint4 gv = ldg_stream16_pred(a.final_gain + o, true);
+        const float hv[8] = {__uint_as_float(h0.x), __uint_as_float(h0.y), __uint_as_float(h0.z), __uint_as_float(h0.w),
+                             __uint_as_float(h1.x), __uint_as_float(h1.y), __uint_as_float(h1.z), __uint_as_float(h1.w)};
+        const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w};
+        uint32_t xo[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            xo[q] = pack_bf16(hv[2 * q] * __uint_as_float(gw[q] << 16), hv[2 * q + 1] * __uint_as_float(gw[q] & 0xffff0000u));
+            sq += hv[2 * q] * hv[2 * q] + hv[2 * q + 1] * hv[2 * q + 1];
+        }
+        *reinterpret_cast<uint4 *>(x + o) = make_uint4(xo[0], xo[1], xo[2], xo[3]);
     }
     const float total = block_sum(sq);
     if (threadIdx.x == 0) a.B.RS[blockIdx.x] = rsqrtf(total / (float)d + a.D.eps) * 1.4426950408889634f;
