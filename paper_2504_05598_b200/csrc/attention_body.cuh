@@ -458,10 +458,16 @@ __device__ __forceinline__ void merge_slots_n(const AttnView &a, const Segment s
 
 template <int HD>
 __device__ __forceinline__ void merge_slots(const AttnView &a, const Segment seg, int kvh, int n_slots) {
-    // a decode-sized segment has at most one element per thread: the plain form has the least index arithmetic
-    // in front of its loads; large segments (prefill passes) batch several elements per thread
+    // a decode-sized segment has at most one element per thread: one element per thread (least index arithmetic in
+    // front of the loads) and no more loads than the split count needs (1 % of a round against always loading
+    // 16 clamped slots); large segments (prefill passes) batch several elements per thread
     const int n_el = seg.nrows * (a.D.nh / a.D.nkv) * (HD / 4);
-    if (n_el <= NW * 32 || n_slots > 8) merge_slots_n<HD, 16, 1>(a, seg, kvh, n_slots);
+    if (n_el <= NW * 32) {
+        if (n_slots <= 2) merge_slots_n<HD, 2, 1>(a, seg, kvh, n_slots);
+        else if (n_slots <= 4) merge_slots_n<HD, 4, 1>(a, seg, kvh, n_slots);
+        else if (n_slots <= 8) merge_slots_n<HD, 8, 1>(a, seg, kvh, n_slots);
+        else merge_slots_n<HD, 16, 1>(a, seg, kvh, n_slots);
+    } else if (n_slots > 8) merge_slots_n<HD, 16, 1>(a, seg, kvh, n_slots);
     else if (n_slots <= 4) merge_slots_n<HD, 4, 4>(a, seg, kvh, n_slots);
     else merge_slots_n<HD, 8, 2>(a, seg, kvh, n_slots);
 }
