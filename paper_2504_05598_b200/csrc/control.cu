@@ -159,7 +159,8 @@ __device__ __forceinline__ bool locate_row(const UpdatePlan *up, int L, int mode
 // Stacked LM head input: row (seq, layer, slot) of the hidden stack times the final norm's gain, as
 // bf16.  The norm's 1/rms is a positive per-row scalar and cannot change the arg-max, so it is left out
 // of the product; it is stored (times log2 e) for the confidence score, which does depend on it.
-__global__ void __launch_bounds__(CTL_THREADS) prep_rows_kernel(const CtlArgs a, const UpdatePlan *up) {
+__global__ void __launch_bounds__(CTL_THREADS) prep_rows_kernel(const CtlArgs a, const __grid_constant__ UpdatePlan up_v) {
+    const UpdatePlan *up = &up_v;
     pdl_launch();
     pdl_wait();
     int seq, layer, slot;
@@ -188,9 +189,10 @@ __global__ void __launch_bounds__(CTL_THREADS) prep_rows_kernel(const CtlArgs a,
 }
 
 // Reduce the vocabulary-tile partials of one stacked row into its shadow token.
-__global__ void __launch_bounds__(CTL_THREADS) shadow_reduce_kernel(const CtlArgs a, const UpdatePlan *up, const float *pv,
+__global__ void __launch_bounds__(CTL_THREADS) shadow_reduce_kernel(const CtlArgs a, const __grid_constant__ UpdatePlan up_v, const float *pv,
                                                                     const int32_t *pi, const float *ps, int n_part, int pstride,
                                                                     int cstride, int row_base) {
+    const UpdatePlan *up = &up_v;
     pdl_launch();
     pdl_wait();
     const int c = blockIdx.x;
@@ -225,7 +227,8 @@ __global__ void refresh_tau_kernel(const CtlArgs a, int seq) {
 
 // Prefix acceptance, per-layer match counts over the valid context and decayed statistics
 // (S <- omega * S + a, no fused multiply-add so that the host oracle's doubles are reproduced).
-__global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const UpdatePlan *up, del_round_out *out) {
+__global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const __grid_constant__ UpdatePlan up_v, del_round_out *out) {
+    const UpdatePlan *up = &up_v;
     __shared__ int s_n;
     pdl_launch();
     pdl_wait();
@@ -297,7 +300,8 @@ __global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const Upda
 }
 
 // (E, gamma) = argmax of (sum_{k<=gamma} alpha_E^k) / (gamma*E + L), first maximum in E-major order.
-__global__ void __launch_bounds__(64) select_kernel(const CtlArgs a, const UpdatePlan *up, del_round_out *out) {
+__global__ void __launch_bounds__(64) select_kernel(const CtlArgs a, const __grid_constant__ UpdatePlan up_v, del_round_out *out) {
+    const UpdatePlan *up = &up_v;
     __shared__ double s_best[64];
     __shared__ int s_g[64];
     pdl_launch();
@@ -417,20 +421,20 @@ cudaError_t launch_draft_finalize_embed(const CtlArgs &a, int m, bool embed_next
     return launch(draft_finalize_embed_kernel, m, CTL_THREADS, st, pdl, a, (int)embed_next);
 }
 cudaError_t launch_prep_rows(const CtlArgs &a, const UpdatePlan *up, int n_rows, cudaStream_t st, bool pdl) {
-    return launch(prep_rows_kernel, n_rows, CTL_THREADS, st, pdl, a, up);
+    return launch(prep_rows_kernel, n_rows, CTL_THREADS, st, pdl, a, *up);
 }
 cudaError_t launch_shadow_reduce(const CtlArgs &a, const UpdatePlan *up, const float *pv, const int32_t *pi, const float *ps,
                                  int n_part, int pstride, int cstride, int row_base, int n_rows, cudaStream_t st, bool pdl) {
-    return launch(shadow_reduce_kernel, n_rows, CTL_THREADS, st, pdl, a, up, pv, pi, ps, n_part, pstride, cstride, row_base);
+    return launch(shadow_reduce_kernel, n_rows, CTL_THREADS, st, pdl, a, *up, pv, pi, ps, n_part, pstride, cstride, row_base);
 }
 cudaError_t launch_refresh_tau(const CtlArgs &a, int seq, cudaStream_t st) {
     return launch(refresh_tau_kernel, 1, 128, st, false, a, seq);
 }
 cudaError_t launch_update(const CtlArgs &a, const UpdatePlan *up, void *out_dev, int n_seq, cudaStream_t st, bool pdl) {
-    return launch(update_kernel, n_seq, 128, st, pdl, a, up, (del_round_out *)out_dev);
+    return launch(update_kernel, n_seq, 128, st, pdl, a, *up, (del_round_out *)out_dev);
 }
 cudaError_t launch_select(const CtlArgs &a, const UpdatePlan *up, void *out_dev, int n_seq, cudaStream_t st, bool pdl) {
-    return launch(select_kernel, n_seq, 64, st, pdl, a, up, (del_round_out *)out_dev);
+    return launch(select_kernel, n_seq, 64, st, pdl, a, *up, (del_round_out *)out_dev);
 }
 cudaError_t launch_debug_logits(const CtlArgs &a, int layer, int seq, int slot, float *out_dev, cudaStream_t st) {
     return launch(debug_logits_kernel, 296, CTL_THREADS, st, false, a, layer, seq, slot, out_dev);

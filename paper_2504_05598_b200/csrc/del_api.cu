@@ -674,22 +674,20 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
     }
     up->n_rows = rows;
     if (rows > c->R_max) return DEL_EINVAL;
-    CK(cudaMemcpyAsync(c->up_dev, up, sizeof(UpdatePlan), cudaMemcpyHostToDevice, c->st));
-    c->h2d_bytes += sizeof(UpdatePlan);
     const bool P = pdl(c);
     CtlArgs ca = ctl_base(c, -1);
     ca.mode = mode;
     ca.n_rows = rows;
-    LAUNCH(launch_prep_rows(ca, c->up_dev, rows, c->st, P));
+    LAUNCH(launch_prep_rows(ca, up, rows, c->st, P));
     if ((c->flags & FLAG_TC) && c->tc_ok) {
         // one pass over W_lm on the tensor cores, arg-max fused; partials [row][vocabulary tile]
         const int nvt = lmhead_tc_vtiles(c->D.V);
         TAG(CLS_LMSTACK, 2.0 * c->D.V * c->D.d);
         LAUNCH(launch_lmhead_tc(c->map_x, c->map_w, c->B.TPV, c->B.TPI, c->B.TPS, c->B.RS, rows, c->D.V, c->D.d, c->B.ERR,
                                 c->n_sms, c->st, P));
-        LAUNCH(launch_shadow_reduce(ca, c->up_dev, c->B.TPV, c->B.TPI, c->B.TPS, nvt, 1, nvt, 0, rows, c->st, P));
-        LAUNCH(launch_update(ca, c->up_dev, c->out_dev, up->n_seq, c->st, P));
-        if (do_select) LAUNCH(launch_select(ca, c->up_dev, c->out_dev, up->n_seq, c->st, P));
+        LAUNCH(launch_shadow_reduce(ca, up, c->B.TPV, c->B.TPI, c->B.TPS, nvt, 1, nvt, 0, rows, c->st, P));
+        LAUNCH(launch_update(ca, up, c->out_dev, up->n_seq, c->st, P));
+        if (do_select) LAUNCH(launch_select(ca, up, c->out_dev, up->n_seq, c->st, P));
         return DEL_OK;
     }
     // streaming LM head in chunks of 64 stacked rows
@@ -717,11 +715,11 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
         TAG(CLS_LMSTACK, 2.0 * c->D.V * c->D.d);
         LAUNCH(launch_rowgemm(EPI_LMHEAD, a, m, c->n_sms, c->st, P));
         const int n_part = rowgemm_lmhead_grid(a.n_items, m, c->n_sms);
-        LAUNCH(launch_shadow_reduce(ca, c->up_dev, c->B.LPV, c->B.LPI, c->B.LPS, n_part, DEL_ROWS_MAX, 1, k * DEL_ROWS_MAX, m,
+        LAUNCH(launch_shadow_reduce(ca, up, c->B.LPV, c->B.LPI, c->B.LPS, n_part, DEL_ROWS_MAX, 1, k * DEL_ROWS_MAX, m,
                                     c->st, P));
     }
-    LAUNCH(launch_update(ca, c->up_dev, c->out_dev, up->n_seq, c->st, P));
-    if (do_select) LAUNCH(launch_select(ca, c->up_dev, c->out_dev, up->n_seq, c->st, P));
+    LAUNCH(launch_update(ca, up, c->out_dev, up->n_seq, c->st, P));
+    if (do_select) LAUNCH(launch_select(ca, up, c->out_dev, up->n_seq, c->st, P));
     return DEL_OK;
 }
 
@@ -1014,9 +1012,8 @@ int del_select(del_ctx *c, int sq, int32_t *E, int32_t *gamma) {
     up->n_seq = 1;
     up->s[0].seq = sq;
     up->s[0].g = s.cur_g;            // the +-1 controller looks at the round just accepted
-    CK(cudaMemcpyAsync(c->up_dev + 1, up, sizeof(UpdatePlan), cudaMemcpyHostToDevice, c->st));
     CtlArgs ca = ctl_base(c, -1);
-    LAUNCH(launch_select(ca, c->up_dev + 1, c->out_dev, 1, c->st, pdl(c)));
+    LAUNCH(launch_select(ca, up, c->out_dev, 1, c->st, pdl(c)));
     int rc = read_out(c);
     if (rc) return rc;
     s.E = c->out_host[sq].next_E;

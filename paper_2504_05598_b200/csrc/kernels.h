@@ -52,7 +52,8 @@ struct CtlArgs {
     double omega;
 };
 
-// rows of the stacked LM head: (seq, layer, slot) per row, plus per-sequence bookkeeping of the update
+// rows of the stacked LM head: (seq, layer, slot) per row, plus per-sequence bookkeeping of the update.
+// The launchers below take a HOST pointer and pass the plan by value in the kernel parameters.
 struct UpdatePlan {
     int32_t n_seq, n_rows, pad0, pad1;
     struct {
