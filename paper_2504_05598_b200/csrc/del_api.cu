@@ -137,10 +137,10 @@ size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max
     B.TOK = c.take<int32_t>(base, (size_t)D.B * (D.S + 1));
     B.SC = c.take<double>(base, (size_t)D.B * D.L);
     B.ST = c.take<SeqState>(base, (size_t)D.B);
-    B.ERR = c.take<int32_t>(base, 64);
     B.TCNT = c.take<int32_t>(base, CTR_RING);
     *up_dev = c.take<UpdatePlan>(base, 2);
     *out_dev = c.take<del_round_out>(base, (size_t)D.B);
+    B.ERR = c.take<int32_t>(base, 64);           // right behind the results: one copy brings both to the host
     *dbg_dev = c.take<float>(base, (size_t)std::max(D.V, 2 * D.nkv * D.hd));
     // chunk buffers of the bulk prefill (PF_ROWS prompt positions)
     PfArgs pfa;
@@ -724,10 +724,11 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
 }
 
 int read_out(del_ctx *c) {
-    CK(cudaMemcpyAsync(c->out_host, c->out_dev, sizeof(del_round_out) * c->D.B, cudaMemcpyDeviceToHost, c->st));
-    c->d2h_bytes += sizeof(del_round_out) * c->D.B;
-    int32_t *err_host = reinterpret_cast<int32_t *>(c->stage_host) + 1024;
-    CK(cudaMemcpyAsync(err_host, c->B.ERR, sizeof(int32_t), cudaMemcpyDeviceToHost, c->st));
+    // the results of all sequences and the device error word behind them, in one copy
+    const size_t span = (size_t)(reinterpret_cast<const char *>(c->B.ERR) - reinterpret_cast<const char *>(c->out_dev)) + sizeof(int32_t);
+    CK(cudaMemcpyAsync(c->out_host, c->out_dev, span, cudaMemcpyDeviceToHost, c->st));
+    c->d2h_bytes += span;
+    const int32_t *err_host = reinterpret_cast<const int32_t *>(reinterpret_cast<const char *>(c->out_host) + span - sizeof(int32_t));
     CK(cudaStreamSynchronize(c->st));
     timing_collect(c);
     if (*err_host != 0) {
@@ -815,7 +816,7 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->plan_host, sizeof(PassPlan) * PLAN_RING, cudaHostAllocDefault);
     if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->up_host, sizeof(UpdatePlan) * 2, cudaHostAllocDefault);
-    if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->out_host, sizeof(del_round_out) * DEL_SEQ_MAX, cudaHostAllocDefault);
+    if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->out_host, sizeof(del_round_out) * DEL_SEQ_MAX + 1024, cudaHostAllocDefault);
     if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->stage_host, 1 << 16, cudaHostAllocDefault);
     // zero the workspace (counters, statistics) and the KV pages (stale bit patterns must stay finite)
     if (e == cudaSuccess) e = cudaMemsetAsync(workspace, 0, del_workspace_bytes(shape), c->st);
