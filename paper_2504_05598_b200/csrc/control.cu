@@ -225,6 +225,67 @@ __global__ void refresh_tau_kernel(const CtlArgs a, int seq) {
         a.B.TAU[seq * L + l] = threshold(a.B.STCS[seq * L + l], a.B.SC[seq * L + l], a.B.SFCS[seq * L + l], a.B.ST[seq].Sn);
 }
 
+// (E, gamma) = argmax of (sum_{k<=gamma} alpha_E^k) / (gamma*E + L), first maximum in E-major order.
+// Called by all threads of a block of at least 64 threads; u = index of the sequence in the update plan.
+__device__ __forceinline__ void select_body(const CtlArgs &a, const UpdatePlan *up, del_round_out *out, int u) {
+    __shared__ double s_best[64];
+    __shared__ int s_g[64];
+    const int seq = up->s[u].seq, L = a.D.L;
+    SeqState *st = a.B.ST + seq;
+    int E = a.e_min, G = a.g_min;
+    if (st->fixed_E > 0 && st->fs_mode) {
+        // baseline FS (Sec. 5.1): one more draft after a round whose drafts were all accepted, one fewer after
+        // a rejection, within [max(1, g_min), g_max]; a round without drafts changes nothing
+        E = st->fixed_E;
+        G = st->gamma;
+        const int g = up->s[u].g, n = out[seq].n_accept;
+        const int lo = a.g_min > 1 ? a.g_min : 1;
+        if (a.mode == 0 && g >= 1) G = (n == g) ? min(G + 1, a.g_max) : max(G - 1, lo);
+    } else if (st->fixed_E > 0) {
+        E = st->fixed_E;
+        G = st->fixed_gamma;
+    } else {
+        const double Sn = st->Sn;
+        double bestE = -1.0;
+        for (int l0 = a.e_min; l0 <= a.e_max; l0 += 64) {
+            const int l = l0 + threadIdx.x;
+            double best = -1.0;
+            int bg = a.g_min;
+            if (threadIdx.x < 64 && l <= a.e_max) {
+                const double alpha = __ddiv_rn(a.B.SC[seq * L + l - 1], Sn);
+                double term = 1.0, sum = 1.0;
+                for (int dd = 0; dd <= a.g_max; ++dd) {
+                    if (dd > 0) { term = __dmul_rn(term, alpha); sum = __dadd_rn(sum, term); }
+                    if (dd >= a.g_min) {
+                        const double tpl = __ddiv_rn(sum, (double)(dd * l + L));
+                        if (tpl > best) { best = tpl; bg = dd; }
+                    }
+                }
+            }
+            if (threadIdx.x < 64) { s_best[threadIdx.x] = best; s_g[threadIdx.x] = bg; }
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                for (int j = 0; j < 64 && l0 + j <= a.e_max; ++j)
+                    if (s_best[j] > bestE) { bestE = s_best[j]; E = l0 + j; G = s_g[j]; }
+            }
+            __syncthreads();
+        }
+    }
+    if (threadIdx.x == 0) {
+        st->E = E;
+        st->gamma = G;
+        out[seq].next_E = E;
+        out[seq].next_gamma = G;
+        out[seq].next_tau = a.B.TAU[seq * L + E - 1];
+    }
+}
+
+__global__ void __launch_bounds__(64) select_kernel(const CtlArgs a, const __grid_constant__ UpdatePlan up_v, del_round_out *out) {
+    pdl_launch();
+    pdl_wait();
+    select_body(a, &up_v, out, blockIdx.x);
+}
+
 // Prefix acceptance, per-layer match counts over the valid context and decayed statistics
 // (S <- omega * S + a, no fused multiply-add so that the host oracle's doubles are reproduced).
 __global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const __grid_constant__ UpdatePlan up_v, del_round_out *out) {
@@ -263,6 +324,10 @@ __global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const __gr
             o->n_emitted = 1;
             o->tokens[0] = verified[W - 1];
         }
+        if (a.do_select) {
+            __syncthreads();
+            select_body(a, up, out, u);
+        }
         return;
     }
     if (threadIdx.x == 0) {
@@ -297,64 +362,7 @@ __global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const __gr
     }
     __syncthreads();
     if (threadIdx.x == 0) tok[0] = verified[n];      // next round's input token
-}
-
-// (E, gamma) = argmax of (sum_{k<=gamma} alpha_E^k) / (gamma*E + L), first maximum in E-major order.
-__global__ void __launch_bounds__(64) select_kernel(const CtlArgs a, const __grid_constant__ UpdatePlan up_v, del_round_out *out) {
-    const UpdatePlan *up = &up_v;
-    __shared__ double s_best[64];
-    __shared__ int s_g[64];
-    pdl_launch();
-    pdl_wait();
-    const int seq = up->s[blockIdx.x].seq, L = a.D.L;
-    SeqState *st = a.B.ST + seq;
-    int E = a.e_min, G = a.g_min;
-    if (st->fixed_E > 0 && st->fs_mode) {
-        // baseline FS (Sec. 5.1): one more draft after a round whose drafts were all accepted, one fewer after
-        // a rejection, within [max(1, g_min), g_max]; a round without drafts changes nothing
-        E = st->fixed_E;
-        G = st->gamma;
-        const int g = up->s[blockIdx.x].g, n = out[seq].n_accept;
-        const int lo = a.g_min > 1 ? a.g_min : 1;
-        if (a.mode == 0 && g >= 1) G = (n == g) ? min(G + 1, a.g_max) : max(G - 1, lo);
-    } else if (st->fixed_E > 0) {
-        E = st->fixed_E;
-        G = st->fixed_gamma;
-    } else {
-        const double Sn = st->Sn;
-        double bestE = -1.0;
-        for (int l0 = a.e_min; l0 <= a.e_max; l0 += 64) {
-            const int l = l0 + threadIdx.x;
-            double best = -1.0;
-            int bg = a.g_min;
-            if (l <= a.e_max) {
-                const double alpha = __ddiv_rn(a.B.SC[seq * L + l - 1], Sn);
-                double term = 1.0, sum = 1.0;
-                for (int dd = 0; dd <= a.g_max; ++dd) {
-                    if (dd > 0) { term = __dmul_rn(term, alpha); sum = __dadd_rn(sum, term); }
-                    if (dd >= a.g_min) {
-                        const double tpl = __ddiv_rn(sum, (double)(dd * l + L));
-                        if (tpl > best) { best = tpl; bg = dd; }
-                    }
-                }
-            }
-            s_best[threadIdx.x] = best;
-            s_g[threadIdx.x] = bg;
-            __syncthreads();
-            if (threadIdx.x == 0) {
-                for (int j = 0; j < 64 && l0 + j <= a.e_max; ++j)
-                    if (s_best[j] > bestE) { bestE = s_best[j]; E = l0 + j; G = s_g[j]; }
-            }
-            __syncthreads();
-        }
-    }
-    if (threadIdx.x == 0) {
-        st->E = E;
-        st->gamma = G;
-        out[seq].next_E = E;
-        out[seq].next_gamma = G;
-        out[seq].next_tau = a.B.TAU[seq * L + E - 1];
-    }
+    if (a.do_select) select_body(a, up, out, u);     // (the statistics above are visible after the barrier)
 }
 
 // Test-only: logits of the exit head on one hidden row, straightforward one-warp-per-vocab-row dots.

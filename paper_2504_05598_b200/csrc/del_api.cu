@@ -686,8 +686,8 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
         LAUNCH(launch_lmhead_tc(c->map_x, c->map_w, c->B.TPV, c->B.TPI, c->B.TPS, c->B.RS, rows, c->D.V, c->D.d, c->B.ERR,
                                 c->n_sms, c->st, P));
         LAUNCH(launch_shadow_reduce(ca, up, c->B.TPV, c->B.TPI, c->B.TPS, nvt, 1, nvt, 0, rows, c->st, P));
+        ca.do_select = do_select;             // the selection runs at the end of the update kernel
         LAUNCH(launch_update(ca, up, c->out_dev, up->n_seq, c->st, P));
-        if (do_select) LAUNCH(launch_select(ca, up, c->out_dev, up->n_seq, c->st, P));
         return DEL_OK;
     }
     // streaming LM head in chunks of 64 stacked rows
@@ -718,8 +718,8 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
         LAUNCH(launch_shadow_reduce(ca, up, c->B.LPV, c->B.LPI, c->B.LPS, n_part, DEL_ROWS_MAX, 1, k * DEL_ROWS_MAX, m,
                                     c->st, P));
     }
+    ca.do_select = do_select;
     LAUNCH(launch_update(ca, up, c->out_dev, up->n_seq, c->st, P));
-    if (do_select) LAUNCH(launch_select(ca, up, c->out_dev, up->n_seq, c->st, P));
     return DEL_OK;
 }
 
