@@ -62,7 +62,7 @@ struct del_ctx {
     int ctr_cur = 0;                     // next free slot of the tile-claim counter ring
     PassPlan *plan_host = nullptr;       // host ring of pass plans (passed to kernels by value)
     int plan_cur = 0;
-    UpdatePlan *up_host = nullptr, *up_dev = nullptr;      // [2]
+    UpdatePlan *up_host = nullptr;                         // [2] pinned; passed to the kernels by value
     del_round_out *out_host = nullptr, *out_dev = nullptr; // [B]
     void *stage_host = nullptr;                            // small pinned scratch
     float *dbg_dev = nullptr;                              // [V] debug logits / kv rows
@@ -90,7 +90,7 @@ struct del_ctx {
 namespace {
 
 size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max, int &n_vtiles,
-                 UpdatePlan **up_dev, del_round_out **out_dev, float **dbg_dev, PfArgs *pf) {
+                 del_round_out **out_dev, float **dbg_dev, PfArgs *pf) {
     D.L = s.n_layers; D.d = s.d_model; D.nh = s.n_heads; D.nkv = s.n_kv_heads; D.hd = s.head_dim; D.F = s.d_ffn; D.V = s.vocab;
     D.B = s.max_batch;
     // slots of the hidden stack per sequence: what a round needs (g_max + 1 rows, the prefill window), raised to
@@ -138,7 +138,6 @@ size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max
     B.SC = c.take<double>(base, (size_t)D.B * D.L);
     B.ST = c.take<SeqState>(base, (size_t)D.B);
     B.TCNT = c.take<int32_t>(base, CTR_RING);
-    *up_dev = c.take<UpdatePlan>(base, 2);
     *out_dev = c.take<del_round_out>(base, (size_t)D.B);
     B.ERR = c.take<int32_t>(base, 64);           // right behind the results: one copy brings both to the host
     *dbg_dev = c.take<float>(base, (size_t)std::max(D.V, 2 * D.nkv * D.hd));
@@ -774,8 +773,8 @@ extern "C" {
 
 size_t del_workspace_bytes(const del_shape *shape) {
     if (validate(shape) != DEL_OK) return 0;
-    Dims D; Buffers B; int R, nv; UpdatePlan *u; del_round_out *o; float *dbg;
-    return carve_all(*shape, nullptr, D, B, R, nv, &u, &o, &dbg, nullptr);
+    Dims D; Buffers B; int R, nv; del_round_out *o; float *dbg;
+    return carve_all(*shape, nullptr, D, B, R, nv, &o, &dbg, nullptr);
 }
 
 int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const del_kv *kv, void *workspace,
@@ -791,7 +790,7 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
     del_ctx *c = new (std::nothrow) del_ctx();
     if (!c) return DEL_ENOSPC;
     c->sh = *shape;
-    carve_all(*shape, workspace, c->D, c->B, c->R_max, c->n_vtiles, &c->up_dev, &c->out_dev, &c->dbg_dev, &c->pf);
+    carve_all(*shape, workspace, c->D, c->B, c->R_max, c->n_vtiles, &c->out_dev, &c->dbg_dev, &c->pf);
     c->B.KP = (bf16 *)kv->k_pages; c->B.VP = (bf16 *)kv->v_pages; c->B.PT = kv->page_table;
     c->B.rope_cos = w->rope_cos; c->B.rope_sin = w->rope_sin;
     c->tok_emb = (const bf16 *)w->tok_emb; c->final_norm = (const bf16 *)w->final_norm; c->lm_head = (const bf16 *)w->lm_head;
