@@ -137,6 +137,11 @@ __global__ void __launch_bounds__(CTL_THREADS) draft_finalize_embed_kernel(const
         s_tok = idx;
         a.B.TOK[rd.seq * (a.D.S + 1) + rd.slot + 1] = idx;
         a.B.DCONF[rd.seq * (a.D.S + 1) + rd.slot + 1] = conf;
+        if (a.post_conf != nullptr) {
+            a.post_conf[rd.seq] = conf;
+            __threadfence_system();              // the confidence is in host memory before the stamp that announces it
+            a.post_stamp[rd.seq] = a.stamp;
+        }
     }
     __syncthreads();
     if (embed_next) write_embedding(a, s_tok, rd.seq, rd.slot + 1);

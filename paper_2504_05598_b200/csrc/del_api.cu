@@ -5,6 +5,7 @@
 #include "kernels.h"
 
 #include <algorithm>
+#include <chrono>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -73,6 +74,10 @@ struct del_ctx {
     TMap pf_xs, pf_att, pf_xm, pf_act;
     std::vector<TMap> pf_wq, pf_wk, pf_wv, pf_wo, pf_wg, pf_wu, pf_wd;
     bool pf_ok = false;
+    // mailbox of the draft loop's confidence check: pinned host memory that the finalise kernel writes directly
+    volatile float *post_conf = nullptr;
+    volatile uint32_t *post_stamp = nullptr;
+    uint32_t post_seq = 0;
     bool tc_ok = false;
     int64_t launches = 0, h2d_bytes = 0, d2h_bytes = 0;
     // optional per-launch timing (FLAG_TIMING): events around every launch, summed per kernel class
@@ -453,7 +458,7 @@ void plan_draft_step(del_ctx *c, PlanBatch &pb, const std::vector<Job> &act, con
 }
 
 // layers 1..E of every drafting row, the exit head in one pass over W_lm, arg-max + confidence, next embedding
-int launch_draft_step(del_ctx *c, const DraftStep &st, const std::vector<int> &Es, int i) {
+int launch_draft_step(del_ctx *c, const DraftStep &st, const std::vector<int> &Es, int i, uint32_t stamp = 0) {
     const bool P = pdl(c);
     const PassInfo full = pass_info(c, st.full_idx);
     if (i == 0) {
@@ -478,6 +483,11 @@ int launch_draft_step(del_ctx *c, const DraftStep &st, const std::vector<int> &E
     LAUNCH(launch_rowgemm(EPI_LMHEAD, a, full.m, c->n_sms, c->st, P));
     CtlArgs ca = ctl_base(c, full.plan_idx);
     ca.n_part = rowgemm_lmhead_grid(a.n_items, full.m, c->n_sms);
+    if (stamp != 0 && c->post_conf != nullptr) {
+        ca.post_conf = c->post_conf;
+        ca.post_stamp = c->post_stamp;
+        ca.stamp = stamp;
+    }
     LAUNCH(launch_draft_finalize_embed(ca, full.m, true, c->st, P));
     return DEL_OK;
 }
@@ -534,17 +544,37 @@ int draft_with_exit(del_ctx *c, std::vector<Job> &jobs) {
         plan_draft_step(c, pb, act, Es, i, st);
         rc = plan_commit(c, pb);
         if (rc) return rc;
-        rc = launch_draft_step(c, st, Es, i);
+        const uint32_t stamp = ++c->post_seq ? c->post_seq : ++c->post_seq;     // never 0
+        rc = launch_draft_step(c, st, Es, i, stamp);
         if (rc) return rc;
-        bool any = false;
-        for (size_t k : who)
-            if (c->seq[jobs[k].seq].exit_mode) {
-                CK(cudaMemcpyAsync(conf_host + k, c->B.DCONF + (size_t)jobs[k].seq * (c->D.S + 1) + i + 1, sizeof(float),
-                                   cudaMemcpyDeviceToHost, c->st));
-                c->d2h_bytes += sizeof(float);
-                any = true;
+        // The finalise kernel posts each sequence's confidence in pinned host memory; the host polls the stamp
+        // (about a second at most), so the next step can be enqueued while that kernel is still writing the
+        // next embedding.  Without the mailbox, or if the stamp does not arrive: copy + synchronise.
+        bool posted = c->post_conf != nullptr && !(c->flags & FLAG_TIMING);
+        if (posted) {
+            const auto t0 = std::chrono::steady_clock::now();
+            for (size_t k : who) {
+                const int sq = jobs[k].seq;
+                if (!c->seq[sq].exit_mode) continue;
+                while (c->post_stamp[sq] != stamp) {
+                    if (std::chrono::steady_clock::now() - t0 > std::chrono::seconds(1)) { posted = false; break; }
+                }
+                if (!posted) break;
+                conf_host[k] = c->post_conf[sq];
+                c->d2h_bytes += sizeof(float) + sizeof(uint32_t);
             }
-        if (any) CK(cudaStreamSynchronize(c->st));
+        }
+        if (!posted) {
+            bool any = false;
+            for (size_t k : who)
+                if (c->seq[jobs[k].seq].exit_mode) {
+                    CK(cudaMemcpyAsync(conf_host + k, c->B.DCONF + (size_t)jobs[k].seq * (c->D.S + 1) + i + 1, sizeof(float),
+                                       cudaMemcpyDeviceToHost, c->st));
+                    c->d2h_bytes += sizeof(float);
+                    any = true;
+                }
+            if (any) CK(cudaStreamSynchronize(c->st));
+        }
         for (size_t k : who) {
             const SeqHost &s = c->seq[jobs[k].seq];
             if (s.exit_mode && (double)conf_host[k] < s.cur_tau) jobs[k].stopped = 1;   // Algorithm 1: break, token dropped
@@ -817,6 +847,22 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
     if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->up_host, sizeof(UpdatePlan) * 2, cudaHostAllocDefault);
     if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->out_host, sizeof(del_round_out) * DEL_SEQ_MAX + 1024, cudaHostAllocDefault);
     if (e == cudaSuccess) e = cudaHostAlloc((void **)&c->stage_host, 1 << 16, cudaHostAllocDefault);
+    if (e == cudaSuccess) {
+        // mailbox for the draft loop's confidence check (device-writable pinned memory); optional
+        void *mb = nullptr;
+        if (cudaHostAlloc(&mb, 2 * DEL_SEQ_MAX * sizeof(uint32_t), cudaHostAllocMapped) == cudaSuccess) {
+            memset(mb, 0, 2 * DEL_SEQ_MAX * sizeof(uint32_t));
+            void *dp = nullptr;
+            if (cudaHostGetDevicePointer(&dp, mb, 0) == cudaSuccess && dp == mb) {
+                c->post_conf = reinterpret_cast<volatile float *>(mb);
+                c->post_stamp = reinterpret_cast<volatile uint32_t *>(mb) + DEL_SEQ_MAX;
+            } else {
+                cudaFreeHost(mb);
+            }
+        } else {
+            cudaGetLastError();
+        }
+    }
     // zero the workspace (counters, statistics) and the KV pages (stale bit patterns must stay finite)
     if (e == cudaSuccess) e = cudaMemsetAsync(workspace, 0, del_workspace_bytes(shape), c->st);
     const size_t kv_bytes = (size_t)shape->n_pages * L * shape->n_kv_heads * 16 * shape->head_dim * sizeof(bf16);
@@ -867,6 +913,7 @@ void del_destroy(del_ctx *c) {
     if (c->up_host) cudaFreeHost(c->up_host);
     if (c->out_host) cudaFreeHost(c->out_host);
     if (c->stage_host) cudaFreeHost(c->stage_host);
+    if (c->post_conf) cudaFreeHost(const_cast<float *>(c->post_conf));
     for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
     delete c;
 }

@@ -50,6 +50,11 @@ struct CtlArgs {
     int32_t n_rows;            // rows of the stacked LM-head problem
     int32_t n_vtiles;
     double omega;
+    // draft loop with the confidence break: the finalise kernel also posts (confidence, stamp) per sequence in
+    // host memory that the device can write, so that the host sees it without a copy and a stream synchronisation
+    volatile float *post_conf;          // [DEL_SEQ_MAX] device-visible host memory, or nullptr
+    volatile uint32_t *post_stamp;      // [DEL_SEQ_MAX]
+    uint32_t stamp;
 };
 
 // rows of the stacked LM head: (seq, layer, slot) per row, plus per-sequence bookkeeping of the update.
