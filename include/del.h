@@ -157,9 +157,12 @@ int del_layer_accept(del_ctx *ctx, int seq, del_round_out *out);
 int del_select(del_ctx *ctx, int seq, int32_t *E, int32_t *gamma);
 
 /* One whole round for every live sequence at once (each with its own E, gamma and state): draft,
- * verify, layer_accept and select with layer passes shared by the sequences, one host
- * synchronisation at the end.  out: HOST array [max_batch]; entries of sequences that are not live
- * get n_emitted = 0.  Returns DEL_ESTATE if no sequence is live. */
+ * verify, layer_accept and select with layer passes shared by the sequences, and one host round trip
+ * at the end: the last kernel posts the results in pinned host memory and the call returns as soon as
+ * they are there (that kernel may still be retiring; anything enqueued on the stream afterwards is
+ * ordered behind it, and every other call of this library synchronises before it reads device state).
+ * out: HOST array [max_batch]; entries of sequences that are not live get n_emitted = 0.  Returns
+ * DEL_ESTATE if no sequence is live. */
 int del_round(del_ctx *ctx, del_round_out *out);
 
 /* Fix the policy of a sequence: del_round uses (E, gamma) as given instead of the selection

@@ -368,6 +368,19 @@ __global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const __gr
     __syncthreads();
     if (threadIdx.x == 0) tok[0] = verified[n];      // next round's input token
     if (a.do_select) select_body(a, up, out, u);     // (the statistics above are visible after the barrier)
+    if (a.post_out != nullptr) {
+        // the finished result goes to device-writable host memory, then the stamp that announces it
+        __syncthreads();
+        constexpr int NWORD = (int)(sizeof(del_round_out) / sizeof(int32_t));
+        const int32_t *src = reinterpret_cast<const int32_t *>(o);
+        volatile int32_t *dst = a.post_out + (size_t)seq * NWORD;
+        constexpr int STATUS_WORD = (int)(offsetof(del_round_out, status) / sizeof(int32_t));
+        for (int w = threadIdx.x; w < NWORD; w += blockDim.x)
+            dst[w] = w == STATUS_WORD ? *reinterpret_cast<volatile int32_t *>(a.B.ERR) : src[w];
+        __threadfence_system();
+        __syncthreads();
+        if (threadIdx.x == 0) a.post_done[seq] = a.stamp;
+    }
 }
 
 // Test-only: logits of the exit head on one hidden row, straightforward one-warp-per-vocab-row dots.

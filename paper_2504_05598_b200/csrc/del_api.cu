@@ -77,6 +77,8 @@ struct del_ctx {
     // mailbox of the draft loop's confidence check: pinned host memory that the finalise kernel writes directly
     volatile float *post_conf = nullptr;
     volatile uint32_t *post_stamp = nullptr;
+    volatile int32_t *post_out = nullptr;                 // round results posted by the update kernel
+    volatile uint32_t *post_done = nullptr;
     uint32_t post_seq = 0;
     bool tc_ok = false;
     int64_t launches = 0, h2d_bytes = 0, d2h_bytes = 0;
@@ -692,7 +694,7 @@ int enqueue_verify(del_ctx *c, const std::vector<Job> &jobs) {
 }
 
 // ---- stacked LM head + arg-max over all layers' hidden rows (a6), then accept / counts (a7-a8)
-int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bool do_select) {
+int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bool do_select, uint32_t post_stamp = 0) {
     UpdatePlan *up = &c->up_host[0];
     memset(up, 0, sizeof(*up));
     int rows = 0;
@@ -707,6 +709,11 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
     CtlArgs ca = ctl_base(c, -1);
     ca.mode = mode;
     ca.n_rows = rows;
+    if (post_stamp != 0 && c->post_out != nullptr) {
+        ca.post_out = c->post_out;
+        ca.post_done = c->post_done;
+        ca.stamp = post_stamp;
+    }
     LAUNCH(launch_prep_rows(ca, up, rows, c->st, P));
     if ((c->flags & FLAG_TC) && c->tc_ok) {
         // one pass over W_lm on the tensor cores, arg-max fused; partials [row][vocabulary tile]
@@ -850,12 +857,15 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
     if (e == cudaSuccess) {
         // mailbox for the draft loop's confidence check (device-writable pinned memory); optional
         void *mb = nullptr;
-        if (cudaHostAlloc(&mb, 2 * DEL_SEQ_MAX * sizeof(uint32_t), cudaHostAllocMapped) == cudaSuccess) {
-            memset(mb, 0, 2 * DEL_SEQ_MAX * sizeof(uint32_t));
+        const size_t mb_bytes = 3 * DEL_SEQ_MAX * sizeof(uint32_t) + DEL_SEQ_MAX * sizeof(del_round_out);
+        if (cudaHostAlloc(&mb, mb_bytes, cudaHostAllocMapped) == cudaSuccess) {
+            memset(mb, 0, mb_bytes);
             void *dp = nullptr;
             if (cudaHostGetDevicePointer(&dp, mb, 0) == cudaSuccess && dp == mb) {
                 c->post_conf = reinterpret_cast<volatile float *>(mb);
                 c->post_stamp = reinterpret_cast<volatile uint32_t *>(mb) + DEL_SEQ_MAX;
+                c->post_done = reinterpret_cast<volatile uint32_t *>(mb) + 2 * DEL_SEQ_MAX;
+                c->post_out = reinterpret_cast<volatile int32_t *>(reinterpret_cast<uint32_t *>(mb) + 3 * DEL_SEQ_MAX);
             } else {
                 cudaFreeHost(mb);
             }
@@ -1097,10 +1107,31 @@ int del_round(del_ctx *c, del_round_out *out) {
     for (const Job &j : jobs) { c->seq[j.seq].cur_g = j.g; c->seq[j.seq].cur_stopped = j.stopped; }
     rc = enqueue_verify(c, jobs);
     if (rc) return rc;
-    rc = enqueue_update(c, jobs, 0, 0, true);
+    // The update kernel posts every sequence's result and a stamp in pinned host memory; polling that is a
+    // shorter way home than a copy and a stream synchronisation.  Timing mode and the fall-back use the copy.
+    const bool mailbox = c->post_out != nullptr && !(c->flags & FLAG_TIMING);
+    const uint32_t stamp = ++c->post_seq ? c->post_seq : ++c->post_seq;
+    rc = enqueue_update(c, jobs, 0, 0, true, mailbox ? stamp : 0);
     if (rc) return rc;
-    rc = read_out(c);
-    if (rc) return rc;
+    bool posted = mailbox;
+    if (posted) {
+        const auto t0 = std::chrono::steady_clock::now();
+        constexpr int NWORD = (int)(sizeof(del_round_out) / sizeof(int32_t));
+        for (const Job &j : jobs) {
+            while (c->post_done[j.seq] != stamp) {
+                if (std::chrono::steady_clock::now() - t0 > std::chrono::seconds(2)) { posted = false; break; }
+            }
+            if (!posted) break;
+            int32_t *dst = reinterpret_cast<int32_t *>(&c->out_host[j.seq]);
+            for (int w = 0; w < NWORD; ++w) dst[w] = c->post_out[(size_t)j.seq * NWORD + w];
+            c->d2h_bytes += sizeof(del_round_out);
+            if (c->out_host[j.seq].status != 0) posted = false;      // let the copy path report and clear the error
+        }
+    }
+    if (!posted) {
+        rc = read_out(c);
+        if (rc) return rc;
+    }
     for (const Job &j : jobs) finish_round(c, j.seq, &out[j.seq], true);
     return DEL_OK;
 }

@@ -55,6 +55,10 @@ struct CtlArgs {
     volatile float *post_conf;          // [DEL_SEQ_MAX] device-visible host memory, or nullptr
     volatile uint32_t *post_stamp;      // [DEL_SEQ_MAX]
     uint32_t stamp;
+    // end of a round: the update kernel also posts every sequence's result (with the device error word as its
+    // status) and a stamp there
+    volatile int32_t *post_out;         // [DEL_SEQ_MAX][sizeof(del_round_out) / 4], or nullptr
+    volatile uint32_t *post_done;       // [DEL_SEQ_MAX]
 };
 
 // rows of the stacked LM head: (seq, layer, slot) per row, plus per-sequence bookkeeping of the update.
