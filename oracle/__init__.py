@@ -54,6 +54,12 @@ class RoundInfo(C.Structure):
                 ("draft_conf", C.c_double * (MAX_GAMMA + 1))]
 
 
+class SampleInfo(C.Structure):
+    _fields_ = [("n_tests", C.c_int32), ("from_residual", C.c_int32), ("u_draft", C.c_double * MAX_GAMMA),
+                ("u_accept", C.c_double * MAX_GAMMA), ("u_final", C.c_double), ("q_x", C.c_double * MAX_GAMMA),
+                ("p_x", C.c_double * MAX_GAMMA)]
+
+
 def lib():
     global _lib
     if _lib is not None:
@@ -103,6 +109,17 @@ def lib():
     L.ora_confidence.argtypes = [vp, i32]
     L.ora_threshold.restype = f64
     L.ora_threshold.argtypes = [f64, f64, f64, f64]
+    L.ora_uniform.restype = f64
+    L.ora_uniform.argtypes = [C.c_uint64, C.c_int64, i32]
+    L.ora_nucleus.argtypes = [vp, i32, f64, f64, vp]
+    L.ora_sample_cdf.restype = i32
+    L.ora_sample_cdf.argtypes = [vp, i32, f64]
+    L.ora_residual.restype = f64
+    L.ora_residual.argtypes = [vp, vp, i32, vp]
+    L.ora_set_sampling.argtypes = [vp, f64, f64, C.c_uint64]
+    L.ora_get_sample_info.argtypes = [vp, C.POINTER(SampleInfo)]
+    L.ora_round_logits.restype = C.POINTER(f32)
+    L.ora_round_logits.argtypes = [vp, i32, i32]
     _lib = L
     return L
 
@@ -190,6 +207,20 @@ class OracleSeq:
     def set_exit_mode(self, on: bool):
         """Dynamic draft-exiting (Sec. 4.4): draft up to g_max tokens, stop at the first low-confidence one."""
         lib().ora_set_exit_mode(self._h, 1 if on else 0)
+
+    def set_sampling(self, temperature: float, top_p: float, seed: int):
+        """Speculative sampling (Sec. 2) with temperature and nucleus filtering; temperature <= 0: greedy."""
+        lib().ora_set_sampling(self._h, float(temperature), float(top_p), int(seed))
+
+    def sample_info(self) -> SampleInfo:
+        out = SampleInfo()
+        lib().ora_get_sample_info(self._h, C.byref(out))
+        return out
+
+    def round_logits(self, which: int, row: int) -> np.ndarray:
+        """Logits of the last round: which = 0 the exit head's row of draft `row`, 1 the target's row."""
+        p = lib().ora_round_logits(self._h, which, row)
+        return np.ctypeslib.as_array(p, shape=(self.cfg.vocab,)).copy()
 
     def get_conf_stats(self):
         L = self.cfg.n_layers
@@ -302,6 +333,30 @@ def softmax(x: np.ndarray) -> np.ndarray:
 def confidence(logits: np.ndarray) -> float:
     x = np.ascontiguousarray(logits, dtype=np.float32)
     return lib().ora_confidence(x.ctypes.data, x.size)
+
+
+def uniform(seed: int, pos: int, purpose: int) -> float:
+    return lib().ora_uniform(int(seed), int(pos), int(purpose))
+
+
+def nucleus(logits: np.ndarray, temperature: float, top_p: float) -> np.ndarray:
+    x = np.ascontiguousarray(logits, dtype=np.float32)
+    p = np.zeros(x.size, dtype=np.float64)
+    lib().ora_nucleus(x.ctypes.data, x.size, float(temperature), float(top_p), p.ctypes.data)
+    return p
+
+
+def sample_cdf(probs: np.ndarray, u: float) -> int:
+    p = np.ascontiguousarray(probs, dtype=np.float64)
+    return lib().ora_sample_cdf(p.ctypes.data, p.size, float(u))
+
+
+def residual(p: np.ndarray, q: np.ndarray):
+    p = np.ascontiguousarray(p, dtype=np.float64)
+    q = np.ascontiguousarray(q, dtype=np.float64)
+    r = np.zeros_like(p)
+    R = lib().ora_residual(p.ctypes.data, q.ctypes.data, p.size, r.ctypes.data)
+    return r, R
 
 
 def threshold(Stcs: float, Sc: float, Sfcs: float, Smis: float) -> float:

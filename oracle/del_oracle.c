@@ -39,6 +39,10 @@ struct ora_seq {
     double *tau;        /* [L] thresholds of Eq. 3 from the current statistics */
     double *conf;       /* [L][rows] confidence of every shadow token of the last round / prefill window */
     int32_t exit_mode;  /* 1: the draft loop runs up to g_max steps and stops on a low confidence */
+    double temperature, top_p; /* speculative sampling (temperature <= 0: greedy) */
+    uint64_t seed;
+    float *qlog, *plog; /* [g_max + 1][V] logits of the exit head per draft / of the target per row, last round */
+    ora_sample_info sinfo;
     float *K, *V;       /* [L][max_seq][n_kv*hd] */
     float *H;           /* [L+1][rows][d] hidden stack */
     int32_t rows;       /* rows per layer in H */
@@ -192,7 +196,7 @@ ora_seq *ora_seq_create(const ora_shape *shape, const ora_weights *w) {
 void ora_seq_destroy(ora_seq *s) {
     if (!s) return;
     free(s->K); free(s->V); free(s->H); free(s->Sc); free(s->rope_cos); free(s->rope_sin);
-    free(s->Stcs); free(s->Sfcs); free(s->tau); free(s->conf);
+    free(s->Stcs); free(s->Sfcs); free(s->tau); free(s->conf); free(s->qlog); free(s->plog);
     free(s);
 }
 
@@ -409,6 +413,88 @@ int32_t ora_accept_len(const int32_t *drafts, const int32_t *verified, int32_t g
     return n;
 }
 
+/* ---------------------------------------------------------------- speculative sampling (Sec. 2) */
+
+/* finaliser of the splitmix64 generator (a bijective 64-bit mixer) */
+static uint64_t mix64(uint64_t x) {
+    x ^= x >> 30; x *= 0xBF58476D1CE4E5B9ull;
+    x ^= x >> 27; x *= 0x94D049BB133111EBull;
+    x ^= x >> 31;
+    return x;
+}
+
+double ora_uniform(uint64_t seed, int64_t pos, int32_t purpose) {
+    const uint64_t ctr = (uint64_t)pos * 4u + (uint64_t)purpose + 1u;
+    const uint64_t x = mix64(seed ^ mix64(ctr * 0x9E3779B97F4A7C15ull));
+    return (double)(x >> 11) * (1.0 / 9007199254740992.0);      /* 53 bits */
+}
+
+typedef struct { double p; int32_t id; } prob_id;
+static int by_prob_desc(const void *a, const void *b) {
+    const prob_id *x = (const prob_id *)a, *y = (const prob_id *)b;
+    if (x->p > y->p) return -1;
+    if (x->p < y->p) return 1;
+    return x->id < y->id ? -1 : (x->id > y->id ? 1 : 0);
+}
+
+void ora_nucleus(const float *logits, int32_t V, double temperature, double top_p, double *probs) {
+    double mx = logits[0];
+    for (int32_t t = 1; t < V; ++t)
+        if (logits[t] > mx) mx = logits[t];
+    double Z = 0.0;
+    for (int32_t t = 0; t < V; ++t) { probs[t] = exp(((double)logits[t] - mx) / temperature); Z += probs[t]; }
+    for (int32_t t = 0; t < V; ++t) probs[t] /= Z;
+    if (top_p >= 1.0) return;
+    prob_id *o = (prob_id *)malloc(sizeof(prob_id) * (size_t)V);
+    for (int32_t t = 0; t < V; ++t) { o[t].p = probs[t]; o[t].id = t; }
+    qsort(o, (size_t)V, sizeof(prob_id), by_prob_desc);
+    double before = 0.0;                /* mass of the tokens ahead in the descending order */
+    int32_t k = 0;
+    while (k < V && before < top_p) { before += o[k].p; ++k; }
+    for (int32_t j = k; j < V; ++j) probs[o[j].id] = 0.0;
+    free(o);
+    double K = 0.0;
+    for (int32_t t = 0; t < V; ++t) K += probs[t];
+    for (int32_t t = 0; t < V; ++t) probs[t] /= K;
+}
+
+int32_t ora_sample_cdf(const double *probs, int32_t V, double u) {
+    double c = 0.0;
+    int32_t last = 0;
+    for (int32_t t = 0; t < V; ++t) {
+        if (probs[t] <= 0.0) continue;
+        c += probs[t];
+        last = t;
+        if (u < c) return t;
+    }
+    return last;                        /* u beyond the rounded total: the last token with mass */
+}
+
+double ora_residual(const double *p, const double *q, int32_t V, double *r) {
+    double R = 0.0;
+    for (int32_t t = 0; t < V; ++t) { r[t] = p[t] > q[t] ? p[t] - q[t] : 0.0; R += r[t]; }
+    if (R <= 0.0) { memcpy(r, p, sizeof(double) * (size_t)V); return 0.0; }
+    for (int32_t t = 0; t < V; ++t) r[t] /= R;
+    return R;
+}
+
+void ora_set_sampling(ora_seq *s, double temperature, double top_p, uint64_t seed) {
+    s->temperature = temperature;
+    s->top_p = top_p;
+    s->seed = seed;
+    if (temperature > 0.0 && !s->qlog) {
+        const size_t n = (size_t)(s->sh.g_max + 1) * s->sh.vocab;
+        s->qlog = (float *)calloc(n, sizeof(float));
+        s->plog = (float *)calloc(n, sizeof(float));
+    }
+}
+
+void ora_get_sample_info(const ora_seq *s, ora_sample_info *out) { *out = s->sinfo; }
+
+const float *ora_round_logits(const ora_seq *s, int32_t which, int32_t row) {
+    return (which ? s->plog : s->qlog) + (size_t)row * s->sh.vocab;
+}
+
 /* One step of S(a) = sum_i omega^(r-i-1) a[i], written as the recursion S <- omega*S + a (Sec. 4.2). */
 double ora_decay_step(double S, double omega, double a) {
     double t = omega * S;
@@ -494,6 +580,14 @@ int32_t ora_prefill(ora_seq *s, const int32_t *prompt, int32_t P, int32_t *shado
     s->T = P;
     s->x_in = sd[(size_t)(L - 1) * W + (W - 1)];
     free(sd);
+    if (s->temperature > 0.0) {
+        /* the first generated token is drawn from the target's filtered distribution at the last prompt position */
+        double *pp = (double *)malloc(sizeof(double) * (size_t)sh->vocab);
+        ora_exit_head(s, hidden_at(s, L, W - 1), NULL, NULL, s->plog);
+        ora_nucleus(s->plog, sh->vocab, s->temperature, s->top_p, pp);
+        s->x_in = ora_sample_cdf(pp, sh->vocab, ora_uniform(s->seed, P, 2));
+        free(pp);
+    }
     choose_next(s, 0, 0);
     if (info) {
         memset(info, 0, sizeof(*info));
@@ -521,14 +615,36 @@ int ora_round(ora_seq *s, int32_t remaining, ora_round_info *info, int32_t *shad
     double draft_conf[ORA_MAX_GAMMA + 1];
     const double tau_E = s->tau[E - 1];
     int32_t in = s->x_in, g = 0, stopped = 0;
+    const int samp = s->temperature > 0.0;
+    const int32_t V = sh->vocab;
+    double *pp = NULL, *qq = NULL, *rr = NULL;
+    if (samp) {
+        pp = (double *)malloc(sizeof(double) * (size_t)V);
+        qq = (double *)malloc(sizeof(double) * (size_t)V);
+        rr = (double *)malloc(sizeof(double) * (size_t)V);
+        memset(&s->sinfo, 0, sizeof(s->sinfo));
+    }
     /* draft: tokens through layers 1..E + exit head (Algorithm 1, draft loop); a token whose confidence is
      * below the threshold ends the loop and is not appended */
     for (int32_t i = 0; i < g_cap; ++i) {
         int32_t tok;
         ora_embed(s, in, hidden_at(s, 0, i));
         for (int32_t l = 1; l <= E; ++l) ora_layer_rows(s, l, hidden_at(s, l - 1, i), s->T + i, 1, hidden_at(s, l, i));
-        exit_head_conf(s, hidden_at(s, E, i), &tok, NULL, &draft_conf[i]);
-        if (s->exit_mode && draft_conf[i] < tau_E) { stopped = 1; break; }
+        if (samp) {
+            /* the confidence stays the top-1 probability at temperature 1 (Sec. 4.4); the token is drawn from the
+             * exit head's filtered distribution */
+            float *lg = s->qlog + (size_t)i * V;
+            ora_exit_head(s, hidden_at(s, E, i), &tok, NULL, lg);
+            draft_conf[i] = ora_confidence(lg, V);
+            if (s->exit_mode && draft_conf[i] < tau_E) { stopped = 1; break; }
+            ora_nucleus(lg, V, s->temperature, s->top_p, qq);
+            s->sinfo.u_draft[i] = ora_uniform(s->seed, (int64_t)s->T + 1 + i, 0);
+            tok = ora_sample_cdf(qq, V, s->sinfo.u_draft[i]);
+            s->sinfo.q_x[i] = qq[tok];
+        } else {
+            exit_head_conf(s, hidden_at(s, E, i), &tok, NULL, &draft_conf[i]);
+            if (s->exit_mode && draft_conf[i] < tau_E) { stopped = 1; break; }
+        }
         drafts[g++] = tok;
         in = tok;
     }
@@ -547,7 +663,39 @@ int ora_round(ora_seq *s, int32_t remaining, ora_round_info *info, int32_t *shad
             if (margin) margin[(size_t)(l - 1) * stride + i] = mg;
         }
     const int32_t *verified = sd + (size_t)(L - 1) * stride;
-    const int32_t n = ora_accept_len(drafts, verified, g);
+    int32_t n, last_token;
+    if (samp) {
+        /* Sec. 2: draft i is accepted with probability min(1, p(x)/q(x)); after the first rejection the token
+         * comes from the normalised max(0, p - q) of that position, after g acceptances from p at position g */
+        for (int32_t i = 0; i <= g; ++i) ora_exit_head(s, hidden_at(s, L, i), NULL, NULL, s->plog + (size_t)i * V);
+        n = 0;
+        int rejected = 0;
+        while (n < g) {
+            const int32_t x = drafts[n];
+            ora_nucleus(s->plog + (size_t)n * V, V, s->temperature, s->top_p, pp);
+            ora_nucleus(s->qlog + (size_t)n * V, V, s->temperature, s->top_p, qq);
+            const double u = ora_uniform(s->seed, (int64_t)s->T + 1 + n, 1);
+            s->sinfo.u_accept[n] = u;
+            s->sinfo.p_x[n] = pp[x];
+            s->sinfo.n_tests = n + 1;
+            const double ratio = pp[x] / qq[x];
+            if (u < (ratio < 1.0 ? ratio : 1.0)) ++n;
+            else { rejected = 1; break; }
+        }
+        s->sinfo.u_final = ora_uniform(s->seed, (int64_t)s->T + 1 + n, 2);
+        s->sinfo.from_residual = rejected;
+        if (rejected) {
+            ora_residual(pp, qq, V, rr);
+            last_token = ora_sample_cdf(rr, V, s->sinfo.u_final);
+        } else {
+            ora_nucleus(s->plog + (size_t)g * V, V, s->temperature, s->top_p, pp);
+            last_token = ora_sample_cdf(pp, V, s->sinfo.u_final);
+        }
+        free(pp); free(qq); free(rr);
+    } else {
+        n = ora_accept_len(drafts, verified, g);
+        last_token = verified[n];
+    }
     /* matches within the valid context i = 0..n, decayed statistics (Eq. 2); the number of valid
      * positions is n + 1 */
     for (int32_t l = 1; l <= L; ++l) {
@@ -571,14 +719,15 @@ int ora_round(ora_seq *s, int32_t remaining, ora_round_info *info, int32_t *shad
         info->E = E; info->gamma = s->gamma; info->g = g;
         info->n_accept = n; info->n_emitted = n + 1;
         for (int32_t i = 0; i < g; ++i) info->drafts[i] = drafts[i];
-        for (int32_t i = 0; i <= n; ++i) info->emitted[i] = verified[i];
+        for (int32_t i = 0; i < n; ++i) info->emitted[i] = drafts[i];   /* (greedy: equal to the target's tokens) */
+        info->emitted[n] = last_token;
         info->loaded_layers = g * E + L;
         info->stopped = stopped;
         info->tau = tau_E;
         for (int32_t i = 0; i < g + stopped; ++i) info->draft_conf[i] = draft_conf[i];
     }
     s->T += n + 1;
-    s->x_in = verified[n];
+    s->x_in = last_token;
     free(sd);
     choose_next(s, g, n);
     if (info) { info->next_E = s->E; info->next_gamma = s->gamma; info->Sn = s->Sn; info->next_tau = s->tau[s->E - 1]; }

@@ -18,6 +18,11 @@
  * definition, exhaustive evaluation of the tokens-per-layer formula, and for
  * dynamic draft-exiting: the softmax definition of the confidence, Eq. 3 from
  * explicit histories, and the two limits of the threshold (never / always stop).
+ * Speculative sampling: the uniform numbers by a Kolmogorov-Smirnov test, the
+ * filtered distribution by scipy / numpy on the same rows and its limits, the
+ * inverse CDF by numpy's searchsorted, acceptance and residual by the identity
+ * that makes speculative sampling exact and by a Monte-Carlo run, the round by
+ * a replay of its decisions from the logits it exposes.
  * Parity unpinned: the absolute values of logits of the random model (no
  * published activations exist) and any distribution-level behaviour that would
  * need the paper's trained checkpoints.
@@ -132,6 +137,42 @@ double ora_tpl(double alpha, int32_t l, int32_t d, int32_t L);
 void ora_select(const double *Sc /*index l-1*/, double Sn, int32_t L, int32_t e_min, int32_t e_max, int32_t g_min,
                 int32_t g_max, int32_t *E, int32_t *gamma);
 int ora_num_threads(void);
+
+/* ---- speculative sampling (Sec. 2: accept a draft with probability min(1, p/q), otherwise resample from
+ * the normalised max(0, p - q); one more token from p when every draft was accepted), with the temperature
+ * and nucleus (top-p) filtering of Sec. 5 / the inference setup applied to both distributions. */
+
+/* Uniform number in [0, 1) of a counter-based generator: a function of (seed, absolute position of the token
+ * being decided, purpose) only, so that no generator state has to be carried.  purpose 0: drawing the draft
+ * token, 1: the acceptance test of that draft, 2: the token that ends the round (residual or extra token). */
+double ora_uniform(uint64_t seed, int64_t pos, int32_t purpose);
+/* probs[i] = softmax(logits / temperature) restricted to the nucleus and renormalised.  The nucleus is the
+ * shortest prefix, in order of descending probability (equal probabilities: lower token id first), whose mass
+ * reaches top_p: a token is kept iff the mass strictly before it is < top_p.  top_p >= 1 keeps everything. */
+void ora_nucleus(const float *logits, int32_t V, double temperature, double top_p, double *probs);
+/* inverse CDF in token-id order: the first token whose cumulative probability exceeds u */
+int32_t ora_sample_cdf(const double *probs, int32_t V, double u);
+/* r = max(0, p - q) normalised to sum 1; returns the mass before normalisation (0: r is set to p) */
+double ora_residual(const double *p, const double *q, int32_t V, double *r);
+
+/* temperature <= 0 switches sampling off (greedy verification, the default).  Call before ora_prefill: the
+ * first token is drawn too (purpose 2 at position n_prompt). */
+void ora_set_sampling(ora_seq *s, double temperature, double top_p, uint64_t seed);
+
+typedef struct {
+    int32_t n_tests;                    /* acceptance tests made: min(n_accept + 1, g) */
+    int32_t from_residual;              /* 1: the round's last token came from the residual distribution */
+    double u_draft[ORA_MAX_GAMMA];      /* uniform numbers used */
+    double u_accept[ORA_MAX_GAMMA];
+    double u_final;
+    double q_x[ORA_MAX_GAMMA];          /* filtered draft probability of each drafted token */
+    double p_x[ORA_MAX_GAMMA];          /* filtered target probability of each tested draft */
+} ora_sample_info;
+/* record of the last round (sampling on) */
+void ora_get_sample_info(const ora_seq *s, ora_sample_info *out);
+/* logits of the last round: which = 0 the exit head's row of draft i (i < g, plus the dropped one when the
+ * loop stopped), which = 1 the target's row i (i <= g); valid until the next round */
+const float *ora_round_logits(const ora_seq *s, int32_t which, int32_t row);
 
 #ifdef __cplusplus
 }
