@@ -12,7 +12,9 @@
  *   Sec. 4.1 (Eq. 1) and Sec. 4.3: pick the next (E, gamma) maximising expected tokens per loaded layer;
  *   Sec. 4.4 and Eq. 3: confidence of a token = its softmax probability; decayed confidence sums over
  *          matched and mismatched shadow tokens give each layer a threshold;
- *   Algorithm 1: the loop, with its confidence break when a sequence is in exit mode (del_set_exit_mode).
+ *   Algorithm 1: the loop, with its confidence break when a sequence is in exit mode (del_set_exit_mode);
+ *   Sec. 2 ("Speculative decoding", general case) with the temperature and top-p of the inference setup:
+ *          speculative sampling for a sequence that asks for it (del_set_sampling).
  *
  * Conventions
  *   - Plain C ABI.  Every pointer is either HOST or DEVICE memory as stated per field/argument.
@@ -183,6 +185,42 @@ int del_set_policy_fs(del_ctx *ctx, int seq, int E, int gamma0);
  * host polls), so a round then has one host round trip per drafted token instead of one per round.  mode 0 (default) drafts exactly gamma tokens.  The
  * confidence statistics and thresholds are maintained in both modes. */
 int del_set_exit_mode(del_ctx *ctx, int seq, int mode);
+
+/* Speculative sampling (Sec. 2) for a sequence slot, with temperature and nucleus (top-p) filtering applied to
+ * the draft and to the target distribution alike.  temperature > 0 switches it on (top_p > 0 then), <= 0 back
+ * to greedy verification (the default).  While it is on:
+ *   - draft i is drawn from softmax(exit-head logits / temperature) restricted to its nucleus and renormalised
+ *     (the nucleus: tokens in order of descending probability, equal ones by ascending id, kept while the mass
+ *     before them is < top_p), by inverse CDF in token-id order;
+ *   - it is accepted when u < min(1, p(x) / q(x)), p and q the filtered target / draft probabilities; the first
+ *     rejected position gets its token from the normalised max(0, p - q); after g acceptances one more token
+ *     comes from the target's filtered row g; the first token of del_prefill is drawn from the target's row of
+ *     the last prompt position;
+ *   - shadow tokens, confidences, statistics and the (E, gamma) selection are unchanged (greedy tokens of
+ *     every layer compared with the last layer's; the valid context is rows 0..n_accept).
+ * The uniform numbers are a function of (seed, absolute position of the token decided, purpose: 0 draft draw,
+ * 1 acceptance test, 2 last token of the round) only: the splitmix64 finaliser applied twice, 53 bits.
+ * The setting belongs to the slot and survives del_prefill / del_release.  Costs one more pass over the LM
+ * head per round (the target's logits are materialised).  Errors: DEL_EINVAL, DEL_ESTATE (a round is half done). */
+int del_set_sampling(del_ctx *ctx, int seq, double temperature, double top_p, uint64_t seed);
+
+/* Record of the last sampled round (synchronises; any pointer may be NULL): acceptance tests made, whether
+ * the last token came from the residual distribution, and the filtered draft / target probability of draft i
+ * (HOST float [32] each; p_x is valid for the tested drafts only). */
+int del_get_sample_info(del_ctx *ctx, int seq, int32_t *n_tests, int32_t *from_residual, float *q_x, float *p_x);
+
+/* Test reader: logits row (HOST float [vocab]) of the last sampled round: which = 0 the exit head's row of
+ * draft `row`, which = 1 the target's row `row` (0..g).  Synchronises. */
+int del_get_round_logits(del_ctx *ctx, int seq, int which, int row, float *out);
+
+/* Test hook: the sampling kernels' device functions on one caller-supplied pair of rows (HOST float [vocab],
+ * vocab <= the model's).  out (HOST int32 [4]): the token drawn from the filtered draft row with u_draft; 1 if
+ * u_accept accepts it; the token the residual distribution gives with u_final; the token the filtered target
+ * row gives with u_final.  prob (HOST double [2]): filtered q(x), p(x).  stat (HOST int32 [8], may be NULL):
+ * per row (draft, target) the key of the smallest kept weight, ties kept, ties present, 0.  Uses sequence 0's
+ * sampling buffers as scratch.  Synchronises. */
+int del_sample_probe(del_ctx *ctx, const float *p_logits, const float *q_logits, int vocab, double temperature, double top_p,
+                     double u_draft, double u_accept, double u_final, int32_t *out, double *prob, int32_t *stat);
 
 /* Confidence statistics (Sec. 4.4).  HOST double [n_layers] each, entry l-1 for layer l: decayed sums of
  * the confidences of matched / mismatched shadow tokens, and the thresholds of Eq. 3 (a mean over no

@@ -28,7 +28,7 @@ EXPORTS = ["del_workspace_bytes", "del_init", "del_prefill", "del_draft", "del_v
            "del_select", "del_round", "del_set_policy", "del_get_stats", "del_set_stats", "del_get_shadow",
            "del_get_drafts", "del_force_token", "del_get_hidden", "del_debug_logits", "del_get_kv", "del_committed_len", "del_release",
            "del_launch_count", "del_get_traffic", "del_set_flags", "del_get_kernel_times", "del_head_argmax_static",
-           "del_set_policy_fs", "del_set_exit_mode", "del_get_conf_stats", "del_set_conf_stats", "del_get_conf", "del_strerror", "del_last_cuda_error", "del_destroy"]
+           "del_set_policy_fs", "del_set_exit_mode", "del_set_sampling", "del_get_sample_info", "del_get_round_logits", "del_sample_probe", "del_get_conf_stats", "del_set_conf_stats", "del_get_conf", "del_strerror", "del_last_cuda_error", "del_destroy"]
 
 
 class Shape(C.Structure):
@@ -100,6 +100,14 @@ def load_library(build_if_missing: bool = True):
     L.del_set_policy_fs.argtypes = [vp, ci, ci, ci]
     L.del_set_exit_mode.restype = ci
     L.del_set_exit_mode.argtypes = [vp, ci, ci]
+    L.del_set_sampling.restype = ci
+    L.del_set_sampling.argtypes = [vp, ci, C.c_double, C.c_double, C.c_uint64]
+    L.del_get_sample_info.restype = ci
+    L.del_get_sample_info.argtypes = [vp, ci, vp, vp, vp, vp]
+    L.del_get_round_logits.restype = ci
+    L.del_get_round_logits.argtypes = [vp, ci, ci, ci, vp]
+    L.del_sample_probe.restype = ci
+    L.del_sample_probe.argtypes = [vp, vp, vp, ci, C.c_double, C.c_double, C.c_double, C.c_double, C.c_double, vp, vp, vp]
     L.del_get_conf_stats.restype = ci
     L.del_get_conf_stats.argtypes = [vp, ci, vp, vp, vp]
     L.del_set_conf_stats.restype = ci
@@ -282,6 +290,33 @@ class DelContext:
     def set_exit_mode(self, seq: int, on: bool):
         """Dynamic draft-exiting: the draft loop stops at the first token whose confidence is below the threshold."""
         self._ck(self.lib.del_set_exit_mode(self._h, seq, 1 if on else 0), "del_set_exit_mode")
+
+    def set_sampling(self, seq: int, temperature: float, top_p: float = 1.0, seed: int = 0):
+        """Speculative sampling with temperature and nucleus filtering for this slot; temperature <= 0: greedy."""
+        self._ck(self.lib.del_set_sampling(self._h, seq, float(temperature), float(top_p), int(seed)), "del_set_sampling")
+
+    def get_sample_info(self, seq: int):
+        """(acceptance tests made, last token from the residual?, q(x) per draft, p(x) per tested draft)."""
+        n, r = C.c_int32(), C.c_int32()
+        qx, px = np.zeros(32, dtype=np.float32), np.zeros(32, dtype=np.float32)
+        self._ck(self.lib.del_get_sample_info(self._h, seq, C.byref(n), C.byref(r), qx.ctypes.data, px.ctypes.data),
+                 "del_get_sample_info")
+        return n.value, bool(r.value), qx, px
+
+    def get_round_logits(self, seq: int, which: int, row: int) -> np.ndarray:
+        out = np.zeros(self.shape.vocab, dtype=np.float32)
+        self._ck(self.lib.del_get_round_logits(self._h, seq, which, row, out.ctypes.data), "del_get_round_logits")
+        return out
+
+    def sample_probe(self, p_logits, q_logits, temperature, top_p, u_draft, u_accept, u_final):
+        """Test hook: the sampling kernels on one pair of logit rows."""
+        p = np.ascontiguousarray(p_logits, dtype=np.float32)
+        q = np.ascontiguousarray(q_logits, dtype=np.float32)
+        out, prob, stat = np.zeros(4, dtype=np.int32), np.zeros(2, dtype=np.float64), np.zeros(8, dtype=np.int32)
+        self._ck(self.lib.del_sample_probe(self._h, p.ctypes.data, q.ctypes.data, p.size, float(temperature), float(top_p),
+                                           float(u_draft), float(u_accept), float(u_final), out.ctypes.data,
+                                           prob.ctypes.data, stat.ctypes.data), "del_sample_probe")
+        return out, prob, stat
 
     def get_conf_stats(self, seq: int):
         L = self.shape.n_layers

@@ -40,6 +40,25 @@ struct SeqState {
     int32_t pad;
 };
 
+// ---- speculative sampling (Sec. 2): per-row description of the filtered distribution and per-sequence results
+#define DEL_SAMPLE_ROWS 32     // logit rows kept per sequence and kind: g_max + 1 <= 32
+
+// Weights are integers W = round(exp((z - m) / T) * 2^40), so that sums do not depend on the order of addition.
+// The nucleus keeps every token whose weight key (the fp32 bit pattern of the weight) is above kstar and the
+// first tie_keep tokens, in token-id order, whose key equals kstar.
+struct RowStat {
+    float m;                     // largest logit of the row
+    uint32_t kstar;
+    int32_t tie_keep, cnt_eq;
+    unsigned long long K;        // mass of the kept tokens
+    unsigned long long Z;        // mass of all tokens
+};
+
+struct SampleOut {
+    int32_t n_accept, last_token, n_tests, from_residual;
+    float q_x[DEL_SAMPLE_ROWS], p_x[DEL_SAMPLE_ROWS];     // filtered draft / target probability of draft i
+};
+
 // Device view of the model shape and of the workspace carve-up (passed by value to kernels).
 struct Dims {
     int32_t L, d, nh, nkv, hd, F, V;
@@ -75,6 +94,9 @@ struct Buffers {
     float *DCONF;                // [B][S+1] confidence of draft i at [1 + i] (indexed like TOK)
     float *SCONF;                // [B][L][S] confidence (top-1 probability) of the shadow tokens
     double *STCS, *SFCS, *TAU;   // [B][L] decayed confidence sums over matched / mismatched shadow tokens, thresholds
+    float *QLOG, *PLOG;          // [B][DEL_SAMPLE_ROWS][V] sampling: logits of the exit head per draft / of the target per row
+    RowStat *QSTAT, *PSTAT;      // [B][DEL_SAMPLE_ROWS]
+    SampleOut *SMP;              // [B]
     int32_t *PROMPT_ALL;         // [max_seq] prompt tokens of the sequence being prefilled
     bf16 *XN;                    // [R_max][d] normalised rows for the batched LM head
     int32_t *SHADOW;             // [B][L][S] shadow tokens

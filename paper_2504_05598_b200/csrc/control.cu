@@ -323,11 +323,13 @@ __global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const __gr
             a.B.TAU[seq * L + l] = threshold(tcs, (double)c, fcs, (double)W);
         }
         if (threadIdx.x == 0) {
+            // first token: the target's greedy token, or (speculative sampling) the one drawn from its row
+            const int32_t first = up->s[u].sampling ? a.B.SMP[seq].last_token : verified[W - 1];
             a.B.ST[seq].Sn = (double)W;
-            tok[0] = verified[W - 1];
+            tok[0] = first;
             o->n_accept = 0;
             o->n_emitted = 1;
-            o->tokens[0] = verified[W - 1];
+            o->tokens[0] = first;
         }
         if (a.do_select) {
             __syncthreads();
@@ -335,13 +337,18 @@ __global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const __gr
         }
         return;
     }
+    const bool samp = up->s[u].sampling != 0;
     if (threadIdx.x == 0) {
+        // greedy: the longest prefix of drafts equal to the target's tokens; speculative sampling: the accept
+        // length and the last token decided by the sampling kernels (Sec. 2)
         int n = 0;
-        while (n < g && tok[1 + n] == verified[n]) ++n;
+        if (samp) n = a.B.SMP[seq].n_accept;
+        else while (n < g && tok[1 + n] == verified[n]) ++n;
         s_n = n;
         o->n_accept = n;
         o->n_emitted = n + 1;
-        for (int i = 0; i <= n; ++i) o->tokens[i] = verified[i];
+        for (int i = 0; i < n; ++i) o->tokens[i] = tok[1 + i];
+        o->tokens[n] = samp ? a.B.SMP[seq].last_token : verified[n];
         a.B.ST[seq].Sn = __dadd_rn(__dmul_rn(a.omega, a.B.ST[seq].Sn), (double)(n + 1));
     }
     __syncthreads();
@@ -366,7 +373,7 @@ __global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const __gr
         a.B.TAU[seq * L + l] = threshold(St, Sc, Sf, Sn_new);
     }
     __syncthreads();
-    if (threadIdx.x == 0) tok[0] = verified[n];      // next round's input token
+    if (threadIdx.x == 0) tok[0] = samp ? a.B.SMP[seq].last_token : verified[n];      // next round's input token
     if (a.do_select) select_body(a, up, out, u);     // (the statistics above are visible after the barrier)
     if (a.post_out != nullptr) {
         // the finished result goes to device-writable host memory, then the stamp that announces it

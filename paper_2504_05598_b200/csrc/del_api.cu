@@ -81,6 +81,8 @@ struct del_ctx {
     volatile uint32_t *post_done = nullptr;
     uint32_t post_seq = 0;
     bool tc_ok = false;
+    // speculative sampling per sequence slot (temperature <= 0: greedy); kept across prefills of the slot
+    struct Sampling { double temperature = 0.0, top_p = 1.0; unsigned long long seed = 0; } samp[DEL_SEQ_MAX];
     int64_t launches = 0, h2d_bytes = 0, d2h_bytes = 0;
     // optional per-launch timing (FLAG_TIMING): events around every launch, summed per kernel class
     struct TimeRec { int cls, ev; double bytes; };
@@ -137,6 +139,11 @@ size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max
     B.STCS = c.take<double>(base, (size_t)D.B * D.L);
     B.SFCS = c.take<double>(base, (size_t)D.B * D.L);
     B.TAU = c.take<double>(base, (size_t)D.B * D.L);
+    B.QLOG = c.take<float>(base, (size_t)D.B * DEL_SAMPLE_ROWS * D.V);
+    B.PLOG = c.take<float>(base, (size_t)D.B * DEL_SAMPLE_ROWS * D.V);
+    B.QSTAT = c.take<RowStat>(base, (size_t)D.B * DEL_SAMPLE_ROWS);
+    B.PSTAT = c.take<RowStat>(base, (size_t)D.B * DEL_SAMPLE_ROWS);
+    B.SMP = c.take<SampleOut>(base, (size_t)D.B);
     B.PROMPT_ALL = c.take<int32_t>(base, (size_t)D.max_seq);
     B.XN = c.take<bf16>(base, (size_t)(R_max + 128) * D.d);
     B.SHADOW = c.take<int32_t>(base, (size_t)D.B * D.L * D.S);
@@ -428,11 +435,23 @@ struct Job { int seq, E, g; int stopped = 0; };
 int plans_needed_draft(const std::vector<Job> &jobs) {
     int gmax = 0;
     for (const Job &j : jobs) gmax = std::max(gmax, j.g);
-    return gmax * ((int)jobs.size() + 1);
+    return gmax * ((int)jobs.size() + 2);
 }
 
 // plans of one draft step: all drafting rows, and per distinct exit layer the rows that go on beyond it
-struct DraftStep { int full_idx = -1; std::vector<int> sub_idx; };
+struct DraftStep { int full_idx = -1; std::vector<int> sub_idx; int samp_idx = -1; };
+
+bool samples(const del_ctx *c, int sq) { return c->samp[sq].temperature > 0.0; }
+
+SampleSeq sample_seq(const del_ctx *c, int sq, int slot, int g, int64_t pos0) {
+    SampleSeq s;
+    memset(&s, 0, sizeof(s));
+    s.seq = sq; s.slot = slot; s.g = g; s.pos0 = pos0;
+    s.inv_T = 1.0 / c->samp[sq].temperature;
+    s.top_p = c->samp[sq].top_p;
+    s.seed = c->samp[sq].seed;
+    return s;
+}
 
 std::vector<int> exit_layers(const std::vector<Job> &jobs) {
     // distinct exit layers, ascending: the rows of a pass thin out as sequences reach their exit
@@ -457,6 +476,11 @@ void plan_draft_step(del_ctx *c, PlanBatch &pb, const std::vector<Job> &act, con
         if (!sub.empty()) fill_plan(c, pb.add(&idx), sub, false);
         st.sub_idx.push_back(idx);
     }
+    // sequences that sample: their drawn token is embedded as the next row by a launch of its own
+    std::vector<RowSpec> smp;
+    for (const Job &j : act)
+        if (samples(c, j.seq)) smp.push_back(RowSpec{j.seq, i + 1, 1});
+    if (!smp.empty()) fill_plan(c, pb.add(&st.samp_idx), smp, false);
 }
 
 // layers 1..E of every drafting row, the exit head in one pass over W_lm, arg-max + confidence, next embedding
@@ -481,6 +505,7 @@ int launch_draft_step(del_ctx *c, const DraftStep &st, const std::vector<int> &E
     a.n_items = c->D.V / 16;
     a.X = c->B.XE;
     a.W0 = c->lm_head;
+    if (st.samp_idx >= 0) a.logits_out = c->B.QLOG;      // the whole row of each draft is kept for the sampling kernels
     TAG(CLS_LMHEAD, 2.0 * c->D.V * c->D.d);
     LAUNCH(launch_rowgemm(EPI_LMHEAD, a, full.m, c->n_sms, c->st, P));
     CtlArgs ca = ctl_base(c, full.plan_idx);
@@ -491,6 +516,21 @@ int launch_draft_step(del_ctx *c, const DraftStep &st, const std::vector<int> &E
         ca.stamp = stamp;
     }
     LAUNCH(launch_draft_finalize_embed(ca, full.m, true, c->st, P));
+    if (st.samp_idx >= 0) {
+        // speculative sampling: the draft is drawn from the filtered exit-head distribution (it replaces the
+        // arg-max token stored above) and embedded as the next row
+        const PassPlan &sp = c->plan_host[st.samp_idx];
+        SampleArgs sa;
+        memset(&sa, 0, sizeof(sa));
+        sa.D = c->D; sa.B = c->B;
+        for (int r = 0; r < sp.m; ++r) {
+            const int sq = sp.rows[r].seq;
+            sa.s[sa.n++] = sample_seq(c, sq, i, 0, c->seq[sq].T);
+        }
+        LAUNCH(launch_sample_draft(sa, c->st, P));
+        CtlArgs ce = ctl_base(c, st.samp_idx);
+        LAUNCH(launch_embed(ce, sp.m, c->st, P));
+    }
     return DEL_OK;
 }
 
@@ -539,7 +579,7 @@ int draft_with_exit(del_ctx *c, std::vector<Job> &jobs) {
         for (size_t k = 0; k < jobs.size(); ++k)
             if (!jobs[k].stopped && i < cap[k]) { act.push_back(jobs[k]); who.push_back(k); }
         if (act.empty()) break;
-        int rc = plan_begin(c, (int)Es.size() + 1);
+        int rc = plan_begin(c, (int)Es.size() + 2);
         if (rc) return rc;
         PlanBatch pb(c);
         DraftStep st;
@@ -693,6 +733,53 @@ int enqueue_verify(del_ctx *c, const std::vector<Job> &jobs) {
     return DEL_OK;
 }
 
+// ---- speculative sampling at the end of a round (Sec. 2): logits of the target's rows (one more pass over
+// W_lm per sampling sequence, on the normalised rows the stacked head already prepared), their filtered
+// distributions, the acceptance tests and the last token.  mode 1 (prefill): only the first token is drawn,
+// from the row of the last prompt position.
+int enqueue_sampling(del_ctx *c, const std::vector<Job> &jobs, const UpdatePlan *up, int mode, int W) {
+    std::vector<int> who;
+    for (size_t u = 0; u < jobs.size(); ++u)
+        if (samples(c, jobs[u].seq)) who.push_back((int)u);
+    if (who.empty()) return DEL_OK;
+    const bool P = pdl(c);
+    int rc = plan_begin(c, (int)who.size());
+    if (rc) return rc;
+    PlanBatch pb(c);
+    std::vector<int> pidx(who.size());
+    for (size_t k = 0; k < who.size(); ++k) {
+        PassPlan *p = pb.add(&pidx[k]);
+        memset(p, 0, sizeof(*p));
+        p->m = mode ? 1 : jobs[who[k]].g + 1;
+    }
+    rc = plan_commit(c, pb);
+    if (rc) return rc;
+    SampleArgs sa;
+    memset(&sa, 0, sizeof(sa));
+    sa.D = c->D; sa.B = c->B;
+    int max_rows = 0;
+    for (size_t k = 0; k < who.size(); ++k) {
+        const Job &j = jobs[who[k]];
+        const int per = mode ? W : j.g + 1, m = mode ? 1 : j.g + 1;
+        const size_t row = (size_t)up->s[who[k]].row0 + (size_t)(c->D.L - 1) * per + (mode ? W - 1 : 0);
+        GemmArgs a = gemm_base(c, pidx[k], 0);
+        a.K = c->D.d;
+        a.n_items = c->D.V / 16;
+        a.X = c->B.XN + row * c->D.d;
+        a.W0 = c->lm_head;
+        a.x_by_row = 1;
+        a.row_scale = c->B.RS + row;
+        a.logits_out = c->B.PLOG + (size_t)j.seq * DEL_SAMPLE_ROWS * c->D.V;
+        TAG(CLS_LMHEAD, 2.0 * c->D.V * c->D.d);
+        LAUNCH(launch_rowgemm(EPI_LMHEAD, a, m, c->n_sms, c->st, P));
+        sa.s[sa.n++] = sample_seq(c, j.seq, 0, mode ? 0 : j.g, mode ? c->seq[j.seq].T - 1 : c->seq[j.seq].T);
+        max_rows = std::max(max_rows, m);
+    }
+    LAUNCH(launch_sample_stats(sa, max_rows, c->st, P));
+    LAUNCH(launch_sample_verify(sa, c->st, P));
+    return DEL_OK;
+}
+
 // ---- stacked LM head + arg-max over all layers' hidden rows (a6), then accept / counts (a7-a8)
 int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bool do_select, uint32_t post_stamp = 0) {
     UpdatePlan *up = &c->up_host[0];
@@ -701,6 +788,7 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
     for (const Job &j : jobs) {
         auto &e = up->s[up->n_seq++];
         e.seq = j.seq; e.row0 = rows; e.g = j.g; e.E = j.E; e.n_valid_init = W;
+        e.sampling = samples(c, j.seq) ? 1 : 0;
         rows += c->D.L * (mode ? W : j.g + 1);
     }
     up->n_rows = rows;
@@ -722,6 +810,8 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
         LAUNCH(launch_lmhead_tc(c->map_x, c->map_w, c->B.TPV, c->B.TPI, c->B.TPS, c->B.RS, rows, c->D.V, c->D.d, c->B.ERR,
                                 c->n_sms, c->st, P));
         LAUNCH(launch_shadow_reduce(ca, up, c->B.TPV, c->B.TPI, c->B.TPS, nvt, 1, nvt, 0, rows, c->st, P));
+        int rs = enqueue_sampling(c, jobs, up, mode, W);
+        if (rs) return rs;
         ca.do_select = do_select;             // the selection runs at the end of the update kernel
         LAUNCH(launch_update(ca, up, c->out_dev, up->n_seq, c->st, P));
         return DEL_OK;
@@ -754,6 +844,8 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
         LAUNCH(launch_shadow_reduce(ca, up, c->B.LPV, c->B.LPI, c->B.LPS, n_part, DEL_ROWS_MAX, 1, k * DEL_ROWS_MAX, m,
                                     c->st, P));
     }
+    rc = enqueue_sampling(c, jobs, up, mode, W);
+    if (rc) return rc;
     ca.do_select = do_select;
     LAUNCH(launch_update(ca, up, c->out_dev, up->n_seq, c->st, P));
     return DEL_OK;
@@ -1187,6 +1279,66 @@ int del_set_stats(del_ctx *c, int sq, const double *Sc, double Sn, int32_t E, in
 int del_set_exit_mode(del_ctx *c, int sq, int mode) {
     if (!seq_ok(c, sq)) return DEL_EINVAL;
     c->seq[sq].exit_mode = mode ? 1 : 0;
+    return DEL_OK;
+}
+
+int del_set_sampling(del_ctx *c, int sq, double temperature, double top_p, uint64_t seed) {
+    if (!seq_ok(c, sq)) return DEL_EINVAL;
+    if (temperature > 0.0 && !(top_p > 0.0)) return DEL_EINVAL;
+    if (c->seq[sq].phase != 0) return DEL_ESTATE;
+    c->samp[sq].temperature = temperature > 0.0 ? temperature : 0.0;
+    c->samp[sq].top_p = top_p;
+    c->samp[sq].seed = seed;
+    return DEL_OK;
+}
+
+int del_get_sample_info(del_ctx *c, int sq, int32_t *n_tests, int32_t *from_residual, float *q_x, float *p_x) {
+    if (!seq_ok(c, sq)) return DEL_EINVAL;
+    SampleOut so;
+    CK(cudaStreamSynchronize(c->st));
+    CK(cudaMemcpy(&so, c->B.SMP + sq, sizeof(so), cudaMemcpyDeviceToHost));
+    if (n_tests) *n_tests = so.n_tests;
+    if (from_residual) *from_residual = so.from_residual;
+    if (q_x) memcpy(q_x, so.q_x, sizeof(so.q_x));
+    if (p_x) memcpy(p_x, so.p_x, sizeof(so.p_x));
+    return DEL_OK;
+}
+
+int del_get_round_logits(del_ctx *c, int sq, int which, int row, float *out) {
+    if (!seq_ok(c, sq) || !out || row < 0 || row >= DEL_SAMPLE_ROWS) return DEL_EINVAL;
+    const float *src = (which ? c->B.PLOG : c->B.QLOG) + ((size_t)sq * DEL_SAMPLE_ROWS + row) * c->D.V;
+    CK(cudaStreamSynchronize(c->st));
+    CK(cudaMemcpy(out, src, sizeof(float) * c->D.V, cudaMemcpyDeviceToHost));
+    return DEL_OK;
+}
+
+int del_sample_probe(del_ctx *c, const float *p_logits, const float *q_logits, int vocab, double temperature, double top_p,
+                     double u_draft, double u_accept, double u_final, int32_t *out, double *prob, int32_t *stat) {
+    if (!c || !p_logits || !q_logits || !out || !prob || vocab < 1 || vocab > c->D.V || !(temperature > 0.0) || !(top_p > 0.0))
+        return DEL_EINVAL;
+    // scratch: the two logit buffers of sequence 0 hold the rows, its statistics slots the results
+    float *zp = c->B.PLOG, *zq = c->B.QLOG;
+    int32_t *o_dev = reinterpret_cast<int32_t *>(c->B.SMP);
+    double *pr_dev = reinterpret_cast<double *>(c->B.PSTAT);
+    RowStat *st_dev = c->B.QSTAT;
+    CK(cudaStreamSynchronize(c->st));
+    CK(cudaMemcpy(zp, p_logits, sizeof(float) * vocab, cudaMemcpyHostToDevice));
+    CK(cudaMemcpy(zq, q_logits, sizeof(float) * vocab, cudaMemcpyHostToDevice));
+    cudaError_t e = launch_sample_probe(zp, zq, vocab, 1.0 / temperature, top_p, u_draft, u_accept, u_final, o_dev, pr_dev, st_dev, c->st);
+    if (e != cudaSuccess) return fail(c, e);
+    CK(cudaStreamSynchronize(c->st));
+    CK(cudaMemcpy(out, o_dev, sizeof(int32_t) * 4, cudaMemcpyDeviceToHost));
+    CK(cudaMemcpy(prob, pr_dev, sizeof(double) * 2, cudaMemcpyDeviceToHost));
+    if (stat) {
+        RowStat rs[2];
+        CK(cudaMemcpy(rs, st_dev, sizeof(rs), cudaMemcpyDeviceToHost));
+        for (int k = 0; k < 2; ++k) {
+            stat[4 * k + 0] = (int32_t)rs[k].kstar;
+            stat[4 * k + 1] = rs[k].tie_keep;
+            stat[4 * k + 2] = rs[k].cnt_eq;
+            stat[4 * k + 3] = 0;
+        }
+    }
     return DEL_OK;
 }
 

@@ -18,6 +18,8 @@ struct GemmArgs {
     int32_t *tile_ctr;         // per-launch zeroed counter for dynamic tile claims (nullptr: static round-robin)
     int32_t x_by_row;          // LMHEAD: activations are X[c] (stacked rows) instead of XE[seq][slot]
     const float *row_scale;    // LMHEAD with x_by_row: log2(e) / rms per row (nullptr: taken from B.SSE)
+    float *logits_out;         // LMHEAD: also store the normalised logits, row c at logits_out[c * V] with x_by_row,
+                               // else at logits_out[(seq * DEL_SAMPLE_ROWS + slot) * V]  (nullptr: not stored)
 };
 
 cudaError_t launch_rowgemm(int epi, const GemmArgs &a, int m, int n_sms, cudaStream_t st, bool pdl);
@@ -68,7 +70,8 @@ struct UpdatePlan {
     struct {
         int32_t seq, row0, g, E;     // rows row0 + (l-1)*(g+1) + i ; E = draft layer of the round
         int32_t n_valid_init;        // prefill: window width W (rows per layer = W)
-        int32_t pad[3];
+        int32_t sampling;            // 1: accept length and last token come from B.SMP (speculative sampling)
+        int32_t pad[2];
     } s[DEL_SEQ_MAX];
 };
 
@@ -82,6 +85,31 @@ cudaError_t launch_update(const CtlArgs &a, const UpdatePlan *up, void *out_dev,
 cudaError_t launch_select(const CtlArgs &a, const UpdatePlan *up, void *out_dev, int n_seq, cudaStream_t st, bool pdl);
 cudaError_t launch_debug_logits(const CtlArgs &a, int layer, int seq, int slot, float *out_dev, cudaStream_t st);
 cudaError_t launch_gather_kv(const CtlArgs &a, int layer, int seq, int pos, float *k_out, float *v_out, cudaStream_t st);
+
+// Speculative sampling (sampling.cu).  One entry per sequence that samples in this launch.
+struct SampleSeq {
+    int32_t seq, slot, g, pad;   // slot: the draft index (draft kernel); g: drafts of the round (verify kernel)
+    int64_t pos0;                // committed positions T: draft i is the token at position T + 1 + i
+    double inv_T, top_p;
+    unsigned long long seed;
+};
+struct SampleArgs {
+    Dims D;
+    Buffers B;
+    int32_t n, pad;
+    SampleSeq s[DEL_SEQ_MAX];
+};
+// draft i of every listed sequence: filtered distribution of its exit-head row, token drawn, stored as draft i
+cudaError_t launch_sample_draft(const SampleArgs &a, cudaStream_t st, bool pdl);
+// filtered-distribution statistics of the target rows 0..g of every listed sequence
+cudaError_t launch_sample_stats(const SampleArgs &a, int max_rows, cudaStream_t st, bool pdl);
+// acceptance tests and the token that ends the round (or, with g = 0 and pos0 = n_prompt - 1, the first token)
+cudaError_t launch_sample_verify(const SampleArgs &a, cudaStream_t st, bool pdl);
+// test hook: one (target, draft) pair of logit rows in device memory -> out[0..2] = drafted token, accepted?, last
+// token; prob[0..1] = filtered q(x), p(x); stat[0..1] = RowStat of q, p
+cudaError_t launch_sample_probe(const float *p_logits, const float *q_logits, int V, double inv_T, double top_p, double u_draft,
+                                double u_accept, double u_final, int32_t *out, double *prob, RowStat *stat, cudaStream_t st);
+int sample_smem_bytes(int V);
 
 // Stacked LM head on tcgen05 / TMEM with fused arg-max (lmhead_tc.cu).  The tensor maps are 128-byte
 // opaque blobs (CUtensorMap) kept by the host context.

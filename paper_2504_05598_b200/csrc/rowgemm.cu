@@ -274,6 +274,11 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
             } else if (EPI == EPI_LMHEAD) {
                 float v = valid ? ra : -INFINITY;      // the row's 1/rms is positive: it cannot change the arg-max
                 int idx = 16 * item + i;
+                if (a.logits_out != nullptr && valid) {
+                    // speculative sampling needs the whole row: normalised logit = raw / rms
+                    const size_t lr = a.x_by_row ? (size_t)c : (size_t)rd.seq * DEL_SAMPLE_ROWS + rd.slot;
+                    a.logits_out[lr * a.D.V + idx] = ra * (rscale[c] * 0.6931471805599453f);
+                }
 #pragma unroll
                 for (int o = 8; o > 0; o >>= 1) {
                     const float v2 = __shfl_xor_sync(0xffffffffu, v, o);

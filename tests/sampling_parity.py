@@ -1,0 +1,222 @@
+"""Round-by-round comparison of the CUDA library with the oracle under speculative sampling (Sec. 2).
+
+Both sides run freely from the same state with the same counter-based uniform numbers.  What is compared:
+
+  * the logits rows the sampling decisions are taken from (exit head per draft, target per row): element-wise
+    within EPS_LOGIT; the largest difference seen in a round, eps, sets that round's decision bands;
+  * every decision (drafted token, accept / reject, last token): identical, or inside the band that logits eps
+    apart allow: each filtered probability then differs by at most a factor exp(4 eps / T) (numerator,
+    normaliser and nucleus mass), so a cumulative probability moves by at most delta = exp(4 eps / T) - 1 and
+    an acceptance ratio by twice that (relative).  A decision inside its band is a tolerated flip: it is
+    counted and the library is put back into the oracle's state (re-prefill on the oracle's tokens);
+  * the filtered probabilities q(x), p(x) the library reports: relative tolerance delta;
+  * shadow tokens (margin rule), match counts, decayed statistics, the next (E, gamma): as in the greedy
+    comparison, bit for bit once the integers agree.
+
+The exact behaviour of the sampling kernels on given rows is pinned separately (same rows on both sides).
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List
+
+import numpy as np
+
+from parity import CONF_RTOL, EPS_LOGIT, MARGIN
+
+
+@dataclass
+class SReport:
+    rounds: int = 0
+    drafts: int = 0
+    tests: int = 0
+    rejections: int = 0
+    flips: int = 0
+    resyncs: int = 0
+    eps_max: float = 0.0
+    prob_max_rel: float = 0.0
+    failures: List[str] = field(default_factory=list)
+
+    def ok(self) -> bool:
+        return not self.failures
+
+
+def _cdf_interval(probs, x):
+    c = np.cumsum(probs)
+    return c[x] - probs[x], c[x]
+
+
+def run_sequence_sampling(ctx, seq, cfg, weights, prompt, temperature, top_p, seed, exit_mode=False, policy=None,
+                          max_rounds=None) -> SReport:
+    import oracle
+    rep = SReport()
+    total = cfg.gen_len
+    o = oracle.OracleSeq(cfg, weights)
+    o.set_sampling(temperature, top_p, seed)
+    o.set_exit_mode(exit_mode)
+    tok, init = o.prefill(prompt)
+    if policy:
+        o.set_policy(*policy)
+    tokens = [tok]
+
+    def sync_library():
+        """Library into the oracle's present state."""
+        ctx.set_sampling(seq, temperature, top_p, seed)
+        ctx.prefill(seq, list(prompt) + tokens[:-1], total - len(tokens) + 1)
+        ctx.force_token(seq, tokens[-1])
+        Sc, Sn, E, g = o.get_stats()
+        Stcs, Sfcs, _ = o.get_conf_stats()
+        ctx.set_conf_stats(seq, Stcs, Sfcs)
+        ctx.set_stats(seq, Sc, Sn, E, g)
+        if policy:
+            ctx.set_policy(seq, *policy)
+        ctx.set_exit_mode(seq, exit_mode)
+
+    # prefill: the first token is drawn from the target's row of the last prompt position
+    ctx.set_sampling(seq, temperature, top_p, seed)
+    first = ctx.prefill(seq, prompt, total)
+    lg_lib, lg_or = ctx.get_round_logits(seq, 1, 0), o.round_logits(1, 0)
+    eps = float(np.abs(lg_lib - lg_or).max())
+    rep.eps_max = max(rep.eps_max, eps)
+    if eps > EPS_LOGIT:
+        rep.failures.append(f"prefill: target logits differ by {eps:.4f}")
+    if first.tokens[0] != tok:
+        delta = float(np.exp(4 * eps / temperature) - 1.0) + 1e-6
+        lo, hi = _cdf_interval(oracle.nucleus(lg_or, temperature, top_p), first.tokens[0])
+        u = oracle.uniform(seed, len(prompt), 2)
+        if not (lo - delta <= u <= hi + delta):
+            rep.failures.append(f"prefill: first token {first.tokens[0]} vs {tok}, u {u:.6f} outside [{lo:.6f}, {hi:.6f}]")
+        rep.flips += 1
+    # (the statistics of the window do not depend on the drawn token; put the library on the oracle's state anyway)
+    sync_library()
+
+    L = cfg.n_layers
+    while len(tokens) < total:
+        if max_rounds is not None and rep.rounds >= max_rounds:
+            break
+        T0 = o.T
+        r = o.round(total - len(tokens))
+        si = o.sample_info()
+        out = ctx.round()[seq]
+        rep.rounds += 1
+        tokens.extend(r.emitted)
+        flip = _compare(ctx, seq, o, r, si, out, T0, temperature, top_p, seed, L, rep)
+        if flip:
+            rep.flips += 1
+        if (flip or rep.failures) and len(tokens) < total:
+            rep.resyncs += 1
+            sync_library()
+        if len(rep.failures) > 10:
+            break
+    o.close()
+    return rep
+
+
+def _compare(ctx, seq, o, r, si, out, T0, T, top_p, seed, L, rep: SReport) -> bool:
+    """Returns True when a tolerated difference makes the rest of the round incomparable."""
+    import oracle
+    what = f"round {rep.rounds}"
+    if (out.E, out.gamma) != (r.E, r.gamma):
+        rep.failures.append(f"{what}: ran with (E,gamma) {(out.E, out.gamma)}, oracle {(r.E, r.gamma)}")
+        return True
+    drafts = ctx.get_drafts(seq)
+    n_tests_lib, from_res_lib, qx_lib, px_lib = ctx.get_sample_info(seq)
+    eps = 0.0
+    rows = min(out.g + int(out.stopped), r.g + int(r.stopped))
+    for i in range(rows):
+        d = float(np.abs(ctx.get_round_logits(seq, 0, i) - o.round_logits(0, i)).max())
+        eps = max(eps, d)
+        if d > EPS_LOGIT:
+            rep.failures.append(f"{what}: exit-head logits of draft {i} differ by {d:.4f}")
+            return True
+        if i >= min(out.g, r.g):
+            break                   # the dropped token of a stopped loop: its row exists, no token was drawn
+        delta = float(np.exp(4 * eps / T) - 1.0) + 1e-6
+        rep.drafts += 1
+        if drafts[i] != r.drafts[i]:
+            qq = oracle.nucleus(o.round_logits(0, i), T, top_p)
+            lo, hi = _cdf_interval(qq, drafts[i])
+            if not (lo - delta <= si.u_draft[i] <= hi + delta):
+                rep.failures.append(f"{what}: draft {i} gpu {drafts[i]} oracle {r.drafts[i]}, u {si.u_draft[i]:.6f} "
+                                    f"outside [{lo:.6f}, {hi:.6f}] +- {delta:.2e}")
+            return True
+        rel = abs(float(qx_lib[i]) - si.q_x[i]) / si.q_x[i]
+        rep.prob_max_rel = max(rep.prob_max_rel, rel)
+        if rel > delta:
+            rep.failures.append(f"{what}: q(x) of draft {i} gpu {qx_lib[i]:.6e} oracle {si.q_x[i]:.6e}")
+    rep.eps_max = max(rep.eps_max, eps)
+    if (out.g, bool(out.stopped)) != (r.g, bool(r.stopped)):
+        # the confidence break fell the other way: allowed only inside the confidence band
+        k = min(out.g, r.g)
+        dc = r.draft_conf[k] if k < len(r.draft_conf) else None
+        if dc is None or abs(dc - r.tau) > CONF_RTOL * (dc + r.tau):
+            rep.failures.append(f"{what}: loop ended at g={out.g} stopped={bool(out.stopped)}, oracle g={r.g} "
+                                f"stopped={r.stopped}")
+        return True
+    for i in range(r.g + 1):
+        d = float(np.abs(ctx.get_round_logits(seq, 1, i) - o.round_logits(1, i)).max())
+        eps = max(eps, d)
+        if d > EPS_LOGIT:
+            rep.failures.append(f"{what}: target logits of row {i} differ by {d:.4f}")
+            return True
+    rep.eps_max = max(rep.eps_max, eps)
+    delta = float(np.exp(4 * eps / T) - 1.0) + 1e-6
+    # acceptance tests in order
+    for i in range(min(n_tests_lib, si.n_tests)):
+        rep.tests += 1
+        if si.p_x[i] > 0:
+            rel = abs(float(px_lib[i]) - si.p_x[i]) / si.p_x[i]
+            rep.prob_max_rel = max(rep.prob_max_rel, rel)
+            if rel > delta:
+                rep.failures.append(f"{what}: p(x) of draft {i} gpu {px_lib[i]:.6e} oracle {si.p_x[i]:.6e}")
+        acc_or, acc_lib = i < r.n_accept, i < out.n_accept
+        if acc_or != acc_lib:
+            ratio = min(1.0, si.p_x[i] / si.q_x[i])
+            if abs(si.u_accept[i] - ratio) > 2 * delta * ratio + 1e-6:
+                rep.failures.append(f"{what}: test {i} gpu {'accept' if acc_lib else 'reject'}, oracle u "
+                                    f"{si.u_accept[i]:.6f} vs ratio {ratio:.6f}")
+            return True
+    rep.rejections += int(si.from_residual)
+    if out.n_accept != r.n_accept or from_res_lib != bool(si.from_residual):
+        rep.failures.append(f"{what}: accepted {out.n_accept} (residual {from_res_lib}), oracle {r.n_accept} "
+                            f"({bool(si.from_residual)})")
+        return True
+    n = r.n_accept
+    if out.emitted()[:n] != r.emitted[:n]:
+        rep.failures.append(f"{what}: emitted {out.emitted()} oracle {r.emitted}")
+        return True
+    if out.emitted()[n] != r.emitted[n]:
+        x = out.emitted()[n]
+        pp = oracle.nucleus(o.round_logits(1, n), T, top_p)
+        if si.from_residual:
+            # a difference of two nearly equal probabilities: its support is all that the bands still fix
+            qq = oracle.nucleus(o.round_logits(0, n), T, top_p)
+            if not pp[x] * (1 + delta) > qq[x] * (1 - delta):
+                rep.failures.append(f"{what}: last token {x} has no residual mass within the band")
+        else:
+            lo, hi = _cdf_interval(pp, x)
+            if not (lo - delta <= si.u_final <= hi + delta):
+                rep.failures.append(f"{what}: last token {x} oracle {r.emitted[n]}, u {si.u_final:.6f} outside "
+                                    f"[{lo:.6f}, {hi:.6f}]")
+        return True
+    # integers agree: shadow tokens by the margin rule, then counts and statistics bit for bit
+    sh, counts = ctx.get_shadow(seq)
+    low = False
+    for l in range(L):
+        for i in range(r.g + 1):
+            if sh[l, i] != r.shadow[l, i]:
+                if r.margin[l, i] > MARGIN:
+                    rep.failures.append(f"{what}: shadow l={l + 1} i={i} gpu {sh[l, i]} oracle {r.shadow[l, i]} margin "
+                                        f"{r.margin[l, i]:.3f}")
+                low = True
+    if low:
+        return True
+    Sc, Sn, E, g = ctx.get_stats(seq)
+    Sc_or, Sn_or, _, _ = o.get_stats()
+    if not np.array_equal(counts, r.counts):
+        rep.failures.append(f"{what}: counts {counts.tolist()} oracle {r.counts.tolist()}")
+    if not (np.array_equal(Sc, Sc_or) and Sn == Sn_or):
+        rep.failures.append(f"{what}: statistics differ (Sn {Sn!r} vs {Sn_or!r})")
+    if (out.next_E, out.next_gamma) != (r.next_E, r.next_gamma):
+        rep.failures.append(f"{what}: next (E,gamma) {(out.next_E, out.next_gamma)} oracle {(r.next_E, r.next_gamma)}")
+    return False

@@ -1,0 +1,250 @@
+"""Speculative sampling (Sec. 2) of the CUDA library against the CPU oracle.  Needs a B200."""
+import json
+import os
+
+import numpy as np
+import pytest
+
+import synth
+from cases import TINY, TINY_GQA
+from parity import ref_from_golden, run_sequence
+from sampling_parity import run_sequence_sampling
+
+pytestmark = pytest.mark.gpu
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def make_ctx(cfg, weights, **kw):
+    import paper_2504_05598_b200 as dl
+    dev = dl.upload_weights(weights)
+    return dl.DelContext(dl.make_shape(cfg, **kw), dev)
+
+
+# ---------------------------------------------------------------- the sampling kernels on given rows
+def _rows(rng, V, kind):
+    """Seeded pairs of logit rows (target, draft) with the structure the method meets."""
+    if kind == "random_model":           # near-uniform: what the synthetic random-weight models produce
+        p = rng.standard_normal(V) * 0.35
+        q = p + rng.standard_normal(V) * 0.05
+    elif kind == "peaked":               # a trained model: a few likely tokens, a long tail
+        p = rng.standard_normal(V) * 2.5
+        p[rng.integers(0, V, 3)] += 9.0
+        q = p + rng.standard_normal(V) * 0.8
+    elif kind == "disagree":             # draft and target prefer different tokens: rejections, residual draws
+        p = rng.standard_normal(V) * 2.0
+        q = rng.standard_normal(V) * 2.0
+    elif kind == "quantised":            # many equal logits: ties inside and at the edge of the nucleus
+        p = np.round(rng.standard_normal(V) * 2.0) * 0.5
+        q = np.round(rng.standard_normal(V) * 2.0) * 0.5
+    elif kind == "plateau":              # three levels: the nucleus ends inside a run of equal weights (id order decides)
+        p = np.zeros(V); p[::7] = 1.0; p[3::13] = -1.0
+        q = np.zeros(V); q[2::5] = 1.0; q[1::11] = -1.0
+    else:
+        raise ValueError(kind)
+    return p.astype(np.float32), q.astype(np.float32)
+
+
+def _margin(probs, x, u):
+    c = np.cumsum(probs)
+    return min(abs(u - (c[x] - probs[x])), abs(u - c[x]))
+
+
+def _nucleus_slack(logits, T, top_p):
+    """Distance of the nucleus decision from its threshold, in probability mass."""
+    import oracle
+    full = oracle.nucleus(logits, T, 1.0)
+    order = np.argsort(-full, kind="stable")
+    before = np.concatenate([[0.0], np.cumsum(full[order])[:-1]])
+    return float(np.abs(before - top_p).min())
+
+
+@pytest.mark.parametrize("V", [1024, 32000, 128256])
+def test_sampling_kernels_against_oracle(V):
+    """Same rows, same uniform numbers on both sides: the drafted token, the acceptance decision, the residual draw
+    and the draw from the target row must be identical, the filtered probabilities equal to 1e-6.  Only a
+    decision that the oracle itself takes within 1e-7 of its boundary may differ."""
+    import oracle
+    cfg = synth.small_variant(TINY, name=f"tiny_v{V}", vocab=V, seed=900 + V % 97)
+    ctx = make_ctx(cfg, synth.make_weights(cfg))
+    rng = np.random.default_rng(V)
+    n_cases = 60 if V <= 32000 else 24
+    kinds = ["random_model", "peaked", "disagree", "quantised", "plateau"]
+    settings = [(0.6, 0.95), (1.0, 0.9), (0.3, 0.5), (1.3, 1.0), (0.6, 0.999)]
+    compared = near = 0
+    for k in range(n_cases):
+        kind = kinds[k % len(kinds)]
+        T, top_p = settings[(k // len(kinds)) % len(settings)]
+        p, q = _rows(rng, V, kind)
+        ud, ua, uf = (oracle.uniform(V, k, j) for j in range(3))
+        out, prob, stat = ctx.sample_probe(p, q, T, top_p, ud, ua, uf)
+        qq, pp = oracle.nucleus(q, T, top_p), oracle.nucleus(p, T, top_p)
+        x = oracle.sample_cdf(qq, ud)
+        slack = min(_nucleus_slack(p, T, top_p), _nucleus_slack(q, T, top_p)) if top_p < 1.0 else 1.0
+        tag = f"case {k} ({kind}, T={T}, top_p={top_p})"
+        if slack < 1e-7:
+            near += 1
+            continue                    # the nucleus itself is a coin flip in the last bits
+        compared += 1
+        if out[0] != x:
+            assert _margin(qq, x, ud) < 1e-7, f"{tag}: draft {out[0]} oracle {x}"
+            near += 1
+            continue
+        assert prob[0] == pytest.approx(qq[x], rel=1e-6), tag
+        assert prob[1] == pytest.approx(pp[x], rel=1e-6, abs=1e-30), tag
+        ratio = min(1.0, pp[x] / qq[x])
+        if bool(out[1]) != (ua < ratio):
+            assert abs(ua - ratio) < 1e-7, f"{tag}: acceptance {out[1]} oracle u {ua} ratio {ratio}"
+            near += 1
+        r, R = oracle.residual(pp, qq)
+        xr = oracle.sample_cdf(r, uf)
+        if out[2] != xr:
+            assert R < 1e-6 or _margin(r, xr, uf) < 1e-7 / max(R, 1e-12), f"{tag}: residual draw {out[2]} oracle {xr} (R={R})"
+            near += 1
+        xb = oracle.sample_cdf(pp, uf)
+        if out[3] != xb:
+            assert _margin(pp, xb, uf) < 1e-7, f"{tag}: target draw {out[3]} oracle {xb}"
+            near += 1
+    print(f"V={V}: {compared} pairs compared, {near} decisions at a boundary")
+    assert compared >= n_cases * 0.8 and near <= max(3, n_cases // 6)
+    ctx.close()
+
+
+def test_sampling_kernel_ties_and_limits():
+    import oracle
+    cfg = TINY
+    ctx = make_ctx(cfg, synth.make_weights(cfg))
+    V = 64
+    flat = np.zeros(V, dtype=np.float32)
+    # 64 equal logits, top_p = 0.5: the 32 lowest ids stay; u walks through them in id order
+    for u in (0.0, 0.26, 0.5, 0.999):
+        out, prob, stat = ctx.sample_probe(flat, flat, 1.0, 0.5, u, 0.5, u)
+        assert out[0] == int(u * 32) and prob[0] == pytest.approx(1 / 32)
+        assert stat[1] == 32 and stat[2] == 64           # ties kept / present
+        assert out[1] == 1                               # p == q: always accepted
+        assert out[3] == int(u * 32)
+    # temperature -> 0: the arg-max, whatever u is
+    rng = np.random.default_rng(1)
+    z = rng.standard_normal(1000).astype(np.float32)
+    for u in (0.0, 0.5, 0.999999):
+        out, prob, _ = ctx.sample_probe(z, z, 1e-4, 0.95, u, 0.5, u)
+        assert out[0] == int(np.argmax(z)) and out[3] == int(np.argmax(z)) and prob[0] == pytest.approx(1.0)
+    # one-hot target against one-hot draft on another token: certain rejection, the residual is the target's token
+    p = np.full(100, -50.0, dtype=np.float32); p[7] = 0.0
+    q = np.full(100, -50.0, dtype=np.float32); q[9] = 0.0
+    out, prob, _ = ctx.sample_probe(p, q, 1.0, 1.0, 0.3, 1e-12, 0.8)
+    assert out[0] == 9 and out[1] == 0 and out[2] == 7
+    # top_p = 1 keeps everything: the draw follows the plain softmax CDF
+    z = rng.standard_normal(500).astype(np.float32)
+    cdf = np.cumsum(oracle.nucleus(z, 0.8, 1.0))
+    for u in (0.1, 0.5, 0.9):
+        out, _, _ = ctx.sample_probe(z, z, 0.8, 1.0, u, 0.5, u)
+        assert out[0] == int(np.searchsorted(cdf, u, side="right"))
+    ctx.close()
+
+
+# ---------------------------------------------------------------- whole rounds
+@pytest.mark.parametrize("cfg", [TINY, TINY_GQA], ids=lambda c: c.name)
+@pytest.mark.parametrize("exit_mode", [False, True], ids=["fixed_gamma", "draft_exiting"])
+def test_speculative_sampling_against_oracle(cfg, exit_mode):
+    w = synth.make_weights(cfg)
+    ctx = make_ctx(cfg, w)
+    prompt = synth.make_prompt(cfg)
+    total = SReportTotal()
+    for seed in (11, 12, 13):
+        policy = None if exit_mode else (cfg.e_min, min(3, cfg.g_max))
+        rep = run_sequence_sampling(ctx, 0, cfg, w, prompt, 0.6, 0.95, seed, exit_mode=exit_mode, policy=policy)
+        print(f"{cfg.name} seed {seed} exit {exit_mode}: rounds {rep.rounds} drafts {rep.drafts} tests {rep.tests} rejections "
+              f"{rep.rejections} flips {rep.flips} resyncs {rep.resyncs} max logit diff {rep.eps_max:.4f} max prob rel diff "
+              f"{rep.prob_max_rel:.2e}")
+        assert rep.ok(), rep.failures[:5]
+        total.add(rep)
+    assert total.rounds >= 10 and total.drafts > 0
+    assert total.flips <= total.rounds // 2          # most rounds agree decision by decision
+    ctx.close()
+
+
+class SReportTotal:
+    def __init__(self):
+        self.rounds = self.drafts = self.flips = 0
+
+    def add(self, rep):
+        self.rounds += rep.rounds
+        self.drafts += rep.drafts
+        self.flips += rep.flips
+
+
+def test_dynamic_selection_with_sampling():
+    """Sampling with the dynamic (E, gamma) selection on the deeper small model."""
+    cfg = TINY_GQA
+    w = synth.make_weights(cfg)
+    ctx = make_ctx(cfg, w)
+    rep = run_sequence_sampling(ctx, 0, cfg, w, synth.make_prompt(cfg), 1.0, 0.9, 5)
+    print(f"dynamic selection: rounds {rep.rounds} flips {rep.flips} rejections {rep.rejections}")
+    assert rep.ok(), rep.failures[:5]
+    ctx.close()
+
+
+@pytest.mark.parametrize("name", ["llama2_7b", "llama32_1b"])
+def test_cold_sampling_reproduces_greedy_trace_full_size(name):
+    """Temperature -> 0 puts all filtered mass on the arg-max: the sampling path (logit rows of exit head and target,
+    nucleus, draws, acceptance ratio, residual) must then reproduce the stored greedy oracle trace of the full-size
+    shape, decision by decision."""
+    path = os.path.join(GOLDEN, f"trace_{name}.json")
+    if not os.path.exists(path):
+        pytest.skip("no stored trace")
+    doc = json.load(open(path))
+    cfg = synth.CONFIGS[name]
+    ctx = make_ctx(cfg, synth.make_weights(cfg))
+    ctx.set_sampling(0, 1e-4, 0.95, 77)
+    ref = ref_from_golden(doc, 0, synth.make_prompt(cfg, 0))
+    rep = run_sequence(ctx, 0, ref, doc["gen_len"], max_rounds=30)
+    print(f"{name} (cold sampling): rounds {rep.rounds} compared {rep.compared} flips {rep.flips} resyncs {rep.resyncs}")
+    assert rep.ok(), rep.failures[:8]
+    ctx.close()
+
+
+def test_sampling_full_size_consistency():
+    """Llama-2-7B shape at temperature 0.6 / top-p 0.95: the reported decisions are consistent with the reported
+    probabilities and the uniform numbers of (seed, position, purpose); tokens are valid ids; sampling with the same
+    seed is reproducible."""
+    import oracle
+    name = "llama2_7b"
+    cfg = synth.CONFIGS[name]
+    ctx = make_ctx(cfg, synth.make_weights(cfg))
+    prompt = synth.make_prompt(cfg, 0)
+    streams = []
+    for attempt in range(2):
+        ctx.set_sampling(0, 0.6, 0.95, 2024)
+        first = ctx.prefill(0, prompt, 48)
+        ctx.set_policy(0, 8, 3)
+        toks, T = [first.tokens[0]], len(prompt)
+        while len(toks) < 48:
+            out = ctx.round()[0]
+            n_tests, from_res, qx, px = ctx.get_sample_info(0)
+            assert 0 <= out.n_accept <= out.g and out.n_emitted == out.n_accept + 1
+            assert n_tests == min(out.n_accept + 1, out.g) and from_res == (out.n_accept < out.g)
+            for i in range(n_tests):
+                u = oracle.uniform(2024, T + 1 + i, 1)
+                ratio = min(1.0, float(px[i]) / float(qx[i]))
+                if abs(u - ratio) > 1e-5:
+                    assert (u < ratio) == (i < out.n_accept), (i, u, ratio)
+            assert all(0 <= t < cfg.vocab for t in out.emitted())
+            toks.extend(out.emitted())
+            T += out.n_emitted
+        streams.append(toks)
+    assert streams[0] == streams[1]
+    ctx.close()
+
+
+def test_sampling_error_codes():
+    import paper_2504_05598_b200 as dl
+    cfg = TINY
+    ctx = make_ctx(cfg, synth.make_weights(cfg))
+    assert ctx.lib.del_set_sampling(ctx._h, -1, 0.6, 0.9, 1) == dl.EINVAL
+    assert ctx.lib.del_set_sampling(ctx._h, 0, 0.6, 0.0, 1) == dl.EINVAL
+    assert ctx.lib.del_set_sampling(ctx._h, 0, 0.0, 0.0, 1) == 0          # off: top_p is not looked at
+    buf = np.zeros(cfg.vocab, dtype=np.float32)
+    assert ctx.lib.del_get_round_logits(ctx._h, 0, 0, 99, buf.ctypes.data) == dl.EINVAL
+    assert ctx.lib.del_sample_probe(ctx._h, buf.ctypes.data, buf.ctypes.data, cfg.vocab + 1, 1.0, 1.0, 0.1, 0.1, 0.1,
+                                    buf.ctypes.data, buf.ctypes.data, None) == dl.EINVAL
+    ctx.close()
