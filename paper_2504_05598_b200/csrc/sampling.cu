@@ -34,7 +34,17 @@ __device__ __forceinline__ uint32_t weight_key(float z, float m, double inv_T) {
     // the argument in double (one rounding to fp32), the exponential in fp32
     return __float_as_uint(expf((float)(((double)z - (double)m) * inv_T)));
 }
-__device__ __forceinline__ u64 key_weight(uint32_t key) { return __float2ull_rn(__uint_as_float(key) * 1099511627776.f); }
+// W = round-to-nearest-even(w * 2^40) for the weight w in [0, 1] whose fp32 bit pattern is `key`, with integer
+// shifts only (a float -> integer conversion per token and pass would keep the conversion unit busy)
+__device__ __forceinline__ u64 key_weight(uint32_t key) {
+    const int sh = (int)(key >> 23) - 127 + 17;              // w = mant * 2^(e - 23), W = mant * 2^(e + 17)
+    const uint32_t mant = (key & 0x7fffffu) | 0x800000u;
+    if (sh >= 0) return (u64)mant << sh;                     // (w <= 1: sh <= 17)
+    const int s = -sh;
+    if (s > 24 || key < 0x00800000u) return 0ull;            // below half a unit (or denormal / zero)
+    const uint32_t q = mant >> s, rem = mant & ((1u << s) - 1u), half = 1u << (s - 1);
+    return (u64)(q + ((rem > half) || (rem == half && (q & 1u))));
+}
 
 struct Smem {
     u64 *hist;            // [NBK][SNT]
@@ -89,16 +99,23 @@ __device__ __forceinline__ T block_excl_scan(T v, T *scratch, T &total) {
     return base + inc - v;
 }
 
+// Index of token i in the shared-memory key cache: one pad word per 32 tokens, so that both the strided
+// passes (consecutive lanes, consecutive tokens) and the chunked passes (lane t at token t * c) spread over
+// the banks.
+__device__ __forceinline__ int kidx(int i) { return i + (i >> 5); }
+
 // Statistics of the filtered distribution of one logit row; every thread returns the same values.
 __device__ RowStat row_stats(const float *z, int V, double inv_T, double top_p, const Smem &sm) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     float mx = -INFINITY;
-    for (int i = tid; i < V; i += SNT) mx = fmaxf(mx, ldg_cg_f32(z + i));
+#pragma unroll 8
+    for (int i = tid; i < V; i += SNT) mx = fmaxf(mx, __ldcg(z + i));
     const float m = block_max(mx, reinterpret_cast<float *>(sm.part));
     u64 zsum = 0;
+#pragma unroll 8
     for (int i = tid; i < V; i += SNT) {
-        const uint32_t key = weight_key(ldg_cg_f32(z + i), m, inv_T);
-        if (sm.keys) sm.keys[i] = key;
+        const uint32_t key = weight_key(__ldcg(z + i), m, inv_T);
+        if (sm.keys) sm.keys[kidx(i)] = key;
         zsum += key_weight(key);
     }
     RowStat r;
@@ -115,14 +132,31 @@ __device__ RowStat row_stats(const float *z, int V, double inv_T, double top_p, 
     for (int s = 28; s >= 0; s -= 4) {
 #pragma unroll
         for (int b = 0; b < NBK; ++b) sm.hist[b * SNT + tid] = 0;
+        const uint32_t hi_shift = s == 28 ? 0 : s + 4;       // (a shift by 32 is not defined: the top pass takes all keys)
+        const uint32_t want = s == 28 ? 0 : prefix;
+        // runs of tokens that fall into the same bucket are summed in a register first (in the upper passes
+        // nearly all candidates share one bucket, and a read-modify-write chain through shared memory is slow)
+        int cb = -1;
+        u64 run = 0;
+#pragma unroll 4
         for (int i = tid; i < V; i += SNT) {
-            const uint32_t key = sm.keys ? sm.keys[i] : weight_key(ldg_cg_f32(z + i), m, inv_T);
-            const bool in = s == 28 || (key >> (s + 4)) == prefix;
-            if (in) sm.hist[((key >> s) & 15u) * SNT + tid] += key_weight(key);
+            const uint32_t key = sm.keys ? sm.keys[kidx(i)] : weight_key(__ldcg(z + i), m, inv_T);
+            const bool in = s == 28 || (key >> hi_shift) == want;
+            if (in) {
+                const int b = (int)((key >> s) & 15u);
+                if (b != cb) {
+                    if (cb >= 0) sm.hist[cb * SNT + tid] += run;
+                    cb = b;
+                    run = 0;
+                }
+                run += key_weight(key);
+            }
         }
+        if (cb >= 0) sm.hist[cb * SNT + tid] += run;
         __syncthreads();
         u64 acc = 0;                         // warp w sums bucket w (SNT / 32 == NBK warps)
-        for (int k = lane; k < SNT; k += 32) acc += sm.hist[warp * SNT + k];
+#pragma unroll
+        for (int k = 0; k < SNT / 32; ++k) acc += sm.hist[warp * SNT + lane + 32 * k];
         acc = warp_sum_u64(acc);
         if (lane == 0) sm.part[warp] = acc;
         __syncthreads();
@@ -140,8 +174,9 @@ __device__ RowStat row_stats(const float *z, int V, double inv_T, double top_p, 
         __syncthreads();
     }
     u64 eq = 0;
+#pragma unroll 4
     for (int i = tid; i < V; i += SNT) {
-        const uint32_t key = sm.keys ? sm.keys[i] : weight_key(ldg_cg_f32(z + i), m, inv_T);
+        const uint32_t key = sm.keys ? sm.keys[kidx(i)] : weight_key(__ldcg(z + i), m, inv_T);
         eq += key == prefix;
     }
     const int cnt_eq = (int)block_sum_u64(eq, sm.part);
@@ -166,6 +201,28 @@ __device__ __forceinline__ void chunk_of(int V, int &i0, int &i1) {
     i1 = min(V, i0 + c);
 }
 
+// f(i, key of token i) over the thread's chunk in token-id order: keys from the shared-memory cache when the
+// row has one (`keys` belongs to this row), else recomputed from 16-byte loads of the logits
+template <typename F>
+__device__ __forceinline__ void for_chunk(const float *z, const uint32_t *keys, int V, float m, double inv_T, F f) {
+    int i0, i1;
+    chunk_of(V, i0, i1);
+    if (keys != nullptr) {
+#pragma unroll 4
+        for (int i = i0; i < i1; ++i) f(i, keys[kidx(i)]);
+        return;
+    }
+    int i = i0;
+#pragma unroll 2
+    for (; i + 4 <= i1; i += 4) {
+        const float4 v = __ldcg(reinterpret_cast<const float4 *>(z + i));
+        const uint32_t k0 = weight_key(v.x, m, inv_T), k1 = weight_key(v.y, m, inv_T), k2 = weight_key(v.z, m, inv_T),
+                       k3 = weight_key(v.w, m, inv_T);
+        f(i, k0); f(i + 1, k1); f(i + 2, k2); f(i + 3, k3);
+    }
+    for (; i < i1; ++i) f(i, weight_key(__ldcg(z + i), m, inv_T));
+}
+
 // kept weight of a token met in token-id order (eq_seen counts the tokens with key == kstar met so far)
 __device__ __forceinline__ u64 kept_weight(uint32_t key, const RowStat &st, int &eq_seen) {
     if (key > st.kstar) return key_weight(key);
@@ -174,11 +231,11 @@ __device__ __forceinline__ u64 kept_weight(uint32_t key, const RowStat &st, int 
 }
 
 // tokens with key == kstar in the chunks of the threads before this one (only needed when some ties are dropped)
-__device__ __forceinline__ int ties_before(const float *z, int V, const RowStat &st, double inv_T, int *scratch) {
+__device__ __forceinline__ int ties_before(const float *z, const uint32_t *keys, int V, const RowStat &st, double inv_T,
+                                           int *scratch) {
     if (st.tie_keep >= st.cnt_eq) return 0;                 // every tie is kept: the rank does not matter
-    int i0, i1, n = 0, total;
-    chunk_of(V, i0, i1);
-    for (int i = i0; i < i1; ++i) n += weight_key(ldg_cg_f32(z + i), st.m, inv_T) == st.kstar;
+    int n = 0, total;
+    for_chunk(z, keys, V, st.m, inv_T, [&](int, uint32_t key) { n += key == st.kstar; });
     return block_excl_scan<int>(n, scratch, total);
 }
 
@@ -194,24 +251,29 @@ __device__ __forceinline__ int block_min_int(int v, int *scratch) {
 }
 
 // Inverse CDF in token-id order over the filtered distribution: the first token whose cumulative kept mass
-// exceeds u * K (the last kept token if rounding leaves none).  Same result in every thread.
-__device__ int pick_token(const float *z, int V, const RowStat &st, double inv_T, double u, const Smem &sm) {
-    int i0, i1;
-    chunk_of(V, i0, i1);
-    const int eq0 = ties_before(z, V, st, inv_T, reinterpret_cast<int *>(sm.part));
+// exceeds u * K (the last kept token if rounding leaves none).  Same result in every thread.  `keys`: the
+// row's key cache in shared memory, or nullptr.
+__device__ int pick_token(const float *z, const uint32_t *keys, int V, const RowStat &st, double inv_T, double u, const Smem &sm) {
+    const int eq0 = ties_before(z, keys, V, st, inv_T, reinterpret_cast<int *>(sm.part));
     int eq = eq0;
     u64 mine = 0;
-    for (int i = i0; i < i1; ++i) mine += kept_weight(weight_key(ldg_cg_f32(z + i), st.m, inv_T), st, eq);
+    for_chunk(z, keys, V, st.m, inv_T, [&](int, uint32_t key) { mine += kept_weight(key, st, eq); });
     u64 total;
     u64 cum = block_excl_scan<u64>(mine, sm.part, total);
     const double tu = u * (double)st.K;
     int cand = 0x7fffffff, last = -1;
-    eq = eq0;
-    for (int i = i0; i < i1; ++i) {
-        const u64 w = kept_weight(weight_key(ldg_cg_f32(z + i), st.m, inv_T), st, eq);
-        cum += w;
-        if (w > 0) last = i;
-        if (w > 0 && (double)cum > tu) { cand = i; break; }
+    // only the thread whose chunk holds the crossing walks it again (integers: the test is exact); if rounding
+    // of u * K leaves no crossing at all, every thread with mass reports its last kept token instead
+    const bool crossing = (double)(cum + mine) > tu && !((double)cum > tu);
+    const bool none = !((double)total > tu);
+    if (crossing || (none && mine > 0)) {
+        eq = eq0;
+        for_chunk(z, keys, V, st.m, inv_T, [&](int i, uint32_t key) {
+            const u64 w = kept_weight(key, st, eq);
+            cum += w;
+            if (w > 0) last = i;
+            if (w > 0 && cand == 0x7fffffff && (double)cum > tu) cand = i;
+        });
     }
     const int first = block_min_int(cand, reinterpret_cast<int *>(sm.part));
     if (first != 0x7fffffff) return first;
@@ -220,11 +282,12 @@ __device__ int pick_token(const float *z, int V, const RowStat &st, double inv_T
 
 // filtered probability of token x; same value in every thread
 __device__ double token_prob(const float *z, int V, int x, const RowStat &st, double inv_T, const Smem &sm) {
-    const uint32_t key = weight_key(ldg_cg_f32(z + x), st.m, inv_T);
+    const uint32_t key = weight_key(__ldcg(z + x), st.m, inv_T);
     if (key < st.kstar) return 0.0;
     if (key == st.kstar && st.tie_keep < st.cnt_eq) {
         u64 n = 0;                           // rank of x among the tied tokens
-        for (int i = threadIdx.x; i < x; i += SNT) n += weight_key(ldg_cg_f32(z + i), st.m, inv_T) == st.kstar;
+#pragma unroll 4
+        for (int i = threadIdx.x; i < x; i += SNT) n += weight_key(__ldcg(z + i), st.m, inv_T) == st.kstar;
         if ((int)block_sum_u64(n, sm.part) >= st.tie_keep) return 0.0;
     }
     return (double)key_weight(key) / (double)st.K;
@@ -235,29 +298,49 @@ __device__ int pick_residual(const float *zp, const float *zq, int V, const RowS
                              const Smem &sm) {
     int i0, i1;
     chunk_of(V, i0, i1);
-    const int ep0 = ties_before(zp, V, sp, inv_T, reinterpret_cast<int *>(sm.part));
-    const int eq0 = ties_before(zq, V, sq, inv_T, reinterpret_cast<int *>(sm.part));
+    const int ep0 = ties_before(zp, nullptr, V, sp, inv_T, reinterpret_cast<int *>(sm.part));
+    const int eq0 = ties_before(zq, nullptr, V, sq, inv_T, reinterpret_cast<int *>(sm.part));
     const double ikp = 1.0 / (double)sp.K, ikq = 1.0 / (double)sq.K;
+    // residual mass of tokens i .. i+3 of the two rows (16-byte loads; the chunks are multiples of 4 tokens, V too)
+    auto quad = [&](int i, int &ep, int &eq, double (&r)[4]) {
+        const float4 a = __ldcg(reinterpret_cast<const float4 *>(zp + i)), b = __ldcg(reinterpret_cast<const float4 *>(zq + i));
+        const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const double p = (double)kept_weight(weight_key(av[j], sp.m, inv_T), sp, ep) * ikp;
+            const double q = (double)kept_weight(weight_key(bv[j], sq.m, inv_T), sq, eq) * ikq;
+            r[j] = p > q ? p - q : 0.0;
+        }
+    };
     int ep = ep0, eq = eq0;
     double mine = 0.0;
-    for (int i = i0; i < i1; ++i) {
-        const double p = (double)kept_weight(weight_key(ldg_cg_f32(zp + i), sp.m, inv_T), sp, ep) * ikp;
-        const double q = (double)kept_weight(weight_key(ldg_cg_f32(zq + i), sq.m, inv_T), sq, eq) * ikq;
-        mine += p > q ? p - q : 0.0;
+#pragma unroll 2
+    for (int i = i0; i < i1; i += 4) {
+        double r[4];
+        quad(i, ep, eq, r);
+        mine += r[0]; mine += r[1]; mine += r[2]; mine += r[3];
     }
     double R;
     double cum = block_excl_scan<double>(mine, reinterpret_cast<double *>(sm.part), R);
-    if (!(R > 0.0)) return pick_token(zp, V, sp, inv_T, u, sm);
+    if (!(R > 0.0)) return pick_token(zp, nullptr, V, sp, inv_T, u, sm);
     const double tu = u * R;
     int cand = 0x7fffffff, last = -1;
-    ep = ep0; eq = eq0;
-    for (int i = i0; i < i1; ++i) {
-        const double p = (double)kept_weight(weight_key(ldg_cg_f32(zp + i), sp.m, inv_T), sp, ep) * ikp;
-        const double q = (double)kept_weight(weight_key(ldg_cg_f32(zq + i), sq.m, inv_T), sq, eq) * ikq;
-        const double r = p > q ? p - q : 0.0;
-        cum += r;
-        if (r > 0.0) last = i;
-        if (r > 0.0 && cum > tu) { cand = i; break; }
+    // the threads whose chunk may hold the crossing walk it again; the band is a little wide because a chunk's
+    // mass added at once and added term by term can differ in the last bits
+    const bool near = cum + mine >= tu * (1.0 - 1e-12) && cum <= tu * (1.0 + 1e-12);
+    const bool none = !(R > tu * (1.0 + 1e-9));
+    if (mine > 0.0 && (near || none)) {
+        ep = ep0; eq = eq0;
+        for (int i = i0; i < i1; i += 4) {
+            double r[4];
+            quad(i, ep, eq, r);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                cum += r[j];
+                if (r[j] > 0.0) last = i + j;
+                if (r[j] > 0.0 && cand == 0x7fffffff && cum > tu) cand = i + j;
+            }
+        }
     }
     const int first = block_min_int(cand, reinterpret_cast<int *>(sm.part));
     if (first != 0x7fffffff) return first;
@@ -268,7 +351,7 @@ __device__ __forceinline__ Smem carve_smem(unsigned char *raw, int V, bool with_
     Smem sm;
     sm.part = reinterpret_cast<u64 *>(raw);                       // 64 words of scratch
     sm.hist = with_hist ? sm.part + 64 : nullptr;
-    sm.keys = with_hist && V <= KEY_CACHE_MAX ? reinterpret_cast<uint32_t *>(sm.hist + NBK * SNT) : nullptr;
+    sm.keys = with_hist && V <= KEY_CACHE_MAX ? reinterpret_cast<uint32_t *>(sm.hist + NBK * SNT) : nullptr;   // [V + V / 32]
     return sm;
 }
 
@@ -288,7 +371,7 @@ __global__ void __launch_bounds__(SNT) sample_draft_kernel(const __grid_constant
     const float *z = logit_row(a.B.QLOG, s.seq, s.slot, V);
     const RowStat st = row_stats(z, V, s.inv_T, s.top_p, sm);
     const double u = uniform01(s.seed, s.pos0 + 1 + s.slot, 0);
-    const int x = pick_token(z, V, st, s.inv_T, u, sm);
+    const int x = pick_token(z, sm.keys, V, st, s.inv_T, u, sm);
     if (threadIdx.x == 0) {
         a.B.QSTAT[s.seq * DEL_SAMPLE_ROWS + s.slot] = st;
         a.B.TOK[s.seq * (a.D.S + 1) + s.slot + 1] = x;
@@ -341,7 +424,7 @@ __global__ void __launch_bounds__(SNT) sample_verify_kernel(const __grid_constan
         const RowStat sq = a.B.QSTAT[s.seq * DEL_SAMPLE_ROWS + n];
         last = pick_residual(logit_row(a.B.PLOG, s.seq, n, V), logit_row(a.B.QLOG, s.seq, n, V), V, sp, sq, s.inv_T, u, sm);
     } else {
-        last = pick_token(logit_row(a.B.PLOG, s.seq, n, V), V, sp, s.inv_T, u, sm);
+        last = pick_token(logit_row(a.B.PLOG, s.seq, n, V), nullptr, V, sp, s.inv_T, u, sm);
     }
     if (threadIdx.x == 0) {
         out->n_accept = n;
@@ -359,13 +442,13 @@ __global__ void __launch_bounds__(SNT) sample_probe_kernel(const float *zp, cons
     const Smem sm = carve_smem(raw, V, true);
     const RowStat sq = row_stats(zq, V, inv_T, top_p, sm);
     const RowStat sp = row_stats(zp, V, inv_T, top_p, sm);
-    const int x = pick_token(zq, V, sq, inv_T, u_draft, sm);
+    const int x = pick_token(zq, nullptr, V, sq, inv_T, u_draft, sm);
     const double qx = token_prob(zq, V, x, sq, inv_T, sm), px = token_prob(zp, V, x, sp, inv_T, sm);
     const double ratio = px / qx;
     const int accepted = u_accept < (ratio < 1.0 ? ratio : 1.0);
     // both endings are reported: the residual draw (as if rejected) and the draw from p (as if all were accepted)
     const int res = pick_residual(zp, zq, V, sp, sq, inv_T, u_final, sm);
-    const int bonus = pick_token(zp, V, sp, inv_T, u_final, sm);
+    const int bonus = pick_token(zp, sm.keys, V, sp, inv_T, u_final, sm);
     if (threadIdx.x == 0) {
         out[0] = x; out[1] = accepted; out[2] = res; out[3] = bonus;
         prob[0] = qx; prob[1] = px;
@@ -393,7 +476,7 @@ cudaError_t launch(void (*kern)(KArgs...), dim3 grid, int smem, cudaStream_t st,
 }  // namespace
 
 int sample_smem_bytes(int V) {
-    return 64 * 8 + NBK * SNT * 8 + (V <= KEY_CACHE_MAX ? V * 4 : 0);
+    return 64 * 8 + NBK * SNT * 8 + (V <= KEY_CACHE_MAX ? (V + V / 32 + 1) * 4 : 0);
 }
 cudaError_t launch_sample_draft(const SampleArgs &a, cudaStream_t st, bool pdl) {
     return launch(sample_draft_kernel, dim3(a.n), sample_smem_bytes(a.D.V), st, pdl, a);

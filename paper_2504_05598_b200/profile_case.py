@@ -1,7 +1,7 @@
 """Small driver for profiling and kernel tuning: a model with the layer shape of a named configuration
 but few layers (so that it fits the size limits of a profiler capture), a short prompt, a few rounds.
 
-    python -m paper_2504_05598_b200.profile_case --config llama2_7b --layers 4 --rounds 8 [--policy E,G]
+    python -m paper_2504_05598_b200.profile_case --config llama2_7b --layers 4 --rounds 8 [--policy E,G] [--sampling T,top_p]
 
 Prints per-kernel-class device times (CUDA events around every launch) as JSON.
 """
@@ -32,6 +32,7 @@ def main():
     ap.add_argument("--no-pdl", action="store_true")
     ap.add_argument("--one-cta", action="store_true")
     ap.add_argument("--no-tc", action="store_true")
+    ap.add_argument("--sampling", default="")        # "T,top_p": speculative sampling instead of greedy verification
     a = ap.parse_args()
     base = synth.CONFIGS[a.config]
     L = a.layers
@@ -40,6 +41,9 @@ def main():
     w = synth.make_weights(cfg)
     ctx = dl.DelContext(dl.make_shape(cfg), dl.upload_weights(w))
     for s in range(cfg.batch):
+        if a.sampling:
+            T, top_p = (float(v) for v in a.sampling.split(","))
+            ctx.set_sampling(s, T, top_p, 1234 + s)
         ctx.prefill(s, synth.make_prompt(cfg, s), cfg.gen_len)
         if a.policy:
             E, G = (int(v) for v in a.policy.split(","))
