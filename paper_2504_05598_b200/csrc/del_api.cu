@@ -1285,6 +1285,7 @@ int del_set_exit_mode(del_ctx *c, int sq, int mode) {
 int del_set_sampling(del_ctx *c, int sq, double temperature, double top_p, uint64_t seed) {
     if (!seq_ok(c, sq)) return DEL_EINVAL;
     if (temperature > 0.0 && !(top_p > 0.0)) return DEL_EINVAL;
+    if (temperature > 0.0 && (c->D.V > sample_max_vocab() || c->D.V % 4 != 0)) return DEL_EINVAL;
     if (c->seq[sq].phase != 0) return DEL_ESTATE;
     c->samp[sq].temperature = temperature > 0.0 ? temperature : 0.0;
     c->samp[sq].top_p = top_p;
@@ -1314,7 +1315,7 @@ int del_get_round_logits(del_ctx *c, int sq, int which, int row, float *out) {
 
 int del_sample_probe(del_ctx *c, const float *p_logits, const float *q_logits, int vocab, double temperature, double top_p,
                      double u_draft, double u_accept, double u_final, int32_t *out, double *prob, int32_t *stat) {
-    if (!c || !p_logits || !q_logits || !out || !prob || vocab < 1 || vocab > c->D.V || !(temperature > 0.0) || !(top_p > 0.0))
+    if (!c || !p_logits || !q_logits || !out || !prob || vocab < 1 || vocab > c->D.V || vocab % 4 != 0 || !(temperature > 0.0) || !(top_p > 0.0))
         return DEL_EINVAL;
     // scratch: the two logit buffers of sequence 0 hold the rows, its statistics slots the results
     float *zp = c->B.PLOG, *zq = c->B.QLOG;

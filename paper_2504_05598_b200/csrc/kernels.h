@@ -109,7 +109,7 @@ cudaError_t launch_sample_verify(const SampleArgs &a, cudaStream_t st, bool pdl)
 // token; prob[0..1] = filtered q(x), p(x); stat[0..1] = RowStat of q, p
 cudaError_t launch_sample_probe(const float *p_logits, const float *q_logits, int V, double inv_T, double top_p, double u_draft,
                                 double u_accept, double u_final, int32_t *out, double *prob, RowStat *stat, cudaStream_t st);
-int sample_smem_bytes(int V);
+int sample_max_vocab();
 
 // Stacked LM head on tcgen05 / TMEM with fused arg-max (lmhead_tc.cu).  The tensor maps are 128-byte
 // opaque blobs (CUtensorMap) kept by the host context.
