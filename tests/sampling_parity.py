@@ -46,70 +46,94 @@ def _cdf_interval(probs, x):
     return c[x] - probs[x], c[x]
 
 
-def run_sequence_sampling(ctx, seq, cfg, weights, prompt, temperature, top_p, seed, exit_mode=False, policy=None,
-                          max_rounds=None) -> SReport:
-    import oracle
-    rep = SReport()
-    total = cfg.gen_len
-    o = oracle.OracleSeq(cfg, weights)
-    o.set_sampling(temperature, top_p, seed)
-    o.set_exit_mode(exit_mode)
-    tok, init = o.prefill(prompt)
-    if policy:
-        o.set_policy(*policy)
-    tokens = [tok]
+class SeqSampler:
+    """One sequence of a context followed round by round: the oracle runs beside the library, every round is
+    compared, and after a tolerated difference the library is put back into the oracle's state.  Several of
+    these (and greedy sequences) can share the context's rounds."""
 
-    def sync_library():
+    def __init__(self, ctx, seq, cfg, weights, prompt, temperature, top_p, seed, exit_mode=False, policy=None):
+        import oracle
+        self.ctx, self.seq, self.cfg, self.prompt = ctx, seq, cfg, prompt
+        self.T, self.top_p, self.seed, self.exit_mode, self.policy = temperature, top_p, seed, exit_mode, policy
+        self.total = cfg.gen_len
+        self.rep = SReport()
+        self.o = oracle.OracleSeq(cfg, weights)
+        self.o.set_sampling(temperature, top_p, seed)
+        self.o.set_exit_mode(exit_mode)
+        tok, _ = self.o.prefill(prompt)
+        if policy:
+            self.o.set_policy(*policy)
+        self.tokens = [tok]
+
+    def sync_library(self):
         """Library into the oracle's present state."""
-        ctx.set_sampling(seq, temperature, top_p, seed)
-        ctx.prefill(seq, list(prompt) + tokens[:-1], total - len(tokens) + 1)
-        ctx.force_token(seq, tokens[-1])
+        ctx, seq, o = self.ctx, self.seq, self.o
+        ctx.set_sampling(seq, self.T, self.top_p, self.seed)
+        ctx.prefill(seq, list(self.prompt) + self.tokens[:-1], self.total - len(self.tokens) + 1)
+        ctx.force_token(seq, self.tokens[-1])
         Sc, Sn, E, g = o.get_stats()
         Stcs, Sfcs, _ = o.get_conf_stats()
         ctx.set_conf_stats(seq, Stcs, Sfcs)
         ctx.set_stats(seq, Sc, Sn, E, g)
-        if policy:
-            ctx.set_policy(seq, *policy)
-        ctx.set_exit_mode(seq, exit_mode)
+        if self.policy:
+            ctx.set_policy(seq, *self.policy)
+        ctx.set_exit_mode(seq, self.exit_mode)
 
-    # prefill: the first token is drawn from the target's row of the last prompt position
-    ctx.set_sampling(seq, temperature, top_p, seed)
-    first = ctx.prefill(seq, prompt, total)
-    lg_lib, lg_or = ctx.get_round_logits(seq, 1, 0), o.round_logits(1, 0)
-    eps = float(np.abs(lg_lib - lg_or).max())
-    rep.eps_max = max(rep.eps_max, eps)
-    if eps > EPS_LOGIT:
-        rep.failures.append(f"prefill: target logits differ by {eps:.4f}")
-    if first.tokens[0] != tok:
-        delta = float(np.exp(4 * eps / temperature) - 1.0) + 1e-6
-        lo, hi = _cdf_interval(oracle.nucleus(lg_or, temperature, top_p), first.tokens[0])
-        u = oracle.uniform(seed, len(prompt), 2)
-        if not (lo - delta <= u <= hi + delta):
-            rep.failures.append(f"prefill: first token {first.tokens[0]} vs {tok}, u {u:.6f} outside [{lo:.6f}, {hi:.6f}]")
-        rep.flips += 1
-    # (the statistics of the window do not depend on the drawn token; put the library on the oracle's state anyway)
-    sync_library()
+    def begin(self):
+        """Prefill: the first token is drawn from the target's row of the last prompt position."""
+        import oracle
+        ctx, seq, o, rep = self.ctx, self.seq, self.o, self.rep
+        ctx.set_sampling(seq, self.T, self.top_p, self.seed)
+        first = ctx.prefill(seq, self.prompt, self.total)
+        lg_lib, lg_or = ctx.get_round_logits(seq, 1, 0), o.round_logits(1, 0)
+        eps = float(np.abs(lg_lib - lg_or).max())
+        rep.eps_max = max(rep.eps_max, eps)
+        if eps > EPS_LOGIT:
+            rep.failures.append(f"prefill: target logits differ by {eps:.4f}")
+        if first.tokens[0] != self.tokens[0]:
+            delta = float(np.exp(4 * eps / self.T) - 1.0) + 1e-6
+            lo, hi = _cdf_interval(oracle.nucleus(lg_or, self.T, self.top_p), first.tokens[0])
+            u = oracle.uniform(self.seed, len(self.prompt), 2)
+            if not (lo - delta <= u <= hi + delta):
+                rep.failures.append(f"prefill: first token {first.tokens[0]} vs {self.tokens[0]}, u {u:.6f} outside "
+                                    f"[{lo:.6f}, {hi:.6f}]")
+            rep.flips += 1
+        # (the statistics of the window do not depend on the drawn token; put the library on the oracle's state anyway)
+        self.sync_library()
 
-    L = cfg.n_layers
-    while len(tokens) < total:
-        if max_rounds is not None and rep.rounds >= max_rounds:
-            break
+    @property
+    def done(self) -> bool:
+        return len(self.tokens) >= self.total or len(self.rep.failures) > 10
+
+    def after_round(self, out):
+        """`out`: this sequence's result of the context's latest round."""
+        o, rep = self.o, self.rep
         T0 = o.T
-        r = o.round(total - len(tokens))
+        r = o.round(self.total - len(self.tokens))
         si = o.sample_info()
-        out = ctx.round()[seq]
         rep.rounds += 1
-        tokens.extend(r.emitted)
-        flip = _compare(ctx, seq, o, r, si, out, T0, temperature, top_p, seed, L, rep)
+        self.tokens.extend(r.emitted)
+        flip = _compare(self.ctx, self.seq, o, r, si, out, T0, self.T, self.top_p, self.seed, self.cfg.n_layers, rep)
         if flip:
             rep.flips += 1
-        if (flip or rep.failures) and len(tokens) < total:
+        if (flip or rep.failures) and len(self.tokens) < self.total:
             rep.resyncs += 1
-            sync_library()
-        if len(rep.failures) > 10:
+            self.sync_library()
+
+    def close(self):
+        self.o.close()
+
+
+def run_sequence_sampling(ctx, seq, cfg, weights, prompt, temperature, top_p, seed, exit_mode=False, policy=None,
+                          max_rounds=None) -> SReport:
+    s = SeqSampler(ctx, seq, cfg, weights, prompt, temperature, top_p, seed, exit_mode, policy)
+    s.begin()
+    while not s.done:
+        if max_rounds is not None and s.rep.rounds >= max_rounds:
             break
-    o.close()
-    return rep
+        s.after_round(ctx.round()[seq])
+    s.close()
+    return s.rep
 
 
 def _compare(ctx, seq, o, r, si, out, T0, T, top_p, seed, L, rep: SReport) -> bool:

@@ -184,6 +184,44 @@ def test_dynamic_selection_with_sampling():
     ctx.close()
 
 
+def test_batch_with_sampled_and_greedy_sequences():
+    """Three sequences share every round: one greedy, one sampling with a fixed policy, one sampling with dynamic
+    draft-exiting; each is compared with its own oracle."""
+    from parity import Report, _resync, compare_init, compare_round, ref_from_oracle
+    from sampling_parity import SeqSampler
+    cfg = synth.small_variant(TINY_GQA, name="tiny_gqa_b3", batch=3, gen_len=32)
+    w = synth.make_weights(cfg)
+    ctx = make_ctx(cfg, w)
+    prompts = [synth.make_prompt(cfg, s) for s in range(3)]
+    ref0 = ref_from_oracle(cfg, w, prompts[0])
+    rep0 = Report()
+    compare_init(ctx, 0, ref0, cfg.gen_len, rep0)
+    s1 = SeqSampler(ctx, 1, cfg, w, prompts[1], 0.6, 0.95, 31, policy=(cfg.e_min, 2))
+    s2 = SeqSampler(ctx, 2, cfg, w, prompts[2], 0.8, 0.9, 32, exit_mode=True)
+    s1.begin()
+    s2.begin()
+    k0, done0 = 0, 1
+    while k0 < len(ref0.rounds) or not s1.done or not s2.done:
+        outs = ctx.round()
+        if k0 < len(ref0.rounds):
+            r = ref0.rounds[k0]
+            need = compare_round(ctx, 0, outs[0], r, rep0)
+            done0 += r.n + 1
+            k0 += 1
+            if need and k0 < len(ref0.rounds):
+                rep0.resyncs += 1
+                _resync(ctx, 0, ref0, done0, r.Sc, r.Sn, r.next_E, r.next_gamma, cfg.gen_len, r.Stcs, r.Sfcs)
+        for s in (s1, s2):
+            if not s.done:
+                s.after_round(outs[s.seq])
+        assert len(rep0.failures) + len(s1.rep.failures) + len(s2.rep.failures) == 0, \
+            (rep0.failures[:3], s1.rep.failures[:3], s2.rep.failures[:3])
+    print(f"greedy: rounds {rep0.rounds} flips {rep0.flips}; sampled: rounds {s1.rep.rounds} flips {s1.rep.flips}; "
+          f"sampled + draft-exiting: rounds {s2.rep.rounds} flips {s2.rep.flips}")
+    assert rep0.rounds == len(ref0.rounds) and s1.rep.rounds >= 5 and s2.rep.rounds >= 5
+    s1.close(); s2.close(); ctx.close()
+
+
 @pytest.mark.parametrize("name", ["llama2_7b", "llama32_1b"])
 def test_cold_sampling_reproduces_greedy_trace_full_size(name):
     """Temperature -> 0 puts all filtered mass on the arg-max: the sampling path (logit rows of exit head and target,
