@@ -298,7 +298,8 @@ def run_ours(a):
                      "hbm_gbs": xbytes / 1e9 / (xms / 1e3), "frac_of_measured_peak": xbytes / 1e9 / (xms / 1e3) / measured_peaks()[0]}
 
     # ---- speculative sampling (Sec. 2; temperature 0.6 and top-p 0.95 of the paper's sampling runs): drafts drawn
-    # from the filtered exit-head distribution, acceptance tests, residual draws; one more pass over W_lm per round
+    # from the filtered exit-head distribution, acceptance tests, residual draws; the logit rows the decisions need
+    # are stored by the LM-head kernels that run anyway (no extra pass over W_lm), so a round's algorithmic bytes stay
     samp_info = None
     if cfg.batch == 1:
         ctx.set_sampling(0, 0.6, 0.95, 20250405)
@@ -316,7 +317,7 @@ def run_ours(a):
         sms = e0.elapsed_time(e1)
         stok, sbytes = 0, 0.0
         for o in souts:
-            sbytes += round_bytes(cfg, [(o.E, o.g, Ts)]) + cfg.lm_head_bytes()
+            sbytes += round_bytes(cfg, [(o.E, o.g, Ts)])
             stok += o.n_emitted
             Ts += o.n_emitted
         ctx.set_sampling(0, 0.0, 1.0, 0)

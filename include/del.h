@@ -200,8 +200,8 @@ int del_set_exit_mode(del_ctx *ctx, int seq, int mode);
  *     every layer compared with the last layer's; the valid context is rows 0..n_accept).
  * The uniform numbers are a function of (seed, absolute position of the token decided, purpose: 0 draft draw,
  * 1 acceptance test, 2 last token of the round) only: the splitmix64 finaliser applied twice, 53 bits.
- * The setting belongs to the slot and survives del_prefill / del_release.  Costs one more pass over the LM
- * head per round (the target's logits are materialised).  Errors: DEL_EINVAL, DEL_ESTATE (a round is half done). */
+ * The setting belongs to the slot and survives del_prefill / del_release.  The logit rows the decisions need
+ * are stored by the LM-head kernels that run anyway.  vocab must be a multiple of 4 and <= 262144.  Errors: DEL_EINVAL, DEL_ESTATE (a round is half done). */
 int del_set_sampling(del_ctx *ctx, int seq, double temperature, double top_p, uint64_t seed);
 
 /* Record of the last sampled round (synchronises; any pointer may be NULL): acceptance tests made, whether

@@ -737,41 +737,54 @@ int enqueue_verify(del_ctx *c, const std::vector<Job> &jobs) {
 // W_lm per sampling sequence, on the normalised rows the stacked head already prepared), their filtered
 // distributions, the acceptance tests and the last token.  mode 1 (prefill): only the first token is drawn,
 // from the row of the last prompt position.
-int enqueue_sampling(del_ctx *c, const std::vector<Job> &jobs, const UpdatePlan *up, int mode, int W) {
+// first stacked row and number of rows of the target (last layer) of sequence u of an update
+void target_rows(const del_ctx *c, const UpdatePlan *up, int u, int g, int mode, int W, size_t &row, int &m) {
+    const int per = mode ? W : g + 1;
+    m = mode ? 1 : g + 1;
+    row = (size_t)up->s[u].row0 + (size_t)(c->D.L - 1) * per + (mode ? W - 1 : 0);
+}
+
+int enqueue_sampling(del_ctx *c, const std::vector<Job> &jobs, const UpdatePlan *up, int mode, int W, bool have_logits) {
     std::vector<int> who;
     for (size_t u = 0; u < jobs.size(); ++u)
         if (samples(c, jobs[u].seq)) who.push_back((int)u);
     if (who.empty()) return DEL_OK;
     const bool P = pdl(c);
-    int rc = plan_begin(c, (int)who.size());
-    if (rc) return rc;
-    PlanBatch pb(c);
-    std::vector<int> pidx(who.size());
-    for (size_t k = 0; k < who.size(); ++k) {
-        PassPlan *p = pb.add(&pidx[k]);
-        memset(p, 0, sizeof(*p));
-        p->m = mode ? 1 : jobs[who[k]].g + 1;
+    std::vector<int> pidx(who.size(), -1);
+    if (!have_logits) {
+        int rc = plan_begin(c, (int)who.size());
+        if (rc) return rc;
+        PlanBatch pb(c);
+        for (size_t k = 0; k < who.size(); ++k) {
+            PassPlan *p = pb.add(&pidx[k]);
+            memset(p, 0, sizeof(*p));
+            p->m = mode ? 1 : jobs[who[k]].g + 1;
+        }
+        rc = plan_commit(c, pb);
+        if (rc) return rc;
     }
-    rc = plan_commit(c, pb);
-    if (rc) return rc;
     SampleArgs sa;
     memset(&sa, 0, sizeof(sa));
     sa.D = c->D; sa.B = c->B;
     int max_rows = 0;
     for (size_t k = 0; k < who.size(); ++k) {
         const Job &j = jobs[who[k]];
-        const int per = mode ? W : j.g + 1, m = mode ? 1 : j.g + 1;
-        const size_t row = (size_t)up->s[who[k]].row0 + (size_t)(c->D.L - 1) * per + (mode ? W - 1 : 0);
-        GemmArgs a = gemm_base(c, pidx[k], 0);
-        a.K = c->D.d;
-        a.n_items = c->D.V / 16;
-        a.X = c->B.XN + row * c->D.d;
-        a.W0 = c->lm_head;
-        a.x_by_row = 1;
-        a.row_scale = c->B.RS + row;
-        a.logits_out = c->B.PLOG + (size_t)j.seq * DEL_SAMPLE_ROWS * c->D.V;
-        TAG(CLS_LMHEAD, 2.0 * c->D.V * c->D.d);
-        LAUNCH(launch_rowgemm(EPI_LMHEAD, a, m, c->n_sms, c->st, P));
+        size_t row;
+        int m;
+        target_rows(c, up, who[k], j.g, mode, W, row, m);
+        if (!have_logits) {
+            // the stacked head did not keep the target's logits (streaming head): one more pass over W_lm
+            GemmArgs a = gemm_base(c, pidx[k], 0);
+            a.K = c->D.d;
+            a.n_items = c->D.V / 16;
+            a.X = c->B.XN + row * c->D.d;
+            a.W0 = c->lm_head;
+            a.x_by_row = 1;
+            a.row_scale = c->B.RS + row;
+            a.logits_out = c->B.PLOG + (size_t)j.seq * DEL_SAMPLE_ROWS * c->D.V;
+            TAG(CLS_LMHEAD, 2.0 * c->D.V * c->D.d);
+            LAUNCH(launch_rowgemm(EPI_LMHEAD, a, m, c->n_sms, c->st, P));
+        }
         sa.s[sa.n++] = sample_seq(c, j.seq, 0, mode ? 0 : j.g, mode ? c->seq[j.seq].T - 1 : c->seq[j.seq].T);
         max_rows = std::max(max_rows, m);
     }
@@ -807,10 +820,20 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
         // one pass over W_lm on the tensor cores, arg-max fused; partials [row][vocabulary tile]
         const int nvt = lmhead_tc_vtiles(c->D.V);
         TAG(CLS_LMSTACK, 2.0 * c->D.V * c->D.d);
+        // sequences that sample: the epilogue also stores the logits of the target's rows
+        LogitSel sel[DEL_SEQ_MAX];
+        int n_sel = 0;
+        for (size_t u = 0; u < jobs.size(); ++u)
+            if (samples(c, jobs[u].seq)) {
+                size_t row;
+                int m;
+                target_rows(c, up, (int)u, jobs[u].g, mode, W, row, m);
+                sel[n_sel++] = LogitSel{(int32_t)row, m, c->B.PLOG + (size_t)jobs[u].seq * DEL_SAMPLE_ROWS * c->D.V};
+            }
         LAUNCH(launch_lmhead_tc(c->map_x, c->map_w, c->B.TPV, c->B.TPI, c->B.TPS, c->B.RS, rows, c->D.V, c->D.d, c->B.ERR,
-                                c->n_sms, c->st, P));
+                                sel, n_sel, c->n_sms, c->st, P));
         LAUNCH(launch_shadow_reduce(ca, up, c->B.TPV, c->B.TPI, c->B.TPS, nvt, 1, nvt, 0, rows, c->st, P));
-        int rs = enqueue_sampling(c, jobs, up, mode, W);
+        int rs = enqueue_sampling(c, jobs, up, mode, W, true);
         if (rs) return rs;
         ca.do_select = do_select;             // the selection runs at the end of the update kernel
         LAUNCH(launch_update(ca, up, c->out_dev, up->n_seq, c->st, P));
@@ -844,7 +867,7 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
         LAUNCH(launch_shadow_reduce(ca, up, c->B.LPV, c->B.LPI, c->B.LPS, n_part, DEL_ROWS_MAX, 1, k * DEL_ROWS_MAX, m,
                                     c->st, P));
     }
-    rc = enqueue_sampling(c, jobs, up, mode, W);
+    rc = enqueue_sampling(c, jobs, up, mode, W, false);
     if (rc) return rc;
     ca.do_select = do_select;
     LAUNCH(launch_update(ca, up, c->out_dev, up->n_seq, c->st, P));

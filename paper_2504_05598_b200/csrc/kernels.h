@@ -115,8 +115,11 @@ int sample_max_vocab();
 // opaque blobs (CUtensorMap) kept by the host context.
 int lmhead_tc_make_map(void *map_out, const void *base, uint64_t rows, uint64_t d, uint32_t box_rows);
 int lmhead_tc_vtiles(int V);
+// sel (may be null): stacked rows [row_lo, row_lo + n) whose normalised logits are also stored, row r at dst[(r - row_lo) * V]
+struct LogitSel { int32_t row_lo, n; float *dst; };
 cudaError_t launch_lmhead_tc(const void *map_x, const void *map_w, float *part_v, int32_t *part_i, float *part_s,
-                             const float *row_scale, int n_rows, int V, int d, int32_t *err, int n_sms, cudaStream_t st, bool pdl);
+                             const float *row_scale, int n_rows, int V, int d, int32_t *err, const LogitSel *sel, int n_sel,
+                             int n_sms, cudaStream_t st, bool pdl);
 
 // Prompt prefill on tcgen05 (prefill_tc.cu): tiled GEMMs over up to PF_ROWS prompt positions of one sequence
 // with the layer's element-wise work fused into the epilogues.  All buffers hold PF_ROWS rows.

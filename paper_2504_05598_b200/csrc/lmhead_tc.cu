@@ -14,6 +14,7 @@
 // Every mbarrier wait is bounded: on expiry the kernel records an error code and winds down (TMEM is
 // always released).
 #include <cuda.h>
+#include <cstring>
 
 #include "kernels.h"
 #include "tc_common.cuh"
@@ -33,6 +34,9 @@ struct TcParams {
     const float *row_scale;      // [rows] log2(e) / rms: the logit behind accumulator v is v / rms
     int32_t n_rows, V, d, n_mtiles, n_vtiles, n_tiles;
     int32_t *err;
+    // speculative sampling: rows whose whole logit row is also stored (the target's rows of each sampling sequence)
+    int32_t n_sel, pad;
+    LogitSel sel[DEL_SEQ_MAX];
 };
 
 // 2^x on the special-function unit (one instruction; the confidence score tolerates its 2-ulp error)
@@ -128,12 +132,32 @@ lmhead_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
             const float k = row < p.n_rows ? p.row_scale[row] : 0.f;
             float best = -INFINITY, esum = 0.f;
             int bidx = 0x7fffffff;
+            float *ldst = nullptr;                           // this thread's row is one whose logits are kept
+            for (int s = 0; s < p.n_sel; ++s) {
+                const int rr = row - p.sel[s].row_lo;
+                if (rr >= 0 && rr < p.sel[s].n) ldst = p.sel[s].dst + (size_t)rr * p.V;
+            }
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
                 tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), r);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 const float before = best;
                 const int nv = min(32, p.V - (v0 + c0));     // columns of this chunk inside the vocabulary (whole chunk: 32)
+                if (ldst != nullptr && nv > 0) {
+                    const float ks = k * 0.6931471805599453f;                  // normalised logit = raw / rms
+                    float *o = ldst + v0 + c0;
+                    if (nv >= 32) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<float4 *>(o + j) =
+                                make_float4(__uint_as_float(r[j]) * ks, __uint_as_float(r[j + 1]) * ks,
+                                            __uint_as_float(r[j + 2]) * ks, __uint_as_float(r[j + 3]) * ks);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j < nv) o[j] = __uint_as_float(r[j]) * ks;
+                    }
+                }
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     const float v = __uint_as_float(r[j]);
@@ -207,8 +231,13 @@ int lmhead_tc_make_map(void *map_out, const void *base, uint64_t rows, uint64_t 
 int lmhead_tc_vtiles(int V) { return (V + BN - 1) / BN; }
 
 cudaError_t launch_lmhead_tc(const void *map_x, const void *map_w, float *part_v, int32_t *part_i, float *part_s,
-                             const float *row_scale, int n_rows, int V, int d, int32_t *err, int n_sms, cudaStream_t st, bool pdl) {
+                             const float *row_scale, int n_rows, int V, int d, int32_t *err, const LogitSel *sel, int n_sel,
+                             int n_sms, cudaStream_t st, bool pdl) {
     TcParams p;
+    memset(&p, 0, sizeof(p));
+    if (n_sel > DEL_SEQ_MAX) return cudaErrorInvalidValue;
+    p.n_sel = sel ? n_sel : 0;
+    for (int s = 0; s < p.n_sel; ++s) p.sel[s] = sel[s];
     p.part_v = part_v; p.part_i = part_i; p.part_s = part_s; p.row_scale = row_scale; p.n_rows = n_rows; p.V = V; p.d = d;
     p.n_mtiles = (n_rows + BM - 1) / BM;
     p.n_vtiles = (V + BN - 1) / BN;
