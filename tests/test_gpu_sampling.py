@@ -222,6 +222,46 @@ def test_batch_with_sampled_and_greedy_sequences():
     s1.close(); s2.close(); ctx.close()
 
 
+@pytest.mark.parametrize("exit_mode", [False, True], ids=["fixed_gamma", "draft_exiting"])
+def test_sampling_step_calls_equal_round_call(exit_mode):
+    """del_draft / del_verify / del_layer_accept / del_select with sampling on give the stream of del_round, and
+    three runs with one seed give one stream (no order-dependent arithmetic anywhere on the path)."""
+    cfg = TINY_GQA
+    ctx = make_ctx(cfg, synth.make_weights(cfg))
+    prompt = synth.make_prompt(cfg)
+    ctx.set_sampling(0, 0.7, 0.9, 99)
+
+    def by_steps():
+        first = ctx.prefill(0, prompt, 30)
+        ctx.set_exit_mode(0, exit_mode)
+        toks, E, g, trace = [first.tokens[0]], first.next_E, first.next_gamma, []
+        while len(toks) < 30:
+            ctx.draft(0, E, cfg.g_max if exit_mode else g)
+            ctx.verify(0)
+            out = ctx.layer_accept(0)
+            E, g = ctx.select(0)
+            toks += out.emitted()
+            trace.append((out.E, out.g, bool(out.stopped), out.n_accept, E, g))
+        return toks, trace
+
+    def by_rounds():
+        first = ctx.prefill(0, prompt, 30)
+        ctx.set_exit_mode(0, exit_mode)
+        toks, trace = [first.tokens[0]], []
+        while len(toks) < 30:
+            out = ctx.round()[0]
+            toks += out.emitted()
+            trace.append((out.E, out.g, bool(out.stopped), out.n_accept, out.next_E, out.next_gamma))
+        return toks, trace
+
+    a, b, c = by_steps(), by_rounds(), by_rounds()
+    assert a == b == c and len(a[0]) == 30
+    assert any(t[3] < t[1] for t in a[1]) or exit_mode           # a rejection happened
+    ctx.set_sampling(0, 0.7, 0.9, 100)                           # another seed: another stream
+    assert by_rounds()[0] != a[0]
+    ctx.close()
+
+
 @pytest.mark.parametrize("name", ["llama2_7b", "llama32_1b"])
 def test_cold_sampling_reproduces_greedy_trace_full_size(name):
     """Temperature -> 0 puts all filtered mass on the arg-max: the sampling path (logit rows of exit head and target,
