@@ -255,3 +255,44 @@ def test_sampled_first_tokens_follow_the_target(case):
         counts[r.emitted[0] % bins] += 1
         o.close()
     assert stats.chisquare(counts, expect * N).pvalue > 1e-3
+
+
+# ---------------------------------------------------------------- properties on arbitrary rows
+from hypothesis import given, settings, strategies as st
+
+
+@settings(max_examples=60, deadline=None)
+@given(st.integers(2, 400), st.floats(0.05, 3.0), st.floats(0.05, 1.0), st.floats(0.05, 8.0), st.integers(0, 2 ** 31))
+def test_nucleus_properties(V, T, top_p, scale, seed):
+    rng = np.random.default_rng(seed)
+    x = (np.round(rng.standard_normal(V) * scale * 4) / 4).astype(np.float32)      # quantised: ties are common
+    p = oracle.nucleus(x, T, top_p)
+    full = sp_softmax(x.astype(np.float64) / T)
+    kept = p > 0
+    assert abs(p.sum() - 1.0) < 1e-12 and kept[np.argmax(x)]
+    assert np.allclose(p[kept] / p[kept].sum(), full[kept] / full[kept].sum(), rtol=1e-12)    # renormalised, not reshaped
+    if (~kept).any():
+        assert full[kept].min() >= full[~kept].max() - 1e-18                        # a top set
+        assert full[kept].sum() >= top_p - 1e-12                                    # that reaches top_p
+        # among equal probabilities at the edge the lower ids stay
+        edge = full[kept].min()
+        tied = np.flatnonzero(np.abs(full - edge) <= 1e-18)
+        flags = kept[tied]
+        assert not (np.diff(flags.astype(int)) > 0).any()
+
+
+@settings(max_examples=40, deadline=None)
+@given(st.integers(2, 200), st.integers(0, 2 ** 31))
+def test_inverse_cdf_is_monotone_and_residual_is_a_distribution(V, seed):
+    rng = np.random.default_rng(seed)
+    p = oracle.nucleus(rng.standard_normal(V).astype(np.float32) * 2, 0.8, 0.9)
+    q = oracle.nucleus(rng.standard_normal(V).astype(np.float32) * 2, 0.8, 0.9)
+    us = np.sort(rng.random(50))
+    toks = [oracle.sample_cdf(p, u) for u in us]
+    assert toks == sorted(toks) and all(p[t] > 0 for t in toks)
+    r, R = oracle.residual(p, q)
+    assert abs(r.sum() - 1.0) < 1e-12 and (r >= 0).all() and 0.0 <= R <= 1.0 + 1e-12
+    if R > 0:
+        assert ((r > 0) <= (p > q)).all()
+    else:
+        assert np.array_equal(r, p)         # nothing can be rejected: defined as p itself
