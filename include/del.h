@@ -92,7 +92,9 @@ typedef struct {
 /* Paged KV cache in DEVICE memory.  The library assigns pages to sequences and writes page_table.
  *   k_pages: bf16 [n_pages][n_layers][n_kv_heads][page_size][head_dim]   (keys after rotary embedding)
  *   v_pages: bf16 [n_pages][n_layers][n_kv_heads][head_dim][page_size]   (values, transposed per page)
- *   page_table: int32 [max_batch][max_seq / page_size] */
+ *   page_table: int32 [max_batch][max_seq / page_size]
+ * The pages must hold finite values when handed over (e.g. zeros): slots of a page that are not written yet are
+ * masked with a probability of exactly 0, and 0 times a NaN bit pattern would still be NaN. */
 typedef struct {
     void *k_pages, *v_pages;
     int32_t *page_table;
@@ -266,7 +268,8 @@ int del_get_traffic(const del_ctx *ctx, int64_t *h2d_bytes, int64_t *d2h_bytes);
 /* Switches of the launch machinery (bit 0: programmatic dependent launch, bit 1: reserved,
  * bit 2: tcgen05 LM head instead of the streaming one, bit 3: record CUDA
  * events around every launch, bit 4: one weight-streaming CTA per SM, bit 5: prefill every prompt
- * position through the decode kernels instead of the tensor-core GEMMs).  Returns the previous flags. */
+ * position through the decode kernels instead of the tensor-core GEMMs, bit 6: the decode attention kernel in
+ * passes of 64 rows instead of the flash-style prefill attention).  Returns the previous flags. */
 int del_set_flags(del_ctx *ctx, int flags);
 
 /* With flag bit 3 set, per kernel class (0 QKV, 1 attention, 2 O-proj, 3 gate/up, 4 down, 5 draft LM

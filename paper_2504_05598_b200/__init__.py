@@ -21,7 +21,7 @@ MAX_GAMMA = 31
 MAX_ROWS = 64
 
 OK, EINVAL, ENOSPC, ESTATE, ETIMEOUT, ECUDA = 0, -1, -2, -3, -4, -5
-FLAG_PDL, FLAG_GRAPH, FLAG_TC, FLAG_TIMING, FLAG_ONECTA, FLAG_NO_BULK_PREFILL = 1, 2, 4, 8, 16, 32
+FLAG_PDL, FLAG_GRAPH, FLAG_TC, FLAG_TIMING, FLAG_ONECTA, FLAG_NO_BULK_PREFILL, FLAG_DECODE_ATTN_PREFILL = 1, 2, 4, 8, 16, 32, 64
 KERNEL_CLASSES = ["qkv_rope", "attention", "o_proj", "gate_up", "down", "lm_head_draft", "lm_head_stacked", "other"]
 
 EXPORTS = ["del_workspace_bytes", "del_init", "del_prefill", "del_draft", "del_verify", "del_layer_accept",
@@ -196,8 +196,9 @@ class DelContext:
             self.rope_cos = torch.from_numpy(cos).to(self.device)
             self.rope_sin = torch.from_numpy(sin).to(self.device)
             page_elems = L * shape.n_kv_heads * 16 * shape.head_dim
-            self.k_pages = torch.empty(shape.n_pages * page_elems, dtype=torch.bfloat16, device=self.device)
-            self.v_pages = torch.empty(shape.n_pages * page_elems, dtype=torch.bfloat16, device=self.device)
+            # zeros: page slots that are not written yet take part in the products with probability 0
+            self.k_pages = torch.zeros(shape.n_pages * page_elems, dtype=torch.bfloat16, device=self.device)
+            self.v_pages = torch.zeros(shape.n_pages * page_elems, dtype=torch.bfloat16, device=self.device)
             self.page_table = torch.zeros(shape.max_batch * (shape.max_seq // 16), dtype=torch.int32, device=self.device)
             ws = self.lib.del_workspace_bytes(C.byref(shape))
             if ws == 0:

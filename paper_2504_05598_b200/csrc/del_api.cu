@@ -15,7 +15,8 @@ namespace {
 
 constexpr int PLAN_RING = 192;
 constexpr int CTR_RING = 4096;
-constexpr int FLAG_PDL = 1, FLAG_GRAPH = 2, FLAG_TC = 4, FLAG_TIMING = 8, FLAG_ONECTA = 16, FLAG_NO_BULK_PREFILL = 32;
+constexpr int FLAG_PDL = 1, FLAG_GRAPH = 2, FLAG_TC = 4, FLAG_TIMING = 8, FLAG_ONECTA = 16, FLAG_NO_BULK_PREFILL = 32,
+              FLAG_DECODE_ATTN_PREFILL = 64;
 enum { CLS_QKV = 0, CLS_ATTN, CLS_OPROJ, CLS_GATEUP, CLS_DOWN, CLS_LMHEAD, CLS_LMSTACK, CLS_OTHER, CLS_N };
 
 struct SeqHost {
@@ -649,6 +650,16 @@ int prefill_bulk(del_ctx *c, int sq, int n_pos, int win0) {
             a.n_ntiles = prefill_tc_ntiles(PF_QKV, D);
             LAUNCH(launch_prefill_gemm(PF_QKV, c->pf_xs.b, c->pf_wq[l - 1].b, c->pf_wk[l - 1].b, c->pf_wv[l - 1].b, a, c->n_sms, c->st, P));
             if (l == D.L && !has_window) break;       // of the last layer only the keys and values are needed
+            if (!(c->flags & FLAG_DECODE_ATTN_PREFILL)) {
+                // one flash-style pass over the chunk's rows and all keys up to each row's position
+                PfAttnArgs pa;
+                memset(&pa, 0, sizeof(pa));
+                pa.D = D;
+                pa.Q = a.Q; pa.ATT = a.ATT;
+                pa.KP = c->B.KP; pa.VP = c->B.VP; pa.PT = c->B.PT;
+                pa.M = a.M; pa.layer = l; pa.seq = sq; pa.pos0 = p0;
+                LAUNCH(launch_prefill_attention(pa, c->st, P));
+            } else
             for (int r0 = 0; r0 < a.M; r0 += DEL_ROWS_MAX) {
                 AttnArgs at;
                 memset(&at, 0, sizeof(at));

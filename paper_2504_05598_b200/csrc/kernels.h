@@ -149,6 +149,18 @@ struct PfArgs {
     int32_t win0;
 };
 int prefill_tc_ntiles(int epi, const Dims &D);
+
+// Causal attention of a prefill chunk (prefill_attn.cu): rows 0..M-1 of Q (positions pos0 + row of sequence seq)
+// against the paged cache of `layer` (which already holds the chunk's own keys and values) -> ATT.
+struct PfAttnArgs {
+    Dims D;
+    const bf16 *Q;             // [M][nh * hd]
+    bf16 *ATT;                 // [M][nh * hd]
+    const bf16 *KP, *VP;
+    const int32_t *PT;
+    int32_t M, layer, seq, pos0;
+};
+cudaError_t launch_prefill_attention(const PfAttnArgs &a, cudaStream_t st, bool pdl);
 cudaError_t launch_prefill_gemm(int epi, const void *map_a, const void *map_b0, const void *map_b1, const void *map_b2,
                                 const PfArgs &p, int n_sms, cudaStream_t st, bool pdl);
 cudaError_t launch_prefill_embed(const PfArgs &p, const bf16 *tok_emb, const int32_t *prompt, const bf16 *gain0, cudaStream_t st);

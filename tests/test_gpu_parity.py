@@ -71,7 +71,8 @@ def test_tensor_core_prefill_against_oracle(cfg):
     o.prefill(prompt)
     P, W = len(prompt), min(cfg.init_window, len(prompt))
     ref = ref_from_oracle(cfg, w, prompt)
-    for flags in (dl.FLAG_PDL | dl.FLAG_TC, dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_NO_BULK_PREFILL):
+    for flags in (dl.FLAG_PDL | dl.FLAG_TC, dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_DECODE_ATTN_PREFILL,
+                  dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_NO_BULK_PREFILL):
         ctx.set_flags(flags)
         launches0 = ctx.launch_count()
         ctx.prefill(0, prompt, cfg.gen_len)
