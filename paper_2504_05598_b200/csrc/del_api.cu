@@ -159,7 +159,7 @@ size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max
     // chunk buffers of the bulk prefill (PF_ROWS prompt positions)
     PfArgs pfa;
     memset(&pfa, 0, sizeof(pfa));
-    pfa.n_ssp = prefill_tc_ntiles(PF_DOWN, D);
+    pfa.n_ssp = prefill_tc_nssp(D);
     pfa.H = c.take<float>(base, (size_t)PF_ROWS * D.d);
     pfa.XS = c.take<bf16>(base, (size_t)PF_ROWS * D.d);
     pfa.SSP = c.take<float>(base, (size_t)PF_ROWS * pfa.n_ssp);
@@ -1027,10 +1027,12 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
         maps(c->pf_wq, c->wq, qd, d, 256);
         maps(c->pf_wk, c->wk, kvd, d, 256);
         maps(c->pf_wv, c->wv, kvd, d, 256);
-        maps(c->pf_wo, c->wo, d, qd, 128);
+        const uint32_t bn_narrow = (uint32_t)prefill_tc_narrow(c->D);
+        maps(c->pf_wo, c->wo, d, qd, bn_narrow);
         maps(c->pf_wg, c->w_gate, F, d, 128);
         maps(c->pf_wu, c->w_up, F, d, 128);
-        maps(c->pf_wd, c->w_down, d, F, 128);
+        maps(c->pf_wd, c->w_down, d, F, bn_narrow);
+        c->pf.bn_narrow = (int32_t)bn_narrow;
         c->pf_ok = ok;
         c->pf.D = c->D;
         c->pf.KP = c->B.KP; c->pf.VP = c->B.VP; c->pf.PT = c->B.PT;

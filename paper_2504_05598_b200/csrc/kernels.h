@@ -147,8 +147,11 @@ struct PfArgs {
     // after every layer is also stored in the hidden stack (slot = position - win0)
     float *stackH;
     int32_t win0;
+    int32_t bn_narrow;         // tile width of O-proj and down (prefill_tc_narrow)
 };
 int prefill_tc_ntiles(int epi, const Dims &D);
+int prefill_tc_narrow(const Dims &D);          // tile width of O-proj and down for this shape
+int prefill_tc_nssp(const Dims &D);            // partial sums of squares per row (one per 128 columns)
 
 // Causal attention of a prefill chunk (prefill_attn.cu): rows 0..M-1 of Q (positions pos0 + row of sequence seq)
 // against the paged cache of `layer` (which already holds the chunk's own keys and values) -> ATT.

@@ -30,8 +30,10 @@ using namespace tc;
 constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int PF_THREADS = 192;
-constexpr int BN_NARROW = 128;     // tile width of O-proj and down (N = d_model)
-template <int EPI> __host__ __device__ constexpr int tile_n() { return (EPI == PF_OPROJ || EPI == PF_DOWN) ? BN_NARROW : BN; }
+// O-proj and down (N = d_model) use a narrower tile, p.bn_narrow, chosen per model shape (prefill_tc_narrow)
+template <int EPI> __device__ __forceinline__ int tile_n(const PfArgs &p) {
+    return (EPI == PF_OPROJ || EPI == PF_DOWN) ? p.bn_narrow : BN;
+}
 
 struct PfMaps {
     CUtensorMap a;             // activations [PF_ROWS, K], box 64 x 128
@@ -139,11 +141,11 @@ __device__ __forceinline__ void epilogue(const PfArgs &p, uint32_t taddr, int ro
     } else {   // PF_OPROJ, PF_DOWN: residual update in place, next norm input, sums of squares of the new h
         float ss = 0.f;
         bf16 *xo = EPI == PF_OPROJ ? p.XM : p.XS;
-        for (int c0 = 0; c0 < BN_NARROW; c0 += 32) {
+        for (int c0 = 0; c0 < p.bn_narrow; c0 += 32) {
             __syncwarp();
             tmem_ld32(taddr + (uint32_t)c0, r0);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            const int n = nt * BN_NARROW + c0;
+            const int n = nt * p.bn_narrow + c0;
             if (!live || n >= D.d) continue;                     // d is a multiple of 32
             float *hp = p.H + (size_t)row * D.d + n;
             float h[32];
@@ -169,8 +171,12 @@ __device__ __forceinline__ void epilogue(const PfArgs &p, uint32_t taddr, int ro
                 x[e] = p.gain ? h[e] * bf16_to_f(p.gain[n + e]) : 0.f;
             }
             if (p.gain) store_bf16x32(xo + (size_t)row * D.d + n, x);
+            // one partial sum of squares per 128 columns, whatever the tile width: results do not depend on it
+            if ((c0 & 127) == 96 || n + 32 >= D.d) {
+                (EPI == PF_OPROJ ? p.SSPM : p.SSP)[(size_t)row * p.n_ssp + (n >> 7)] = ss;
+                ss = 0.f;
+            }
         }
-        if (live) (EPI == PF_OPROJ ? p.SSPM : p.SSP)[(size_t)row * p.n_ssp + nt] = ss;
     }
 }
 
@@ -217,7 +223,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1) prefill_gemm_kernel(const __gri
                 for (int kb = 0; kb < n_kb; ++kb, ++it) {
                     const int s = it % STAGES;
                     if (!mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1)) { s_err = 1; break; }
-                    mbar_expect_tx(&full_bar[s], A_BYTES + tile_n<EPI>() * BK * 2);
+                    mbar_expect_tx(&full_bar[s], A_BYTES + tile_n<EPI>(p) * BK * 2);
                     unsigned char *sa = tiles + (size_t)s * STAGE_BYTES;
                     tma_load_2d(sa, &maps.a, kb * BK, mt * BM, &full_bar[s]);
                     if (EPI == PF_QKV) {
@@ -229,7 +235,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1) prefill_gemm_kernel(const __gri
                         tma_load_2d(sa + A_BYTES, &maps.b0, kb * BK, nt * (BN / 2), &full_bar[s]);
                         tma_load_2d(sa + A_BYTES + B_BYTES / 2, &maps.b1, kb * BK, nt * (BN / 2), &full_bar[s]);
                     } else {
-                        tma_load_2d(sa + A_BYTES, &maps.b0, kb * BK, nt * tile_n<EPI>(), &full_bar[s]);
+                        tma_load_2d(sa + A_BYTES, &maps.b0, kb * BK, nt * tile_n<EPI>(p), &full_bar[s]);
                     }
                 }
             }
@@ -238,7 +244,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1) prefill_gemm_kernel(const __gri
         if (lane == 0) {
             // instruction descriptor: fp32 accumulate, bf16 x bf16, both operands K-major, N = tile width, M = 128
             const uint32_t idesc =
-                (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(tile_n<EPI>() >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(tile_n<EPI>(p) >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
             int it = 0;
             for (int i = 0; i < my_tiles && !s_err; ++i) {
                 const int buf = i & 1;
@@ -341,8 +347,26 @@ int prefill_tc_ntiles(int epi, const Dims &D) {
     switch (epi) {
         case PF_QKV: return (D.nh * D.hd + BN - 1) / BN + 2 * ((D.nkv * D.hd + BN - 1) / BN);
         case PF_GATEUP: return (D.F + BN / 2 - 1) / (BN / 2);
-        default: return (D.d + BN_NARROW - 1) / BN_NARROW;
+        default: { const int bn = prefill_tc_narrow(D); return (D.d + bn - 1) / bn; }
     }
+}
+int prefill_tc_nssp(const Dims &D) { return (D.d + 127) / 128; }
+
+// Tile width of the two GEMMs whose N is d_model: 128 or 256 (whole 128-column groups of the per-row sums of
+// squares, so that no result depends on the choice).  A k-block of a 128 x bn tile costs its operand loads,
+// (128 + bn) rows of 128 bytes at what one SM can pull from L2, more than its MMAs (measured: tensor pipe 40-68 %
+// active), so a tile takes about (128 + bn) units; the width that minimises waves x (128 + bn) for a full chunk
+// of PF_ROWS rows on 148 SMs wins: 128 at d = 4096 (128 tiles, one wave), 256 at d = 5120 (80 tiles in one wave
+// instead of 160 in two: the 3072-position prefill of that shape 138 -> 127 ms).
+int prefill_tc_narrow(const Dims &D) {
+    int best = 128;
+    long best_cost = -1;
+    for (int bn = 128; bn <= 256; bn += 128) {
+        const long tiles = (long)(PF_ROWS / BM) * ((D.d + bn - 1) / bn);
+        const long cost = ((tiles + 147) / 148) * (128 + bn);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
+    }
+    return best;
 }
 
 // map_a / map_b*: 128-byte CUtensorMap blobs made by lmhead_tc_make_map (boxes of 256 rows for Wq / Wk / Wv, of
