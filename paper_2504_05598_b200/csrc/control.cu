@@ -151,10 +151,11 @@ __device__ __forceinline__ bool locate_row(const UpdatePlan *up, int L, int mode
     for (int u = 0; u < up->n_seq; ++u) {
         const int per = mode ? up->s[u].n_valid_init : up->s[u].g + 1;
         const int r = rr - up->s[u].row0;
-        if (r >= 0 && r < per * L) {
+        if (r >= 0 && r < per * up->lay_n) {
             seq = up->s[u].seq;
-            layer = r / per + 1;
-            slot = r - (layer - 1) * per;
+            const int j = r / per;
+            layer = plan_layer(up, L, j);
+            slot = r - j * per;
             return true;
         }
     }
@@ -307,7 +308,8 @@ __global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const __gr
     del_round_out *o = out + seq;
     if (a.mode == 1) {
         const int W = up->s[u].n_valid_init;
-        for (int l = threadIdx.x; l < L; l += blockDim.x) {
+        for (int j = threadIdx.x; j < up->lay_n; j += blockDim.x) {
+            const int l = plan_layer(up, L, j) - 1;
             int c = 0;
             double tcs = 0.0, fcs = 0.0;
             for (int j = 0; j < W; ++j) {
@@ -354,7 +356,8 @@ __global__ void __launch_bounds__(128) update_kernel(const CtlArgs a, const __gr
     __syncthreads();
     const int n = s_n;
     const double Sn_new = a.B.ST[seq].Sn;            // written by thread 0 before the barrier
-    for (int l = threadIdx.x; l < L; l += blockDim.x) {
+    for (int j = threadIdx.x; j < up->lay_n; j += blockDim.x) {
+        const int l = plan_layer(up, L, j) - 1;      // (trimmed: the statistics of the other layers are left alone)
         int c = 0;
         double tcs = 0.0, fcs = 0.0;                 // confidence sums over matched / mismatched shadow tokens (Sec. 4.4)
         for (int i = 0; i <= n; ++i) {

@@ -16,7 +16,7 @@ namespace {
 constexpr int PLAN_RING = 192;
 constexpr int CTR_RING = 4096;
 constexpr int FLAG_PDL = 1, FLAG_GRAPH = 2, FLAG_TC = 4, FLAG_TIMING = 8, FLAG_ONECTA = 16, FLAG_NO_BULK_PREFILL = 32,
-              FLAG_DECODE_ATTN_PREFILL = 64;
+              FLAG_DECODE_ATTN_PREFILL = 64, FLAG_TRIM_ROWS = 128;
 enum { CLS_QKV = 0, CLS_ATTN, CLS_OPROJ, CLS_GATEUP, CLS_DOWN, CLS_LMHEAD, CLS_LMSTACK, CLS_OTHER, CLS_N };
 
 struct SeqHost {
@@ -752,7 +752,8 @@ int enqueue_verify(del_ctx *c, const std::vector<Job> &jobs) {
 void target_rows(const del_ctx *c, const UpdatePlan *up, int u, int g, int mode, int W, size_t &row, int &m) {
     const int per = mode ? W : g + 1;
     m = mode ? 1 : g + 1;
-    row = (size_t)up->s[u].row0 + (size_t)(c->D.L - 1) * per + (mode ? W - 1 : 0);
+    (void)c;
+    row = (size_t)up->s[u].row0 + (size_t)(up->lay_n - 1) * per + (mode ? W - 1 : 0);
 }
 
 int enqueue_sampling(del_ctx *c, const std::vector<Job> &jobs, const UpdatePlan *up, int mode, int W, bool have_logits) {
@@ -808,12 +809,16 @@ int enqueue_sampling(del_ctx *c, const std::vector<Job> &jobs, const UpdatePlan 
 int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bool do_select, uint32_t post_stamp = 0) {
     UpdatePlan *up = &c->up_host[0];
     memset(up, 0, sizeof(*up));
+    // rows of the stacked head: every layer, or only the layers the selection can pick plus the last one
+    const bool trim = (c->flags & FLAG_TRIM_ROWS) != 0;
+    up->lay_first = trim ? c->sh.e_min : 1;
+    up->lay_n = trim ? c->sh.e_max - c->sh.e_min + 2 : c->D.L;
     int rows = 0;
     for (const Job &j : jobs) {
         auto &e = up->s[up->n_seq++];
         e.seq = j.seq; e.row0 = rows; e.g = j.g; e.E = j.E; e.n_valid_init = W;
         e.sampling = samples(c, j.seq) ? 1 : 0;
-        rows += c->D.L * (mode ? W : j.g + 1);
+        rows += up->lay_n * (mode ? W : j.g + 1);
     }
     up->n_rows = rows;
     if (rows > c->R_max) return DEL_EINVAL;

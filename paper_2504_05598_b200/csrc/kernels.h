@@ -66,7 +66,10 @@ struct CtlArgs {
 // rows of the stacked LM head: (seq, layer, slot) per row, plus per-sequence bookkeeping of the update.
 // The launchers below take a HOST pointer and pass the plan by value in the kernel parameters.
 struct UpdatePlan {
-    int32_t n_seq, n_rows, pad0, pad1;
+    int32_t n_seq, n_rows;
+    // layers whose hidden rows go through the stacked LM head: all L, or (trimmed) only the candidates of the
+    // selection e_min..e_max plus the last layer; lay_n of them, layer of index j = j < lay_n - 1 ? lay_first + j : L
+    int32_t lay_first, lay_n;
     struct {
         int32_t seq, row0, g, E;     // rows row0 + (l-1)*(g+1) + i ; E = draft layer of the round
         int32_t n_valid_init;        // prefill: window width W (rows per layer = W)
@@ -74,6 +77,9 @@ struct UpdatePlan {
         int32_t pad[2];
     } s[DEL_SEQ_MAX];
 };
+
+// 1-based layer of stacked-layer index j
+__host__ __device__ inline int plan_layer(const UpdatePlan *up, int L, int j) { return j < up->lay_n - 1 ? up->lay_first + j : L; }
 
 cudaError_t launch_embed(const CtlArgs &a, int m, cudaStream_t st, bool pdl);
 cudaError_t launch_draft_finalize_embed(const CtlArgs &a, int m, bool embed_next, cudaStream_t st, bool pdl);

@@ -32,6 +32,7 @@ def main():
     ap.add_argument("--no-pdl", action="store_true")
     ap.add_argument("--one-cta", action="store_true")
     ap.add_argument("--no-tc", action="store_true")
+    ap.add_argument("--trim", action="store_true")   # stacked LM head over the candidate layers only
     ap.add_argument("--sampling", default="")        # "T,top_p": speculative sampling instead of greedy verification
     a = ap.parse_args()
     base = synth.CONFIGS[a.config]
@@ -48,7 +49,8 @@ def main():
         if a.policy:
             E, G = (int(v) for v in a.policy.split(","))
             ctx.set_policy(s, E, G)
-    flags = (0 if a.no_pdl else dl.FLAG_PDL) | (16 if a.one_cta else 0) | (0 if a.no_tc else dl.FLAG_TC)
+    flags = (0 if a.no_pdl else dl.FLAG_PDL) | (16 if a.one_cta else 0) | (0 if a.no_tc else dl.FLAG_TC) | \
+        (dl.FLAG_TRIM_ROWS if a.trim else 0)
     ctx.set_flags(flags)
     ctx.round()
     ctx.round()

@@ -163,17 +163,19 @@ def _compare_conf(rep: Report, what: str, got, want):
             rep.failures.append(f"{what}: element {k} gpu {got.flat[k]:.6f} oracle {want.flat[k]:.6f}")
 
 
-def compare_init(ctx, seq, ref: SeqRef, total_tokens: int, rep: Report, policy=None) -> None:
+def compare_init(ctx, seq, ref: SeqRef, total_tokens: int, rep: Report, policy=None, layers=None) -> None:
+    """layers: 0-based layers to compare (default all; with trimmed stacked-head rows only those are maintained)."""
     out = ctx.prefill(seq, ref.prompt, total_tokens)
     if policy:
         ctx.set_policy(seq, *policy)
     L, W = ref.init_shadow.shape
+    layers = list(range(L)) if layers is None else list(layers)
     # after the prefill the shadow buffer holds the window's tokens in its first W columns; only g_max+1
     # of them are exported, which is enough to pin the head of the window
     sh, _ = ctx.get_shadow(seq)
     ncol = min(W, sh.shape[1])
     flips = 0
-    for l in range(L):
+    for l in layers:
         for j in range(ncol):
             rep.compared += 1
             if sh[l, j] != ref.init_shadow[l, j]:
@@ -184,16 +186,16 @@ def compare_init(ctx, seq, ref: SeqRef, total_tokens: int, rep: Report, policy=N
     Sc, Sn, E, g = ctx.get_stats(seq)
     if flips == 0 and ref.init_conf is not None:
         sc, _ = ctx.get_conf(seq)
-        _compare_conf(rep, "init confidences", sc[:, :ncol], ref.init_conf[:, :ncol])
+        _compare_conf(rep, "init confidences", sc[layers, :ncol], ref.init_conf[layers, :ncol])
         Stcs, Sfcs, tau = ctx.get_conf_stats(seq)
         if ncol == W:       # the sums run over the whole window
-            _compare_conf(rep, "init Stcs", Stcs, ref.init_Stcs)
-            _compare_conf(rep, "init Sfcs", Sfcs, ref.init_Sfcs)
-    same = (out.tokens[0] == ref.first_token and np.array_equal(Sc, ref.init_Sc) and Sn == ref.init_Sn
+            _compare_conf(rep, "init Stcs", Stcs[layers], ref.init_Stcs[layers])
+            _compare_conf(rep, "init Sfcs", Sfcs[layers], ref.init_Sfcs[layers])
+    same = (out.tokens[0] == ref.first_token and np.array_equal(Sc[layers], ref.init_Sc[layers]) and Sn == ref.init_Sn
             and (policy or (E, g) == (ref.init_E, ref.init_gamma)))
     if not same:
         # the statistics sum over the whole window; any difference must come from a low-margin position
-        low = (ref.init_margin <= MARGIN).any()
+        low = (ref.init_margin[layers] <= MARGIN).any()
         if not low:
             rep.failures.append(f"init state differs without a low-margin position: token {out.tokens[0]} vs "
                                 f"{ref.first_token}, (E,g) {(E, g)} vs {(ref.init_E, ref.init_gamma)}")
@@ -209,9 +211,10 @@ def compare_init(ctx, seq, ref: SeqRef, total_tokens: int, rep: Report, policy=N
         ctx.set_exit_mode(seq, True)
 
 
-def compare_round(ctx, seq, out, r: RoundRef, rep: Report, check_choice=True) -> bool:
+def compare_round(ctx, seq, out, r: RoundRef, rep: Report, check_choice=True, layers=None) -> bool:
     """Compares one finished round; returns True if the library must be re-synchronised."""
     L = r.shadow.shape[0]
+    layers = list(range(L)) if layers is None else list(layers)
     rep.rounds += 1
     if r.draft_conf is not None and r.tau > 0.0 and out.tau > 0.0:
         # dynamic draft-exiting: the loop's decisions, wherever the oracle's numbers are clearly apart
@@ -254,7 +257,7 @@ def compare_round(ctx, seq, out, r: RoundRef, rep: Report, check_choice=True) ->
             flips += 1
             last_row = i
             break
-    for l in range(L):
+    for l in layers:
         for i in range(last_row + 1):
             rep.compared += 1
             if sh[l, i] != r.shadow[l, i]:
@@ -264,20 +267,20 @@ def compare_round(ctx, seq, out, r: RoundRef, rep: Report, check_choice=True) ->
                 flips += 1
     if flips == 0 and r.conf is not None:
         sc, dc = ctx.get_conf(seq)
-        _compare_conf(rep, f"round {rep.rounds}: shadow confidences", sc[:, :r.g + 1], r.conf)
+        _compare_conf(rep, f"round {rep.rounds}: shadow confidences", sc[layers, :r.g + 1], r.conf[layers])
         if r.draft_conf:
             _compare_conf(rep, f"round {rep.rounds}: draft confidences", dc[:len(r.draft_conf)], r.draft_conf)
         Stcs, Sfcs, tau = ctx.get_conf_stats(seq)
-        _compare_conf(rep, f"round {rep.rounds}: Stcs", Stcs, r.Stcs)
-        _compare_conf(rep, f"round {rep.rounds}: Sfcs", Sfcs, r.Sfcs)
+        _compare_conf(rep, f"round {rep.rounds}: Stcs", Stcs[layers], r.Stcs[layers])
+        _compare_conf(rep, f"round {rep.rounds}: Sfcs", Sfcs[layers], r.Sfcs[layers])
         _compare_conf(rep, f"round {rep.rounds}: next tau", [out.next_tau], [r.next_tau])
     if flips == 0:
         Sc, Sn, E, g = ctx.get_stats(seq)
         if out.n_accept != r.n or out.emitted() != list(r.emitted):
             rep.failures.append(f"round {rep.rounds}: accept {out.n_accept}/{out.emitted()} oracle {r.n}/{r.emitted}")
-        if not np.array_equal(counts, r.counts):
+        if not np.array_equal(counts[layers], r.counts[layers]):
             rep.failures.append(f"round {rep.rounds}: counts {counts.tolist()} oracle {r.counts.tolist()}")
-        if not (np.array_equal(Sc, r.Sc) and Sn == r.Sn):
+        if not (np.array_equal(Sc[layers], r.Sc[layers]) and Sn == r.Sn):
             rep.failures.append(f"round {rep.rounds}: statistics differ (Sn {Sn!r} vs {r.Sn!r})")
         if check_choice and (out.next_E, out.next_gamma) != (r.next_E, r.next_gamma):
             rep.failures.append(f"round {rep.rounds}: next (E,gamma) {(out.next_E, out.next_gamma)} oracle "
@@ -287,11 +290,11 @@ def compare_round(ctx, seq, out, r: RoundRef, rep: Report, check_choice=True) ->
     return True
 
 
-def run_sequence(ctx, seq, ref: SeqRef, total_tokens: int, policy=None, max_rounds=None, policy_fs=None) -> Report:
+def run_sequence(ctx, seq, ref: SeqRef, total_tokens: int, policy=None, max_rounds=None, policy_fs=None, layers=None) -> Report:
     """Prefill + rounds of one sequence through del_round, compared with the oracle's trace.
     policy = (E, gamma) fixes both; policy_fs = (E, gamma0) fixes E and lets the +-1 controller move gamma."""
     rep = Report()
-    compare_init(ctx, seq, ref, total_tokens, rep, policy)
+    compare_init(ctx, seq, ref, total_tokens, rep, policy, layers=layers)
     if policy_fs:
         ctx.set_policy_fs(seq, *policy_fs)
     done = 1
@@ -299,7 +302,7 @@ def run_sequence(ctx, seq, ref: SeqRef, total_tokens: int, policy=None, max_roun
         if max_rounds is not None and k >= max_rounds:
             break
         outs = ctx.round()
-        need = compare_round(ctx, seq, outs[seq], r, rep, check_choice=policy is None)
+        need = compare_round(ctx, seq, outs[seq], r, rep, check_choice=policy is None, layers=layers)
         done += r.n + 1
         if need and k + 1 < len(ref.rounds):
             rep.resyncs += 1

@@ -51,8 +51,9 @@ class SeqSampler:
     compared, and after a tolerated difference the library is put back into the oracle's state.  Several of
     these (and greedy sequences) can share the context's rounds."""
 
-    def __init__(self, ctx, seq, cfg, weights, prompt, temperature, top_p, seed, exit_mode=False, policy=None):
+    def __init__(self, ctx, seq, cfg, weights, prompt, temperature, top_p, seed, exit_mode=False, policy=None, layers=None):
         import oracle
+        self.layers = list(range(cfg.n_layers)) if layers is None else list(layers)
         self.ctx, self.seq, self.cfg, self.prompt = ctx, seq, cfg, prompt
         self.T, self.top_p, self.seed, self.exit_mode, self.policy = temperature, top_p, seed, exit_mode, policy
         self.total = cfg.gen_len
@@ -113,7 +114,7 @@ class SeqSampler:
         si = o.sample_info()
         rep.rounds += 1
         self.tokens.extend(r.emitted)
-        flip = _compare(self.ctx, self.seq, o, r, si, out, T0, self.T, self.top_p, self.seed, self.cfg.n_layers, rep)
+        flip = _compare(self.ctx, self.seq, o, r, si, out, T0, self.T, self.top_p, self.seed, self.layers, rep)
         if flip:
             rep.flips += 1
         if (flip or rep.failures) and len(self.tokens) < self.total:
@@ -125,8 +126,8 @@ class SeqSampler:
 
 
 def run_sequence_sampling(ctx, seq, cfg, weights, prompt, temperature, top_p, seed, exit_mode=False, policy=None,
-                          max_rounds=None) -> SReport:
-    s = SeqSampler(ctx, seq, cfg, weights, prompt, temperature, top_p, seed, exit_mode, policy)
+                          max_rounds=None, layers=None) -> SReport:
+    s = SeqSampler(ctx, seq, cfg, weights, prompt, temperature, top_p, seed, exit_mode, policy, layers)
     s.begin()
     while not s.done:
         if max_rounds is not None and s.rep.rounds >= max_rounds:
@@ -136,7 +137,7 @@ def run_sequence_sampling(ctx, seq, cfg, weights, prompt, temperature, top_p, se
     return s.rep
 
 
-def _compare(ctx, seq, o, r, si, out, T0, T, top_p, seed, L, rep: SReport) -> bool:
+def _compare(ctx, seq, o, r, si, out, T0, T, top_p, seed, layers, rep: SReport) -> bool:
     """Returns True when a tolerated difference makes the rest of the round incomparable."""
     import oracle
     what = f"round {rep.rounds}"
@@ -226,7 +227,7 @@ def _compare(ctx, seq, o, r, si, out, T0, T, top_p, seed, L, rep: SReport) -> bo
     # integers agree: shadow tokens by the margin rule, then counts and statistics bit for bit
     sh, counts = ctx.get_shadow(seq)
     low = False
-    for l in range(L):
+    for l in layers:
         for i in range(r.g + 1):
             if sh[l, i] != r.shadow[l, i]:
                 if r.margin[l, i] > MARGIN:
@@ -237,9 +238,9 @@ def _compare(ctx, seq, o, r, si, out, T0, T, top_p, seed, L, rep: SReport) -> bo
         return True
     Sc, Sn, E, g = ctx.get_stats(seq)
     Sc_or, Sn_or, _, _ = o.get_stats()
-    if not np.array_equal(counts, r.counts):
+    if not np.array_equal(counts[layers], r.counts[layers]):
         rep.failures.append(f"{what}: counts {counts.tolist()} oracle {r.counts.tolist()}")
-    if not (np.array_equal(Sc, Sc_or) and Sn == Sn_or):
+    if not (np.array_equal(Sc[layers], Sc_or[layers]) and Sn == Sn_or):
         rep.failures.append(f"{what}: statistics differ (Sn {Sn!r} vs {Sn_or!r})")
     if (out.next_E, out.next_gamma) != (r.next_E, r.next_gamma):
         rep.failures.append(f"{what}: next (E,gamma) {(out.next_E, out.next_gamma)} oracle {(r.next_E, r.next_gamma)}")

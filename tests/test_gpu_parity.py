@@ -394,6 +394,33 @@ def test_batch_with_mixed_exit_modes():
         assert rep.rounds == len(refs[s].rounds)
 
 
+@pytest.mark.parametrize("exit_mode", [False, True], ids=["fixed_gamma", "draft_exiting"])
+def test_stacked_head_rows_trimmed_to_candidate_layers(exit_mode):
+    """With the rows of the stacked LM head restricted to the layers the selection can pick (e_min..e_max) plus
+    the last one, everything the method uses is unchanged: the stream, the accept lengths, the statistics of the
+    candidate layers, the thresholds and the (E, gamma) trajectory; fewer rows go through the head."""
+    import paper_2504_05598_b200 as dl
+    cfg = synth.small_variant(TINY_GQA, name="tiny_gqa_trim", e_min=2, e_max=4, gen_len=40)      # L = 6
+    w = synth.make_weights(cfg)
+    ctx = make_ctx(cfg, w)
+    ref = ref_from_oracle(cfg, w, synth.make_prompt(cfg), exit_mode=exit_mode)
+    layers = list(range(cfg.e_min - 1, cfg.e_max)) + [cfg.n_layers - 1]
+    ctx.set_flags(dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_TRIM_ROWS)
+    rep = run_sequence(ctx, 0, ref, cfg.gen_len, layers=layers)
+    print(f"trimmed rows (exit mode {exit_mode}): rounds {rep.rounds} compared {rep.compared} flips {rep.flips}")
+    assert rep.ok(), rep.failures[:5]
+    assert rep.rounds == len(ref.rounds)
+    # the same through the streaming head, and with speculative sampling on top
+    ctx.set_flags(dl.FLAG_PDL | dl.FLAG_TRIM_ROWS)
+    rep = run_sequence(ctx, 0, ref, cfg.gen_len, layers=layers)
+    assert rep.ok(), rep.failures[:5]
+    ctx.set_flags(dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_TRIM_ROWS)
+    from sampling_parity import run_sequence_sampling
+    srep = run_sequence_sampling(ctx, 0, cfg, w, synth.make_prompt(cfg), 0.6, 0.95, 3, exit_mode=exit_mode, layers=layers)
+    assert srep.ok() and srep.rounds >= 5, srep.failures[:5]
+    ctx.close()
+
+
 def test_fs_baseline_policy_against_oracle(small):
     """Baseline FS(E-gamma) of Sec. 5.1 on the same kernels: fixed exit layer, gamma moved by +-1 on the device."""
     cfg, w, ctx = small
