@@ -89,8 +89,9 @@ def test_sampling_kernels_against_oracle(V):
             assert _margin(qq, x, ud) < 1e-7, f"{tag}: draft {out[0]} oracle {x}"
             near += 1
             continue
-        assert prob[0] == pytest.approx(qq[x], rel=1e-6), tag
-        assert prob[1] == pytest.approx(pp[x], rel=1e-6, abs=1e-30), tag
+        # (the library's weights are 40-bit fixed point: a filtered probability carries an absolute error below 2e-12)
+        assert prob[0] == pytest.approx(qq[x], rel=1e-6, abs=2e-12), tag
+        assert prob[1] == pytest.approx(pp[x], rel=1e-6, abs=2e-12), tag
         ratio = min(1.0, pp[x] / qq[x])
         if bool(out[1]) != (ua < ratio):
             assert abs(ua - ratio) < 1e-7, f"{tag}: acceptance {out[1]} oracle u {ua} ratio {ratio}"
