@@ -215,6 +215,12 @@ int del_get_sample_info(del_ctx *ctx, int seq, int32_t *n_tests, int32_t *from_r
  * draft `row`, which = 1 the target's row `row` (0..g).  Synchronises. */
 int del_get_round_logits(del_ctx *ctx, int seq, int which, int row, float *out);
 
+/* Test reader: shadow tokens and their confidences of the first n_cols slots (1 <= n_cols <= 64) of every layer:
+ * after del_prefill the whole initialisation window (n_cols = min(init_window, n_prompt)), which del_get_shadow
+ * and del_get_conf, sized for a round, cut at g_max + 1 columns.  HOST [n_layers][n_cols] each, either may be
+ * NULL.  Synchronises. */
+int del_get_window(del_ctx *ctx, int seq, int n_cols, int32_t *shadow, float *conf);
+
 /* Test hook: the sampling kernels' device functions on one caller-supplied pair of rows (HOST float [vocab],
  * vocab <= the model's).  out (HOST int32 [4]): the token drawn from the filtered draft row with u_draft; 1 if
  * u_accept accepts it; the token the residual distribution gives with u_final; the token the filtered target

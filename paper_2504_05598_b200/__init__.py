@@ -28,7 +28,7 @@ EXPORTS = ["del_workspace_bytes", "del_init", "del_prefill", "del_draft", "del_v
            "del_select", "del_round", "del_set_policy", "del_get_stats", "del_set_stats", "del_get_shadow",
            "del_get_drafts", "del_force_token", "del_get_hidden", "del_debug_logits", "del_get_kv", "del_committed_len", "del_release",
            "del_launch_count", "del_get_traffic", "del_set_flags", "del_get_kernel_times", "del_head_argmax_static",
-           "del_set_policy_fs", "del_set_exit_mode", "del_set_sampling", "del_get_sample_info", "del_get_round_logits", "del_sample_probe", "del_get_conf_stats", "del_set_conf_stats", "del_get_conf", "del_strerror", "del_last_cuda_error", "del_destroy"]
+           "del_set_policy_fs", "del_set_exit_mode", "del_get_window", "del_set_sampling", "del_get_sample_info", "del_get_round_logits", "del_sample_probe", "del_get_conf_stats", "del_set_conf_stats", "del_get_conf", "del_strerror", "del_last_cuda_error", "del_destroy"]
 
 
 class Shape(C.Structure):
@@ -100,6 +100,8 @@ def load_library(build_if_missing: bool = True):
     L.del_set_policy_fs.argtypes = [vp, ci, ci, ci]
     L.del_set_exit_mode.restype = ci
     L.del_set_exit_mode.argtypes = [vp, ci, ci]
+    L.del_get_window.restype = ci
+    L.del_get_window.argtypes = [vp, ci, ci, vp, vp]
     L.del_set_sampling.restype = ci
     L.del_set_sampling.argtypes = [vp, ci, C.c_double, C.c_double, C.c_uint64]
     L.del_get_sample_info.restype = ci
@@ -338,6 +340,14 @@ class DelContext:
         dc = np.zeros(G, dtype=np.float32)
         self._ck(self.lib.del_get_conf(self._h, seq, sc.ctypes.data, dc.ctypes.data), "del_get_conf")
         return sc, dc
+
+    def get_window(self, seq: int, n_cols: int):
+        """(shadow tokens, confidences) of the first n_cols slots of every layer: the prefill's whole window."""
+        L = self.shape.n_layers
+        sh = np.zeros((L, n_cols), dtype=np.int32)
+        cf = np.zeros((L, n_cols), dtype=np.float32)
+        self._ck(self.lib.del_get_window(self._h, seq, n_cols, sh.ctypes.data, cf.ctypes.data), "del_get_window")
+        return sh, cf
 
     def get_shadow(self, seq: int):
         L, G = self.shape.n_layers, self.shape.g_max + 1

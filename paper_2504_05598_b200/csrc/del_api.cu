@@ -1418,6 +1418,25 @@ int del_get_conf(del_ctx *c, int sq, float *shadow_conf, float *draft_conf) {
     return DEL_OK;
 }
 
+int del_get_window(del_ctx *c, int sq, int n_cols, int32_t *shadow, float *conf) {
+    if (!seq_ok(c, sq) || n_cols < 1 || n_cols > c->D.S) return DEL_EINVAL;
+    CK(cudaStreamSynchronize(c->st));
+    const int L = c->D.L, S = c->D.S;
+    if (shadow) {
+        std::vector<int32_t> tmp((size_t)L * S);
+        CK(cudaMemcpy(tmp.data(), c->B.SHADOW + (size_t)sq * L * S, sizeof(int32_t) * L * S, cudaMemcpyDeviceToHost));
+        for (int l = 0; l < L; ++l)
+            for (int i = 0; i < n_cols; ++i) shadow[l * n_cols + i] = tmp[(size_t)l * S + i];
+    }
+    if (conf) {
+        std::vector<float> tmp((size_t)L * S);
+        CK(cudaMemcpy(tmp.data(), c->B.SCONF + (size_t)sq * L * S, sizeof(float) * L * S, cudaMemcpyDeviceToHost));
+        for (int l = 0; l < L; ++l)
+            for (int i = 0; i < n_cols; ++i) conf[l * n_cols + i] = tmp[(size_t)l * S + i];
+    }
+    return DEL_OK;
+}
+
 int del_get_shadow(del_ctx *c, int sq, int32_t *shadow, int32_t *counts) {
     if (!seq_ok(c, sq)) return DEL_EINVAL;
     CK(cudaStreamSynchronize(c->st));

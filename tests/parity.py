@@ -170,10 +170,9 @@ def compare_init(ctx, seq, ref: SeqRef, total_tokens: int, rep: Report, policy=N
         ctx.set_policy(seq, *policy)
     L, W = ref.init_shadow.shape
     layers = list(range(L)) if layers is None else list(layers)
-    # after the prefill the shadow buffer holds the window's tokens in its first W columns; only g_max+1
-    # of them are exported, which is enough to pin the head of the window
-    sh, _ = ctx.get_shadow(seq)
-    ncol = min(W, sh.shape[1])
+    # after the prefill the shadow buffer holds the window's tokens and confidences in its first W columns
+    sh, win_conf = ctx.get_window(seq, W)
+    ncol = W
     flips = 0
     for l in layers:
         for j in range(ncol):
@@ -185,8 +184,7 @@ def compare_init(ctx, seq, ref: SeqRef, total_tokens: int, rep: Report, policy=N
                 flips += 1
     Sc, Sn, E, g = ctx.get_stats(seq)
     if flips == 0 and ref.init_conf is not None:
-        sc, _ = ctx.get_conf(seq)
-        _compare_conf(rep, "init confidences", sc[layers, :ncol], ref.init_conf[layers, :ncol])
+        _compare_conf(rep, "init confidences", win_conf[layers, :ncol], ref.init_conf[layers, :ncol])
         Stcs, Sfcs, tau = ctx.get_conf_stats(seq)
         if ncol == W:       # the sums run over the whole window
             _compare_conf(rep, "init Stcs", Stcs[layers], ref.init_Stcs[layers])

@@ -421,6 +421,36 @@ def test_stacked_head_rows_trimmed_to_candidate_layers(exit_mode):
     ctx.close()
 
 
+def test_random_shapes_against_oracle():
+    """Seeded random small models: depth, candidate-layer and speculation-length ranges (g_min = 0 included),
+    prompt lengths on both sides of the window and of the tensor-core prefill's chunk, batch sizes 1 to 3, greedy
+    and draft-exiting sequences mixed; every one compared with the oracle round by round."""
+    rng = np.random.default_rng(20250405)
+    rounds = compared = 0
+    for k in range(24):
+        base = TINY_GQA if k % 2 else TINY
+        L = int(rng.integers(3, 9))
+        e_min = int(rng.integers(1, L - 1))
+        e_max = min(int(rng.integers(e_min, L)), L - 1)
+        g_max = int(rng.integers(1, 9))
+        g_min = int(rng.integers(0, min(2, g_max) + 1))
+        cfg = synth.small_variant(base, name=f"random{k}", n_layers=L, e_min=e_min, e_max=e_max, g_min=g_min, g_max=g_max,
+                                  prompt_len=int(rng.choice([1, 5, 31, 32, 33, 70, 96, 130, 300, 520, 700])),
+                                  gen_len=int(rng.integers(4, 40)), seed=int(rng.integers(1, 10 ** 6)), emb_scale=10.0,
+                                  batch=int(rng.choice([1, 1, 2, 3])))
+        w = synth.make_weights(cfg)
+        ctx = make_ctx(cfg, w)
+        exit_mode = k % 3 == 0
+        refs = [ref_from_oracle(cfg, w, synth.make_prompt(cfg, s), exit_mode=exit_mode and s % 2 == 0) for s in range(cfg.batch)]
+        reps = run_batch(ctx, refs, cfg.gen_len) if cfg.batch > 1 else [run_sequence(ctx, 0, refs[0], cfg.gen_len)]
+        for ref, rep in zip(refs, reps):
+            assert rep.ok() and rep.rounds == len(ref.rounds), (k, cfg, rep.failures[:3])
+            rounds += rep.rounds
+            compared += rep.compared
+        ctx.close()
+    print(f"24 random shapes: {rounds} rounds, {compared} arg-max results compared")
+
+
 def test_fs_baseline_policy_against_oracle(small):
     """Baseline FS(E-gamma) of Sec. 5.1 on the same kernels: fixed exit layer, gamma moved by +-1 on the device."""
     cfg, w, ctx = small
