@@ -422,13 +422,15 @@ def test_stacked_head_rows_trimmed_to_candidate_layers(exit_mode):
 
 
 def test_random_shapes_against_oracle():
-    """Seeded random small models: depth, candidate-layer and speculation-length ranges (g_min = 0 included),
+    """Seeded random small models: depth, head dimension 64 / 128, candidate-layer and speculation-length ranges (g_min = 0 included),
     prompt lengths on both sides of the window and of the tensor-core prefill's chunk, batch sizes 1 to 3, greedy
     and draft-exiting sequences mixed; every one compared with the oracle round by round."""
     rng = np.random.default_rng(20250405)
     rounds = compared = 0
     for k in range(24):
         base = TINY_GQA if k % 2 else TINY
+        if k % 4 >= 2:                                   # head dimension 128, two query heads on two or one kv head
+            base = synth.small_variant(base, head_dim=128, n_heads=2, n_kv_heads=2 if k % 8 < 4 else 1)
         L = int(rng.integers(3, 9))
         e_min = int(rng.integers(1, L - 1))
         e_max = min(int(rng.integers(e_min, L)), L - 1)
