@@ -163,7 +163,7 @@ def _compare_conf(rep: Report, what: str, got, want):
             rep.failures.append(f"{what}: element {k} gpu {got.flat[k]:.6f} oracle {want.flat[k]:.6f}")
 
 
-def compare_init(ctx, seq, ref: SeqRef, total_tokens: int, rep: Report, policy=None, layers=None) -> None:
+def compare_init(ctx, seq, ref: SeqRef, total_tokens: int, rep: Report, policy=None, layers=None, check_choice=True) -> None:
     """layers: 0-based layers to compare (default all; with trimmed stacked-head rows only those are maintained)."""
     out = ctx.prefill(seq, ref.prompt, total_tokens)
     if policy:
@@ -190,7 +190,7 @@ def compare_init(ctx, seq, ref: SeqRef, total_tokens: int, rep: Report, policy=N
             _compare_conf(rep, "init Stcs", Stcs[layers], ref.init_Stcs[layers])
             _compare_conf(rep, "init Sfcs", Sfcs[layers], ref.init_Sfcs[layers])
     same = (out.tokens[0] == ref.first_token and np.array_equal(Sc[layers], ref.init_Sc[layers]) and Sn == ref.init_Sn
-            and (policy or (E, g) == (ref.init_E, ref.init_gamma)))
+            and (policy or not check_choice or (E, g) == (ref.init_E, ref.init_gamma)))
     if not same:
         # the statistics sum over the whole window; any difference must come from a low-margin position
         low = (ref.init_margin[layers] <= MARGIN).any()
@@ -217,10 +217,19 @@ def compare_round(ctx, seq, out, r: RoundRef, rep: Report, check_choice=True, la
     if r.draft_conf is not None and r.tau > 0.0 and out.tau > 0.0:
         # dynamic draft-exiting: the loop's decisions, wherever the oracle's numbers are clearly apart
         _, dc = ctx.get_conf(seq)
+        got_drafts = ctx.get_drafts(seq)
         n_dec = min(len(r.draft_conf), out.g + int(out.stopped))
         rep.decisions += n_dec
         _compare_conf(rep, f"round {rep.rounds}: tau", [out.tau], [r.tau])
         for i in range(n_dec):
+            if i > 0 and got_drafts[i - 1] != r.drafts[i - 1]:
+                # the previous draft differs (allowed at a low margin): this token saw another input, its
+                # confidence is not comparable any more
+                if r.margin[r.E - 1, i - 1] > MARGIN:
+                    rep.failures.append(f"round {rep.rounds}: draft {i - 1} gpu {got_drafts[i - 1]} oracle {r.drafts[i - 1]} "
+                                        f"margin {r.margin[r.E - 1, i - 1]:.3f}")
+                rep.flips += 1
+                return True
             want_stop, got_stop = r.draft_conf[i] < r.tau, float(dc[i]) < out.tau
             if want_stop != got_stop:
                 band = CONF_RTOL * (r.draft_conf[i] + r.tau)
@@ -292,7 +301,8 @@ def run_sequence(ctx, seq, ref: SeqRef, total_tokens: int, policy=None, max_roun
     """Prefill + rounds of one sequence through del_round, compared with the oracle's trace.
     policy = (E, gamma) fixes both; policy_fs = (E, gamma0) fixes E and lets the +-1 controller move gamma."""
     rep = Report()
-    compare_init(ctx, seq, ref, total_tokens, rep, policy, layers=layers)
+    # (with the FS baseline the reference's first (E, gamma) is the policy's, set after the prefill: nothing to compare)
+    compare_init(ctx, seq, ref, total_tokens, rep, policy, layers=layers, check_choice=policy_fs is None)
     if policy_fs:
         ctx.set_policy_fs(seq, *policy_fs)
     done = 1

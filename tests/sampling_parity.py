@@ -7,7 +7,8 @@ Both sides run freely from the same state with the same counter-based uniform nu
   * every decision (drafted token, accept / reject, last token): identical, or inside the band that logits eps
     apart allow: each filtered probability then differs by at most a factor exp(4 eps / T) (numerator,
     normaliser and nucleus mass), so a cumulative probability moves by at most delta = exp(4 eps / T) - 1 and
-    an acceptance ratio by twice that (relative).  A decision inside its band is a tolerated flip: it is
+    an acceptance ratio by twice that (relative); tokens at the very end of a nucleus may be kept on one side only,
+    which moves the cumulative probabilities behind them by their filtered mass on top of delta.  A decision inside its band is a tolerated flip: it is
     counted and the library is put back into the oracle's state (re-prefill on the oracle's tokens);
   * the filtered probabilities q(x), p(x) the library reports: relative tolerance delta; a token at the very end
     of a nucleus (mass ahead of it within delta of top_p) may be inside on one side and outside on the other: its
@@ -46,6 +47,19 @@ class SReport:
 def _cdf_interval(probs, x):
     c = np.cumsum(probs)
     return c[x] - probs[x], c[x]
+
+
+def _edge_mass(logits, T, top_p, delta) -> float:
+    """Filtered mass of the tokens that may be inside the nucleus on one side and outside on the other (mass
+    ahead of them within delta of top_p): a cumulative probability behind them can move by that much on top of delta."""
+    import oracle
+    if top_p >= 1.0:
+        return 0.0
+    full = oracle.nucleus(logits, T, 1.0)
+    order = np.argsort(-full, kind="stable")
+    ahead = np.concatenate([[0.0], np.cumsum(full[order])[:-1]])
+    unsure = np.abs(ahead - top_p) <= delta + full[order]
+    return float(full[order][unsure].sum() / top_p)
 
 
 def _at_nucleus_edge(logits, x, T, top_p, delta) -> bool:
@@ -107,6 +121,7 @@ class SeqSampler:
             rep.failures.append(f"prefill: target logits differ by {eps:.4f}")
         if first.tokens[0] != self.tokens[0]:
             delta = float(np.exp(4 * eps / self.T) - 1.0) + 1e-6
+            delta += _edge_mass(lg_or, self.T, self.top_p, delta)
             lo, hi = _cdf_interval(oracle.nucleus(lg_or, self.T, self.top_p), first.tokens[0])
             u = oracle.uniform(self.seed, len(self.prompt), 2)
             if not (lo - delta <= u <= hi + delta):
@@ -175,7 +190,8 @@ def _compare(ctx, seq, o, r, si, out, T0, T, top_p, seed, layers, rep: SReport) 
         if drafts[i] != r.drafts[i]:
             qq = oracle.nucleus(o.round_logits(0, i), T, top_p)
             lo, hi = _cdf_interval(qq, drafts[i])
-            if not (lo - delta <= si.u_draft[i] <= hi + delta):
+            band = delta + _edge_mass(o.round_logits(0, i), T, top_p, delta)
+            if not (lo - band <= si.u_draft[i] <= hi + band):
                 rep.failures.append(f"{what}: draft {i} gpu {drafts[i]} oracle {r.drafts[i]}, u {si.u_draft[i]:.6f} "
                                     f"outside [{lo:.6f}, {hi:.6f}] +- {delta:.2e}")
             return True
@@ -240,7 +256,8 @@ def _compare(ctx, seq, o, r, si, out, T0, T, top_p, seed, layers, rep: SReport) 
                 rep.failures.append(f"{what}: last token {x} has no residual mass within the band")
         else:
             lo, hi = _cdf_interval(pp, x)
-            if not (lo - delta <= si.u_final <= hi + delta):
+            band = delta + _edge_mass(o.round_logits(1, n), T, top_p, delta)
+            if not (lo - band <= si.u_final <= hi + band):
                 rep.failures.append(f"{what}: last token {x} oracle {r.emitted[n]}, u {si.u_final:.6f} outside "
                                     f"[{lo:.6f}, {hi:.6f}]")
         return True
