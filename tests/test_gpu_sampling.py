@@ -282,34 +282,49 @@ def test_cold_sampling_reproduces_greedy_trace_full_size(name):
     ctx.close()
 
 
-def test_sampling_full_size_consistency():
-    """Llama-2-7B shape at temperature 0.6 / top-p 0.95: the reported decisions are consistent with the reported
-    probabilities and the uniform numbers of (seed, position, purpose); tokens are valid ids; sampling with the same
-    seed is reproducible."""
+@pytest.mark.parametrize("name", ["llama2_7b", "llama3_8b_b4"])
+def test_sampling_full_size_consistency(name):
+    """Full-size shapes (Llama-2-7B; Llama-3-8B with four sequences, grouped-query attention and a 128 256-token
+    vocabulary) at temperature 0.6 / 1.0, top-p 0.95, one sequence of the batch with draft-exiting: the reported
+    decisions are consistent with the reported probabilities and the uniform numbers of (seed, position, purpose);
+    tokens are valid ids; a second run with the same seeds gives the same streams."""
     import oracle
-    name = "llama2_7b"
     cfg = synth.CONFIGS[name]
     ctx = make_ctx(cfg, synth.make_weights(cfg))
-    prompt = synth.make_prompt(cfg, 0)
+    B, n_tok = cfg.batch, 40
     streams = []
     for attempt in range(2):
-        ctx.set_sampling(0, 0.6, 0.95, 2024)
-        first = ctx.prefill(0, prompt, 48)
-        ctx.set_policy(0, 8, 3)
-        toks, T = [first.tokens[0]], len(prompt)
-        while len(toks) < 48:
-            out = ctx.round()[0]
-            n_tests, from_res, qx, px = ctx.get_sample_info(0)
-            assert 0 <= out.n_accept <= out.g and out.n_emitted == out.n_accept + 1
-            assert n_tests == min(out.n_accept + 1, out.g) and from_res == (out.n_accept < out.g)
-            for i in range(n_tests):
-                u = oracle.uniform(2024, T + 1 + i, 1)
-                ratio = min(1.0, float(px[i]) / float(qx[i]))
-                if abs(u - ratio) > 1e-5:
-                    assert (u < ratio) == (i < out.n_accept), (i, u, ratio)
-            assert all(0 <= t < cfg.vocab for t in out.emitted())
-            toks.extend(out.emitted())
-            T += out.n_emitted
+        T, toks = [], [[] for _ in range(B)]
+        for s in range(B):
+            prompt = synth.make_prompt(cfg, s)
+            ctx.set_sampling(s, 0.6 if s % 2 == 0 else 1.0, 0.95, 2024 + s)
+            first = ctx.prefill(s, prompt, n_tok)
+            if B == 1:
+                ctx.set_policy(s, 8, 3)
+            elif s == B - 1:
+                ctx.set_exit_mode(s, True)
+            toks[s].append(first.tokens[0])
+            T.append(len(prompt))
+        tests = 0
+        while any(len(t) < n_tok for t in toks):
+            outs = ctx.round()
+            for s in range(B):
+                out = outs[s]
+                if out.n_emitted == 0:
+                    continue
+                n_tests, from_res, qx, px = ctx.get_sample_info(s)
+                assert 0 <= out.n_accept <= out.g and out.n_emitted == out.n_accept + 1
+                assert n_tests == min(out.n_accept + 1, out.g) and from_res == (out.n_accept < out.g)
+                for i in range(n_tests):
+                    u = oracle.uniform(2024 + s, T[s] + 1 + i, 1)
+                    ratio = min(1.0, float(px[i]) / float(qx[i]))
+                    if abs(u - ratio) > 1e-5:
+                        assert (u < ratio) == (i < out.n_accept), (s, i, u, ratio)
+                    tests += 1
+                assert all(0 <= t < cfg.vocab for t in out.emitted())
+                toks[s] += out.emitted()
+                T[s] += out.n_emitted
+        assert tests > 0
         streams.append(toks)
     assert streams[0] == streams[1]
     ctx.close()
