@@ -263,22 +263,29 @@ def test_sampling_step_calls_equal_round_call(exit_mode):
     ctx.close()
 
 
-@pytest.mark.parametrize("name", ["llama2_7b", "llama32_1b"])
+@pytest.mark.parametrize("name", ["llama2_7b", "llama32_1b", "llama2_13b", "llama3_8b_b4"])
 def test_cold_sampling_reproduces_greedy_trace_full_size(name):
     """Temperature -> 0 puts all filtered mass on the arg-max: the sampling path (logit rows of exit head and target,
-    nucleus, draws, acceptance ratio, residual) must then reproduce the stored greedy oracle trace of the full-size
-    shape, decision by decision."""
+    nucleus, draws, acceptance ratio, residual) must then reproduce the stored greedy oracle traces of the full-size
+    shapes, decision by decision (the four sequences of the 8B shape share their rounds)."""
+    from parity import run_batch
     path = os.path.join(GOLDEN, f"trace_{name}.json")
     if not os.path.exists(path):
         pytest.skip("no stored trace")
     doc = json.load(open(path))
     cfg = synth.CONFIGS[name]
     ctx = make_ctx(cfg, synth.make_weights(cfg))
-    ctx.set_sampling(0, 1e-4, 0.95, 77)
-    ref = ref_from_golden(doc, 0, synth.make_prompt(cfg, 0))
-    rep = run_sequence(ctx, 0, ref, doc["gen_len"], max_rounds=30)
-    print(f"{name} (cold sampling): rounds {rep.rounds} compared {rep.compared} flips {rep.flips} resyncs {rep.resyncs}")
-    assert rep.ok(), rep.failures[:8]
+    for s in range(cfg.batch):
+        ctx.set_sampling(s, 1e-4, 0.95, 77 + s)
+    refs = [ref_from_golden(doc, s, synth.make_prompt(cfg, s)) for s in range(cfg.batch)]
+    if cfg.batch > 1:
+        reps = run_batch(ctx, refs, doc["gen_len"])
+    else:
+        reps = [run_sequence(ctx, 0, refs[0], doc["gen_len"], max_rounds=40)]
+    for s, rep in enumerate(reps):
+        print(f"{name} seq {s} (cold sampling): rounds {rep.rounds} compared {rep.compared} flips {rep.flips} resyncs {rep.resyncs}")
+        assert rep.ok(), rep.failures[:8]
+        assert rep.rounds >= 20
     ctx.close()
 
 
