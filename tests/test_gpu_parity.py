@@ -453,6 +453,78 @@ def test_random_shapes_against_oracle():
     print(f"24 random shapes: {rounds} rounds, {compared} arg-max results compared")
 
 
+def test_interleaved_sequence_lifetimes_with_few_pages():
+    """Four slots, 22 KV pages: sequences of random prompt and generation lengths start, run, finish and are released
+    at random times (some with draft-exiting), so that pages change hands and some prefills or rounds are refused for
+    lack of pages (DEL_ENOSPC, after which the context goes on).  Every sequence is compared with its own oracle."""
+    import paper_2504_05598_b200 as dl
+    from parity import Report, _resync, compare_init, compare_round
+    rng = np.random.default_rng(1)
+    B = 4
+    base = synth.small_variant(TINY_GQA, name="lifetimes", batch=B, prompt_len=64, gen_len=40, g_max=4)
+    w = synth.make_weights(base)
+    ctx = dl.DelContext(dl.make_shape(base, max_seq=256, n_pages=22), dl.upload_weights(w))
+    slots = [None] * B
+    n = dict(starts=0, refused=0, rounds=0, released=0, finished=0)
+    for step in range(300):
+        act = rng.random()
+        free = [s for s in range(B) if slots[s] is None]
+        live = [s for s in range(B) if slots[s] is not None]
+        if free and (act < 0.3 or not live):
+            s = int(rng.choice(free))
+            G = int(rng.integers(3, 40))
+            cfg = synth.small_variant(base, prompt_len=int(rng.choice([1, 7, 33, 64, 100, 130])), gen_len=G,
+                                      seed=int(rng.integers(1, 10 ** 6)))
+            ref = ref_from_oracle(cfg, w, synth.make_prompt(cfg, s), exit_mode=bool(rng.random() < 0.3))
+            rep = Report()
+            try:
+                compare_init(ctx, s, ref, G, rep)
+            except dl.DelError as e:
+                assert e.code == dl.ENOSPC
+                n["refused"] += 1
+                continue
+            slots[s] = dict(ref=ref, k=0, done=1, rep=rep, G=G)
+            n["starts"] += 1
+        elif live and act < 0.4:
+            s = int(rng.choice(live))
+            ctx.release(s)
+            slots[s] = None
+            n["released"] += 1
+        elif live:
+            try:
+                outs = ctx.round()
+            except dl.DelError as e:                      # no page for some sequence's round: give up the longest one
+                assert e.code == dl.ENOSPC
+                s = max(live, key=lambda q: len(slots[q]["ref"].prompt) + slots[q]["done"])
+                ctx.release(s)
+                slots[s] = None
+                n["refused"] += 1
+                continue
+            n["rounds"] += 1
+            for s in live:
+                st = slots[s]
+                ref = st["ref"]
+                r = ref.rounds[st["k"]]
+                need = compare_round(ctx, s, outs[s], r, st["rep"])
+                assert st["rep"].ok(), (step, s, st["rep"].failures[:3])
+                st["done"] += r.n + 1
+                st["k"] += 1
+                if st["k"] >= len(ref.rounds):
+                    n["finished"] += 1
+                    ctx.release(s)
+                    slots[s] = None
+                elif need:
+                    try:
+                        _resync(ctx, s, ref, st["done"], r.Sc, r.Sn, r.next_E, r.next_gamma, st["G"], r.Stcs, r.Sfcs)
+                    except dl.DelError as e:
+                        assert e.code == dl.ENOSPC
+                        slots[s] = None
+                        n["refused"] += 1
+    print(n)
+    assert n["finished"] >= 15 and n["refused"] >= 3 and n["released"] >= 10
+    ctx.close()
+
+
 def test_fs_baseline_policy_against_oracle(small):
     """Baseline FS(E-gamma) of Sec. 5.1 on the same kernels: fixed exit layer, gamma moved by +-1 on the device."""
     cfg, w, ctx = small
