@@ -1,11 +1,12 @@
 """Benchmark of the DEL self-speculative decode round (libdel) on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+    python bench.py --profile-case --config NAME --layers 4 --rounds 8 [--policy E,G] [--sampling T,top_p] ...
 
 A step is one whole round (draft, verify, stacked LM head + accept + statistics, selection) of every
 live sequence of the configuration, through the C ABI.  Rank 0 prints one JSON line.  With N > 1
 (torchrun) every rank runs an independent replica on its own prompt: the method has no exchange step,
-so there is no collective on the data path.  `--impl reference` times the CPU oracle instead.
+so there is no collective on the data path.  `--impl reference` times the CPU oracle on the same prompt instead.
 """
 from __future__ import annotations
 
@@ -106,24 +107,39 @@ def round_bytes_exit(cfg, E, g, stopped, T):
     return total
 
 
-def oracle_sample(cfg, weights, seconds: float):
-    """Times the oracle (as it stands) on a bounded sample: short prompt prefix, rounds until the time is up."""
+def oracle_rounds(cfg, weights, warmup: int, steps: int = 0, seconds: float = 0.0):
+    """Times the oracle (as it stands) on the benchmark's own workload: its prefill of the configuration's whole
+    prompt (untimed, reported), `warmup` untimed DEL rounds, then `steps` rounds (or rounds until `seconds` have
+    passed) from the same seeded state the GPU arm starts from."""
     import oracle
     o = oracle.OracleSeq(cfg, weights)
-    n_prefix = 8
-    prompt = synth.make_prompt(cfg, 0)[:n_prefix]
+    prompt = synth.make_prompt(cfg, 0)
+    t0 = time.perf_counter()
     o.prefill(prompt)
+    t_prefill = time.perf_counter() - t0
+    left = cfg.gen_len - 1
+    for _ in range(warmup):
+        if left > 0:
+            left -= len(o.round(left).emitted)
     t0 = time.perf_counter()
     toks, rounds = 0, 0
-    while time.perf_counter() - t0 < seconds and toks < cfg.gen_len - 1:
-        r = o.round(cfg.gen_len - 1 - toks)
+    while left > 0 and ((steps and rounds < steps) or (not steps and time.perf_counter() - t0 < seconds)):
+        r = o.round(left)
         toks += len(r.emitted)
+        left -= len(r.emitted)
         rounds += 1
     dt = time.perf_counter() - t0
     o.close()
     return {"value": toks / dt, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"{cfg.name}: {n_prefix}-token prompt prefix, {rounds} DEL rounds ({toks} tokens) in {dt:.1f}s, "
-                      f"decode only"}, dt / max(rounds, 1)
+            "sample": f"{cfg.name}: the {len(prompt)}-token prompt prefilled by the oracle ({t_prefill:.0f}s, untimed), "
+                      f"{warmup} warm-up rounds, then {rounds} DEL rounds ({toks} tokens) in {dt:.1f}s, decode only"}, \
+        dt / max(rounds, 1)
+
+
+def bench_config(cfg, world: int):
+    """The `config` object of the JSON line; both arms print the same one."""
+    return {"workload": workload_name(cfg), "l2": "inputs larger than L2 (weights streamed every pass)",
+            "parallelism": "replicas only" if world > 1 else "single GPU"}
 
 
 def run_reference(a):
@@ -132,12 +148,11 @@ def run_reference(a):
         return
     cfg = synth.CONFIGS[a.config]
     weights = synth.make_weights(cfg)
-    budget = min(240.0, 6.0 * (a.steps + a.warmup))
-    cb, s_per_round = oracle_sample(cfg, weights, budget)
+    cb, s_per_round = oracle_rounds(cfg, weights, min(a.warmup, 3), steps=a.steps)
     line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": "tokens/s", "n_gpus": a.gpus,
             "steps": a.steps, "warmup": a.warmup, "ms_per_step": 1000.0 * s_per_round, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": workload_name(cfg), "l2": "inputs larger than L2"},
+            "config": bench_config(cfg, int(os.environ.get("WORLD_SIZE", "1"))),
             "cpu_baseline": cb, "gpu_launches": 0,
             "e2e": {"value": cb["value"], "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
@@ -146,7 +161,8 @@ def run_reference(a):
 def workload_name(cfg):
     return (f"{cfg.name}: L{cfg.n_layers} d{cfg.d_model} {cfg.n_heads}q/{cfg.n_kv_heads}kv x{cfg.head_dim} F{cfg.d_ffn} "
             f"V{cfg.vocab}, batch {cfg.batch}, prompt {cfg.prompt_len}, DEL dynamic E {cfg.e_min}..{cfg.e_max} "
-            f"gamma {cfg.g_min}..{cfg.g_max}")
+            f"gamma {cfg.g_min}..{cfg.g_max}; random weights N(0, 0.02^2) with depth-decaying o_proj/down_proj, "
+            f"token-embedding table drawn with std 1.0 (with std 0.02 the greedy stream is one constant token)")
 
 
 def aggregate_replicas(dev_ms, wall, tokens, bytes_total, world, device):
@@ -196,10 +212,10 @@ def run_ours(a):
 
     # ---- timed region: K rounds, device-timed on the library's stream, host sync once per round inside
     prefill_all()
+    sampler = ClockSampler(local)           # samples from the warm-up rounds on, so that short runs get several
+    sampler.start()
     for _ in range(W):
         ctx.round()
-    sampler = ClockSampler(local)
-    sampler.start()
     sync_all()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = ctx.launch_count()
@@ -326,6 +342,52 @@ def run_ours(a):
                      "mean_accept": float(np.mean([o.n_accept for o in souts])),
                      "hbm_gbs": sbytes / 1e9 / (sms / 1e3), "frac_of_measured_peak": sbytes / 1e9 / (sms / 1e3) / measured_peaks()[0]}
 
+    # ---- fixed settings LS(E, gamma) with several drafts per round (on this random model DEL itself settles at
+    # gamma = 1): the many-row verify passes and the many-row stacked head, timed and set against their bytes
+    fixed = None
+    if cfg.batch == 1 and not a.no_fixed:
+        fixed = []
+        for (fe, fg) in ((9, 6), (4, 12), (2, 4)):
+            if not (1 <= fe < cfg.n_layers and 0 <= fg <= cfg.g_max):
+                continue
+            ctx.prefill(0, prompts[0], budget)
+            ctx.set_policy(0, fe, fg)
+            for _ in range(3):
+                ctx.round()
+            torch.cuda.synchronize()
+            nf = min(K, 16)
+            Tf = ctx.committed_len(0)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(ctx.stream)
+            fouts = [ctx.round()[0] for _ in range(nf)]
+            e1.record(ctx.stream)
+            torch.cuda.synchronize()
+            fms = e0.elapsed_time(e1)
+            fbytes, ftok = 0.0, 0
+            for o in fouts:
+                fbytes += round_bytes(cfg, [(o.E, o.g, Tf)])
+                ftok += o.n_emitted
+                Tf += o.n_emitted
+            # the stacked head of these rounds alone (events around the launch)
+            ctx.set_flags(dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_TIMING)
+            ctx.kernel_times(reset=True)
+            for _ in range(4):
+                ctx.round()
+            fk = ctx.kernel_times(reset=True)
+            ctx.set_flags(dl.FLAG_PDL | dl.FLAG_TC)
+            ctx.set_policy(0, 0, 0)
+            rows = cfg.n_layers * (fg + 1)
+            hs = fk["lm_head_stacked"]
+            head_us = 1000.0 * hs["ms"] / hs["launches"] if hs["launches"] else None
+            fixed.append({"policy": f"LS(E={fe}, gamma={fg})", "ms_per_round": fms / nf, "tokens_per_round": ftok / nf,
+                          "tokens_per_s": ftok / (fms / 1e3), "algorithmic_gb_per_round": fbytes / nf / 1e9,
+                          "hbm_gbs": fbytes / 1e9 / (fms / 1e3),
+                          "frac_of_measured_peak": fbytes / 1e9 / (fms / 1e3) / measured_peaks()[0],
+                          "frac_of_8tbs": fbytes / 1e9 / (fms / 1e3) / 8000.0,
+                          "stacked_head": {"rows": rows, "us": head_us,
+                                           "tflops": 2.0 * rows * cfg.vocab * cfg.d_model / (head_us * 1e-6) / 1e12 if head_us else None,
+                                           "w_lm_gbs": cfg.lm_head_bytes() / 1e9 / (head_us * 1e-6) if head_us else None}})
+
     # ---- per-kernel durations (CUDA events around every launch; separate pass, launches serialised)
     prefill_all()
     for _ in range(3):
@@ -345,7 +407,7 @@ def run_ours(a):
     tot_ms = sum(v["ms"] for v in kt.values()) or 1.0
     for name in kernels:
         kernels[name]["share"] = kt[name]["ms"] / tot_ms
-    stream_classes = ["qkv_rope", "o_proj", "gate_up", "down", "lm_head_draft", "lm_head_stacked"]
+    stream_classes = ["qkv_rope", "o_proj", "gate_up", "down", "lm_head_draft"]      # every launch of rowgemm_kernel
     sb = sum(kt[n]["bytes"] for n in stream_classes)
     sm_ = sum(kt[n]["ms"] for n in stream_classes) or 1.0
     sl = sum(kt[n]["launches"] for n in stream_classes) or 1
@@ -353,18 +415,23 @@ def run_ours(a):
     roofline = {"bound": "hbm", "kernel": "rowgemm_kernel (weight-streaming skinny GEMM, all epilogues)",
                 "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
                 "bytes_per_launch": sb / sl, "avg_us": 1000.0 * sm_ / sl,
-                # DRAM read+write per launch from the ncu capture of the same kernels (profiles/
-                # round_kernels_m1_llama2_7b_layer.txt): 1.000-1.001 x the weight bytes read plus the ~3 MB of
-                # activation / partial writes ncu attributes to a launch
+                # not measured in this run: the ncu capture of the same kernels on a 4-layer model of this layer shape
+                # gave DRAM read = 1.000-1.001 x the weight bytes plus ~3 MB of writes per launch; scaled to this
+                # run's bytes per launch
                 "traffic": (sb / sl) * 1.0005 + 3.5e6,
+                "traffic_source": "profiles/round_kernels_m1_llama2_7b_layer.txt (ncu dram__bytes_read/write per launch, "
+                                  "ratio to algorithmic bytes 1.000-1.001), scaled; not captured live",
+                "timing": "CUDA events around each launch in a separate pass (launches serialised, no overlap "
+                          "between kernels); the pipelined figure is round.hbm_gbs",
                 "share_of_round": sm_ / tot_ms}
 
     line = {
         "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": dev_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": workload_name(cfg), "l2": "inputs larger than L2 (weights streamed every pass)",
-                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "config": bench_config(cfg, world),
+        "note": "value follows the accept trajectory of the random model (a low-margin arg-max that falls the other way "
+                "changes every later round); round.frac_of_measured_peak and vanilla are the trajectory-free figures",
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
         "round": {"tokens_per_round": tokens / (K * world), "wall_ms_per_step": 1000.0 * wall / K,
                   "algorithmic_gb_per_round": bytes_total / (K * world) / 1e9,
@@ -378,12 +445,13 @@ def run_ours(a):
                     "frac_of_measured_peak": vanilla_bytes / 1e9 / (vanilla_ms / 1e3) / peak},
         "draft_exiting": exit_info,
         "sampling": samp_info,
+        "fixed_policy": fixed,
         "kernels": kernels,
         "paper_context": "paper reports 2.16x-2.62x over auto-regressive decoding (A100-40GB / H100-PCIe, trained "
                          "LayerSkip checkpoints); not comparable to this random-weight model",
     }
     if rank == 0 and world == 1 and not a.no_cpu:
-        cb, _ = oracle_sample(cfg, weights, a.cpu_seconds)
+        cb, _ = oracle_rounds(cfg, weights, 1, seconds=a.cpu_seconds)
         line["cpu_baseline"] = cb
     elif rank == 0:
         line["cpu_baseline"] = None
@@ -392,6 +460,53 @@ def run_ours(a):
     ctx.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_profile_case(a):
+    """A few rounds of a model with the layer shape of the named configuration but few layers, so that the device
+    holds a couple of GB: the case the ncu captures under profiles/ run (a profiler replays every captured launch
+    dozens of times and saves the device memory around the passes).  Prints per-kernel-class device times."""
+    import torch
+    import paper_2504_05598_b200 as dl
+    base = synth.CONFIGS[a.config]
+    L = a.layers
+    cfg = synth.small_variant(base, n_layers=L, e_min=min(base.e_min, L - 1), e_max=min(base.e_max, L - 1),
+                              prompt_len=a.prompt, gen_len=a.rounds * (base.g_max + 1) + 8)
+    w = synth.make_weights(cfg)
+    ctx = dl.DelContext(dl.make_shape(cfg), dl.upload_weights(w))
+    for s in range(cfg.batch):
+        if a.sampling:
+            T, top_p = (float(v) for v in a.sampling.split(","))
+            ctx.set_sampling(s, T, top_p, 1234 + s)
+        ctx.prefill(s, synth.make_prompt(cfg, s), cfg.gen_len)
+        if a.policy:
+            E, G = (int(v) for v in a.policy.split(","))
+            ctx.set_policy(s, E, G)
+    flags = (0 if a.no_pdl else dl.FLAG_PDL) | (dl.FLAG_ONECTA if a.one_cta else 0) | (0 if a.no_tc else dl.FLAG_TC) | \
+        (dl.FLAG_TRIM_ROWS if a.trim else 0)
+    ctx.set_flags(flags)
+    ctx.round()
+    ctx.round()
+    if not a.no_timing:
+        ctx.set_flags(flags | dl.FLAG_TIMING)
+    ctx.kernel_times(reset=True)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(ctx.stream)
+    hist = []
+    for _ in range(a.rounds):
+        o = ctx.round()[0]
+        hist.append((o.E, o.g, o.n_accept))
+    ev1.record(ctx.stream)
+    torch.cuda.synchronize()
+    kt = ctx.kernel_times(reset=True)
+    rep = {"profile_case": f"{cfg.name} with {L} layers", "ms_per_round": ev0.elapsed_time(ev1) / a.rounds, "rounds": hist,
+           "kernels": {}}
+    for k, v in kt.items():
+        if v["launches"]:
+            rep["kernels"][k] = {"launches": v["launches"], "avg_us": round(1000 * v["ms"] / v["launches"], 2),
+                                 "gbs": round(v["bytes"] / 1e9 / (v["ms"] / 1e3), 1) if v["bytes"] else None}
+    print(json.dumps(rep))
+    ctx.close()
 
 
 def main():
@@ -403,8 +518,23 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-fixed", action="store_true", help="skip the fixed-policy block")
+    # --profile-case: the small case of the ncu captures (no JSON bench line)
+    ap.add_argument("--profile-case", action="store_true")
+    ap.add_argument("--layers", type=int, default=4)
+    ap.add_argument("--rounds", type=int, default=8)
+    ap.add_argument("--prompt", type=int, default=512)
+    ap.add_argument("--policy", default="", help="E,G: fixed setting instead of the dynamic one")
+    ap.add_argument("--sampling", default="", help="T,top_p: speculative sampling instead of greedy verification")
+    ap.add_argument("--no-timing", action="store_true")
+    ap.add_argument("--no-pdl", action="store_true")
+    ap.add_argument("--one-cta", action="store_true")
+    ap.add_argument("--no-tc", action="store_true")
+    ap.add_argument("--trim", action="store_true", help="stacked LM head over the candidate layers only")
     a = ap.parse_args()
-    if a.impl == "reference":
+    if a.profile_case:
+        run_profile_case(a)
+    elif a.impl == "reference":
         run_reference(a)
     else:
         run_ours(a)

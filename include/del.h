@@ -49,7 +49,7 @@ enum {
     DEL_EINVAL = -1,              /* bad shape, bad argument, E or gamma out of range */
     DEL_ENOSPC = -2,              /* KV pages or max_seq exhausted, workspace too small */
     DEL_ESTATE = -3,              /* call order wrong (e.g. verify before draft, round before prefill) */
-    DEL_ETIMEOUT = -4,            /* a bounded device-side wait expired (kernel reported it) */
+    DEL_ETIMEOUT = -4,            /* a bounded device-side wait expired (kernel reported it); see below */
     DEL_ECUDA = -5                /* a CUDA call failed; see del_last_cuda_error */
 };
 
@@ -262,6 +262,16 @@ int del_get_hidden(del_ctx *ctx, int seq, int layer, int row, float *out);
 int del_debug_logits(del_ctx *ctx, int seq, int layer, int row, float *out);
 int del_get_kv(del_ctx *ctx, int seq, int layer, int pos, float *k_out, float *v_out);
 
+/* DEL_ETIMEOUT.  The tensor-core kernels (stacked LM head, prefill GEMMs) wait on shared-memory barriers for
+ * their own asynchronous copies and tensor-core instructions.  Every such wait gives up after 2^26 polls
+ * (of the order of seconds to a minute, depending on the clock), records a non-zero code in the workspace's
+ * error word, lets the kernel wind down (tensor memory freed) and return.  The call that next reads results
+ * (del_prefill, del_layer_accept, del_select, del_round) then returns DEL_ETIMEOUT, clears the word, and the
+ * context stays usable: the sequence's round did not complete and should be re-prefilled.
+ * del_debug_inject_error writes `code` (non-zero) into that word with a stream-ordered copy from the host, as
+ * an expired wait would have: a test hook for the error path that makes no kernel wait. */
+int del_debug_inject_error(del_ctx *ctx, int code);
+
 /* Committed length (prompt + emitted tokens) of a sequence, or a negative code. */
 int del_committed_len(del_ctx *ctx, int seq);
 /* Frees the sequence's KV pages and marks it empty. */
@@ -298,7 +308,8 @@ int del_get_kernel_times(del_ctx *ctx, double *ms, int64_t *launches, double *by
  * allocating library routine is called.  All calls on a device share the array: calls that overlap on
  * the GPU (different streams) race, calls on one stream are safe; what a call reads from the array it
  * has written first.  The first call on each device looks up the array's device address: make that
- * call before any stream capture begins. */
+ * call before any stream capture begins.  A row whose logits are all NaN has no largest one: its entry of
+ * tokens is then 0x7fffffff, which is no token id. */
 #define DEL_STATIC_SCRATCH_BYTES ((1 << 19) + 4096)
 int del_head_argmax_static(const void *x, const void *lm_head, int rows, int vocab, int d_model, int32_t *tokens,
                            void *cuda_stream);

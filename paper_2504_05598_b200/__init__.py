@@ -28,7 +28,7 @@ EXPORTS = ["del_workspace_bytes", "del_init", "del_prefill", "del_draft", "del_v
            "del_select", "del_round", "del_set_policy", "del_get_stats", "del_set_stats", "del_get_shadow",
            "del_get_drafts", "del_force_token", "del_get_hidden", "del_debug_logits", "del_get_kv", "del_committed_len", "del_release",
            "del_launch_count", "del_get_traffic", "del_set_flags", "del_get_kernel_times", "del_head_argmax_static",
-           "del_set_policy_fs", "del_set_exit_mode", "del_get_window", "del_set_sampling", "del_get_sample_info", "del_get_round_logits", "del_sample_probe", "del_get_conf_stats", "del_set_conf_stats", "del_get_conf", "del_strerror", "del_last_cuda_error", "del_destroy"]
+           "del_set_policy_fs", "del_set_exit_mode", "del_get_window", "del_set_sampling", "del_get_sample_info", "del_get_round_logits", "del_sample_probe", "del_get_conf_stats", "del_set_conf_stats", "del_get_conf", "del_debug_inject_error", "del_strerror", "del_last_cuda_error", "del_destroy"]
 
 
 class Shape(C.Structure):
@@ -128,6 +128,8 @@ def load_library(build_if_missing: bool = True):
     L.del_debug_logits.argtypes = [vp, ci, ci, ci, vp]
     L.del_get_kv.restype = ci
     L.del_get_kv.argtypes = [vp, ci, ci, ci, vp, vp]
+    L.del_debug_inject_error.restype = ci
+    L.del_debug_inject_error.argtypes = [vp, ci]
     L.del_committed_len.restype = ci
     L.del_committed_len.argtypes = [vp, ci]
     L.del_release.restype = ci
@@ -379,6 +381,9 @@ class DelContext:
         k, v = np.zeros(n, dtype=np.float32), np.zeros(n, dtype=np.float32)
         self._ck(self.lib.del_get_kv(self._h, seq, layer, pos, k.ctypes.data, v.ctypes.data), "del_get_kv")
         return k, v
+
+    def debug_inject_error(self, code: int):
+        self._ck(self.lib.del_debug_inject_error(self._h, int(code)), "del_debug_inject_error")
 
     def committed_len(self, seq: int) -> int:
         return self.lib.del_committed_len(self._h, seq)

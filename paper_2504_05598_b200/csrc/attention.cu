@@ -20,10 +20,9 @@ template <int HD>
 __global__ void __launch_bounds__(NW * 32) attention_kernel(const __grid_constant__ AttnArgs a) {
     extern __shared__ __align__(16) float sm[];
     __shared__ int s_last;
-    pdl_launch();
-    pdl_wait();
+    pdl_launch();                  // (the wait for the producer kernel sits inside partial / partial_staged)
 
-    const AttnView v{a.D, a.B, a.layer};
+    const AttnView v{a.D, a.B, a.layer, a.early_pos[blockIdx.z]};
     const Segment seg = a.plan.seg[blockIdx.z];
     const int kvh = blockIdx.y, split = blockIdx.x, n_splits = a.n_splits;
     const int n_pages = (seg.pos0 + seg.nrows + 15) >> 4;
@@ -54,11 +53,10 @@ template <int HD>
 cudaError_t launch_one(const AttnArgs &a, int n_seg, cudaStream_t st, bool pdl) {
     const size_t smem = attn::staged_smem_bytes(HD);
     auto kern = attention_kernel<HD>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static SmemAttrOnce attr;
+    {
+        cudaError_t e = attr.set(kern, (int)((int)smem));
         if (e != cudaSuccess) return e;
-        attr_done = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(a.n_splits, a.D.nkv, n_seg);

@@ -1,5 +1,7 @@
 // Device-side building blocks of the paged multi-query attention kernel (attention.cu).
 //
+// partial / partial_staged contain the kernel's wait for its producer (programmatic dependent launch): what they
+// read before it does not depend on the producer.
 //   attn::partial         one CTA walks a range of key pages for one (segment, kv head) and leaves, per
 //                         query row and head, an online-softmax state (max, sum, unnormalised output):
 //                         either as the final normalised result (one slot) or in one of several slots;
@@ -11,7 +13,7 @@
 // form 16-row tiles; the 8 warps are divided among up to 4 query tiles, and the warps of one tile walk
 // the key pages (16 tokens each) of the range in a strided fashion.  Scores and the P*V product run on
 // bf16 tensor-core MMAs with fp32 accumulation; row reductions use shuffles inside the 4-lane groups
-// that own a row.
+// that own a row.  The output is stored as a pair of bf16 values (high + low part) for the O-projection.
 //
 // Fragment layout: the MMA sums over its k index, so any permutation of k used for both operands is
 // allowed.  For Q*K^T a thread loads 16 contiguous bytes of a key row (and the same bytes of the query
@@ -26,6 +28,7 @@ struct AttnView {
     const Dims &D;
     const Buffers &B;
     int32_t layer;
+    int32_t early_pos;         // of this CTA's segment, see AttnArgs
 };
 
 namespace attn {
@@ -177,7 +180,10 @@ __device__ __forceinline__ void tile_end(TileState<HD> &ts, const AttnView &a, f
             const int c = seg.row0 + i, qh = kvh * group + hq;
             if (n_slots == 1) {
                 const float inv = 1.f / L;
-                *reinterpret_cast<uint32_t *>(a.B.ATT + (size_t)c * qdim + qh * HD + col) = pack_bf16(o0 * inv, o1 * inv);
+                uint32_t hi, lo;
+                split_bf16x2(o0 * inv, o1 * inv, hi, lo);
+                *reinterpret_cast<uint32_t *>(a.B.ATT + (size_t)c * qdim + qh * HD + col) = hi;
+                *reinterpret_cast<uint32_t *>(a.B.ATTL + (size_t)c * qdim + qh * HD + col) = lo;
             } else {
                 const size_t pi = ((size_t)c * a.D.nh + qh) * n_slots + slot;
                 *reinterpret_cast<float2 *>(a.B.APO + pi * HD + col) = make_float2(o0, o1);
@@ -225,8 +231,10 @@ __device__ __forceinline__ void tile_end(TileState<HD> &ts, const AttnView &a, f
             const int c = seg.row0 + i, qh = kvh * group + hq;
             if (n_slots == 1) {
                 const float inv = 1.f / Lv[h];
-                *reinterpret_cast<uint32_t *>(a.B.ATT + (size_t)c * qdim + qh * HD + 8 * j + 2 * t) =
-                    pack_bf16(ov2[h][0] * inv, ov2[h][1] * inv);
+                uint32_t hi, lo;
+                split_bf16x2(ov2[h][0] * inv, ov2[h][1] * inv, hi, lo);
+                *reinterpret_cast<uint32_t *>(a.B.ATT + (size_t)c * qdim + qh * HD + 8 * j + 2 * t) = hi;
+                *reinterpret_cast<uint32_t *>(a.B.ATTL + (size_t)c * qdim + qh * HD + 8 * j + 2 * t) = lo;
             } else {
                 const size_t pi = ((size_t)c * a.D.nh + qh) * n_slots + slot;
                 *reinterpret_cast<float2 *>(a.B.APO + pi * HD + 8 * j + 2 * t) = make_float2(ov2[h][0], ov2[h][1]);
@@ -255,12 +263,34 @@ __device__ __forceinline__ void partial(const AttnView &a, float *sm, const Segm
     const int n_iter = (n_mt + P - 1) / P;
     const int key0 = 4 * (g >> 1) + (g & 1);        // token of score-tile 0 column g; tile 1: +2
 
+    // Keys and values of positions committed in earlier rounds (below a.early_pos) cannot change any more: every
+    // warp requests its first such page before it waits for the producer kernel, so that the cache's round trip to
+    // memory runs during the producer's tail.
+    const int p_first = p_begin + kl;
+    const bool pre = n_iter == 1 && p_first < p_end && p_first < (a.early_pos >> 4);
+    uint4 kf0[2][KS];
+    uint2 vf0[NJ];
+    if (pre) {
+        const int pg0 = pt[p_first];
+        const bf16 *kpage = a.B.KP + (size_t)pg0 * page_stride + head_off;
+        const bf16 *vpage = a.B.VP + (size_t)pg0 * page_stride + head_off;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            kf0[0][ks] = ldg_act16(kpage + key0 * HD + 32 * ks + 8 * t);
+            kf0[1][ks] = ldg_act16(kpage + (key0 + 2) * HD + 32 * ks + 8 * t);
+        }
+#pragma unroll
+        for (int j = 0; j < NJ; ++j) vf0[j] = ldg_act8(vpage + (8 * j + g) * 16 + 4 * t);
+    }
+    pdl_wait();
+
     for (int it = 0; it < n_iter; ++it) {
         const int mt = it * P + warp % P;
         TileState<HD> ts;
         tile_begin<HD>(ts, a, seg, kvh, mt, n_mt, k_hi);
         if (mt < n_mt) {
-            for (int pb = p_begin + kl; pb < p_end; pb += n_kl * PG) {
+            if (pre) page_update<HD>(ts, kf0, vf0, p_first, k_lo, sc);
+            for (int pb = p_first + (pre ? n_kl : 0); pb < p_end; pb += n_kl * PG) {
                 int pgs[PG];
 #pragma unroll
                 for (int q = 0; q < PG; ++q) {
@@ -333,6 +363,7 @@ __device__ __forceinline__ void partial_staged(const AttnView &a, unsigned char 
     const int n_pages = max(p_end - p_begin, 0), n_chunks = (n_pages + CH - 1) / CH;
     const int n_iter = (n_mt + P - 1) / P;          // groups of P concurrent query tiles; each group stages the pages again
 
+    pdl_wait();
     // every thread copies the same pieces of every page: 2*HD 16-byte pieces of keys, 2*HD of values
     auto issue = [&](int c) {
         if (c < n_chunks) {
@@ -448,10 +479,13 @@ __device__ __forceinline__ void merge_slots_n(const AttnView &a, const Segment s
                 o2 += f * __uint_as_float(ovv[u][s].z); o3 += f * __uint_as_float(ovv[u][s].w);
             }
             const float inv = 1.f / l;
-            uint2 pk;
-            pk.x = pack_bf16(o0 * inv, o1 * inv);
-            pk.y = pack_bf16(o2 * inv, o3 * inv);
-            if (live[u]) *reinterpret_cast<uint2 *>(a.B.ATT + out_off[u]) = pk;
+            uint2 pk, pl;
+            split_bf16x2(o0 * inv, o1 * inv, pk.x, pl.x);
+            split_bf16x2(o2 * inv, o3 * inv, pk.y, pl.y);
+            if (live[u]) {
+                *reinterpret_cast<uint2 *>(a.B.ATT + out_off[u]) = pk;
+                *reinterpret_cast<uint2 *>(a.B.ATTL + out_off[u]) = pl;
+            }
         }
     }
 }

@@ -8,6 +8,7 @@
 #include <stdint.h>
 
 #define DEL_ROWS_MAX 64        // rows of one layer pass
+#define DEL_GEMM_ROWS 32       // rows one launch of a layer GEMM serves (each row takes two MMA columns)
 #define DEL_SEQ_MAX 16         // sequences per context
 #define DEL_GEMM_THREADS 256
 #define DEL_GEMM_WARPS 8
@@ -70,15 +71,18 @@ struct Dims {
 
 struct Buffers {
     float *H;                    // [L+1][B][S][d]    hidden stack (layer 0 = embedding)
-    bf16 *XS;                    // [L+1][B][S][d]    h * gain of the next layer's attention norm
+    bf16 *XS;                    // [L+1][B][S][d]    h * gain of the next layer's attention norm (high part)
+    // Every GEMM input is kept as a pair of bf16 arrays: x ~ hi + lo with hi = bf16(x), lo = bf16(x - hi), i.e.
+    // 16 bits of mantissa.  The low parts have the layout of their high parts.
+    bf16 *XSL;                   // low part of XS
     float *SS;                   // [L+1][B][S][n_sst] partial sums of squares of h
     bf16 *XE;                    // [B][S][d]         h * gain of the final norm at the exit layer
-    bf16 *Q;                     // [ROWS][nh*hd]
-    bf16 *ATT;                   // [ROWS][nh*hd]
+    bf16 *Q, *QL;                // [ROWS][nh*hd]     queries after the rotary embedding, high and low part
+    bf16 *ATT, *ATTL;            // [ROWS][nh*hd]     attention output, high and low part
     float *HM;                   // [ROWS][d]         residual after attention
-    bf16 *XM;                    // [ROWS][d]         HM * gain of the ffn norm
+    bf16 *XM, *XML;              // [ROWS][d]         HM * gain of the ffn norm, high and low part
     float *SSM;                  // [ROWS][n_sst]
-    bf16 *ACT;                   // [ROWS][F]
+    bf16 *ACT, *ACTL;            // [ROWS][F]         silu(gate) * up, high and low part
     float *APO;                  // attention partial outputs [ROWS][nh][splits][hd]
     float *APML;                 // attention partial (max, sum) [ROWS][nh][splits][2]
     int32_t *ACNT;               // [DEL_SEQ_MAX][nkv] arrival counters of the split combine
@@ -189,6 +193,18 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
+}
+// x as a pair of bf16 values: hi = bf16(x), lo = bf16(x - hi); hi + lo carries 16 bits of x's mantissa
+__device__ __forceinline__ void split_bf16(float x, bf16 &hi, bf16 &lo) {
+    hi = __float2bfloat16_rn(x);
+    lo = __float2bfloat16_rn(x - __bfloat162float(hi));
+}
+// two values: packed high parts (element 0 in the low half-word) and packed low parts
+__device__ __forceinline__ void split_bf16x2(float x0, float x1, uint32_t &hi, uint32_t &lo) {
+    const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - __low2float(h), x1 - __high2float(h));
+    hi = *reinterpret_cast<const uint32_t *>(&h);
+    lo = *reinterpret_cast<const uint32_t *>(&l);
 }
 __device__ __forceinline__ float bf16_bits_to_float(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
 __device__ __forceinline__ float bf16_to_f(bf16 v) { return __bfloat162float(v); }

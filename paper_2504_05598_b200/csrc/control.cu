@@ -27,12 +27,12 @@ __device__ __forceinline__ void write_embedding(const CtlArgs &a, int token, int
         for (int r = 0; r < 2; ++r) {
             const uint32_t ew[4] = {ev[r].x, ev[r].y, ev[r].z, ev[r].w}, gw[4] = {gv[r].x, gv[r].y, gv[r].z, gv[r].w};
             float h[8], ss = 0.f;
-            uint32_t xs[4];
+            uint32_t xs[4], xl[4];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 h[2 * q] = __uint_as_float(ew[q] << 16);
                 h[2 * q + 1] = __uint_as_float(ew[q] & 0xffff0000u);
-                xs[q] = pack_bf16(h[2 * q] * __uint_as_float(gw[q] << 16), h[2 * q + 1] * __uint_as_float(gw[q] & 0xffff0000u));
+                split_bf16x2(h[2 * q] * __uint_as_float(gw[q] << 16), h[2 * q + 1] * __uint_as_float(gw[q] & 0xffff0000u), xs[q], xl[q]);
                 ss += h[2 * q] * h[2 * q] + h[2 * q + 1] * h[2 * q + 1];
             }
             ss += __shfl_xor_sync(0xffffffffu, ss, 1);
@@ -41,6 +41,7 @@ __device__ __forceinline__ void write_embedding(const CtlArgs &a, int token, int
                 hp[0] = make_float4(h[0], h[1], h[2], h[3]);
                 hp[1] = make_float4(h[4], h[5], h[6], h[7]);
                 *reinterpret_cast<uint4 *>(a.B.XS + sr * d + o[r]) = make_uint4(xs[0], xs[1], xs[2], xs[3]);
+                *reinterpret_cast<uint4 *>(a.B.XSL + sr * d + o[r]) = make_uint4(xl[0], xl[1], xl[2], xl[3]);
                 if ((threadIdx.x & 1) == 0) a.B.SS[sr * a.D.n_sst + (o[r] >> 4)] = ss;
             }
         }

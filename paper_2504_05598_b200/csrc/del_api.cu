@@ -57,6 +57,7 @@ struct del_ctx {
     cudaStream_t st = nullptr;
     int n_sms = 148;
     int flags = FLAG_PDL | FLAG_TC;
+    bool in_round = false;               // the passes being enqueued belong to a decode round (not to a prefill)
     SeqHost seq[DEL_SEQ_MAX];
     std::vector<int> free_pages;
     std::vector<int32_t> pt_host;
@@ -72,7 +73,8 @@ struct del_ctx {
     // bulk prefill on the tensor cores: chunk buffers in the workspace, tensor maps of them and of every layer's weights
     struct TMap { alignas(64) unsigned char b[128]; };
     PfArgs pf;                                            // buffer pointers (the per-launch fields are filled in later)
-    TMap pf_xs, pf_att, pf_xm, pf_act;
+    TMap pf_xs, pf_att, pf_xm, pf_act;                    // activation buffers, high parts ...
+    TMap pf_xsl, pf_attl, pf_xml, pf_actl;                // ... and low parts
     std::vector<TMap> pf_wq, pf_wk, pf_wv, pf_wo, pf_wg, pf_wu, pf_wd;
     bool pf_ok = false;
     // mailbox of the draft loop's confidence check: pinned host memory that the finalise kernel writes directly
@@ -115,14 +117,19 @@ size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max
     Carve c;
     B.H = c.take<float>(base, L1 * BS * D.d);
     B.XS = c.take<bf16>(base, L1 * BS * D.d);
+    B.XSL = c.take<bf16>(base, L1 * BS * D.d);
     B.SS = c.take<float>(base, L1 * BS * D.n_sst);
     B.XE = c.take<bf16>(base, BS * D.d);
     B.Q = c.take<bf16>(base, DEL_ROWS_MAX * qd);
+    B.QL = c.take<bf16>(base, DEL_ROWS_MAX * qd);
     B.ATT = c.take<bf16>(base, DEL_ROWS_MAX * qd);
+    B.ATTL = c.take<bf16>(base, DEL_ROWS_MAX * qd);
     B.HM = c.take<float>(base, (size_t)DEL_ROWS_MAX * D.d);
     B.XM = c.take<bf16>(base, (size_t)DEL_ROWS_MAX * D.d);
+    B.XML = c.take<bf16>(base, (size_t)DEL_ROWS_MAX * D.d);
     B.SSM = c.take<float>(base, (size_t)DEL_ROWS_MAX * D.n_sst);
     B.ACT = c.take<bf16>(base, (size_t)DEL_ROWS_MAX * D.F);
+    B.ACTL = c.take<bf16>(base, (size_t)DEL_ROWS_MAX * D.F);
     B.APO = c.take<float>(base, (size_t)DEL_ROWS_MAX * D.nh * 16 * D.hd);
     B.APML = c.take<float>(base, (size_t)DEL_ROWS_MAX * D.nh * 16 * 2);
     B.ACNT = c.take<int32_t>(base, (size_t)DEL_SEQ_MAX * D.nkv);
@@ -162,12 +169,17 @@ size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max
     pfa.n_ssp = prefill_tc_nssp(D);
     pfa.H = c.take<float>(base, (size_t)PF_ROWS * D.d);
     pfa.XS = c.take<bf16>(base, (size_t)PF_ROWS * D.d);
+    pfa.XSL = c.take<bf16>(base, (size_t)PF_ROWS * D.d);
     pfa.SSP = c.take<float>(base, (size_t)PF_ROWS * pfa.n_ssp);
     pfa.Q = c.take<bf16>(base, (size_t)PF_ROWS * qd);
+    pfa.QL = c.take<bf16>(base, (size_t)PF_ROWS * qd);
     pfa.ATT = c.take<bf16>(base, (size_t)PF_ROWS * qd);
+    pfa.ATTL = c.take<bf16>(base, (size_t)PF_ROWS * qd);
     pfa.XM = c.take<bf16>(base, (size_t)PF_ROWS * D.d);
+    pfa.XML = c.take<bf16>(base, (size_t)PF_ROWS * D.d);
     pfa.SSPM = c.take<float>(base, (size_t)PF_ROWS * pfa.n_ssp);
     pfa.ACT = c.take<bf16>(base, (size_t)PF_ROWS * D.F);
+    pfa.ACTL = c.take<bf16>(base, (size_t)PF_ROWS * D.F);
     if (pf) *pf = pfa;
     return (c.off + 255) & ~(size_t)255;
 }
@@ -328,6 +340,7 @@ GemmArgs gemm_base(del_ctx *c, int plan_idx, int layer) {
     GemmArgs a;
     memset(&a, 0, sizeof(a));
     a.tile_ctr = next_counter(c);
+    a.ctas_per_sm = (c->flags & FLAG_ONECTA) ? 1 : 2;
     a.D = c->D;
     a.B = c->B;
     a.plan = c->plan_host[plan_idx];
@@ -374,10 +387,13 @@ int run_layer(del_ctx *c, const PassInfo &pi, int l, bool write_exit) {
         GemmArgs a = gemm_base(c, pi.plan_idx, l);
         a.K = D.d;
         a.n_items = (D.nh + 2 * D.nkv) * (D.hd / 16);
-        a.X = c->B.XS;
+        a.X = c->B.XS; a.XL = c->B.XSL;
         a.W0 = c->wq[l - 1]; a.W1 = c->wk[l - 1]; a.W2 = c->wv[l - 1];
-        TAG(CLS_QKV, 2.0 * (D.nh + 2 * D.nkv) * D.hd * D.d);
-        LAUNCH(launch_rowgemm(EPI_QKV, a, pi.m, c->n_sms, c->st, P));
+        for (a.row0 = 0; a.row0 < pi.m; a.row0 += DEL_GEMM_ROWS) {
+            if (a.row0) a.tile_ctr = next_counter(c);
+            TAG(CLS_QKV, 2.0 * (D.nh + 2 * D.nkv) * D.hd * D.d);
+            LAUNCH(launch_rowgemm(EPI_QKV, a, pi.m, c->n_sms, c->st, P));
+        }
     }
     {
         AttnArgs a;
@@ -388,6 +404,8 @@ int run_layer(del_ctx *c, const PassInfo &pi, int l, bool write_exit) {
         const int ns = attention_splits(pages, pi.n_seg * D.nkv, n_mt >= 3 ? 4 : n_mt, c->n_sms);
         a.n_splits = ns;
         a.max_rows = pi.max_rows;
+        if (c->in_round)            // what earlier rounds committed is final (the host has synchronised since)
+            for (int i = 0; i < pi.n_seg; ++i) a.early_pos[i] = c->seq[c->plan_host[pi.plan_idx].seg[i].seq].T;
         {
             double kvb = 0.0;
             const PassPlan &pp = c->plan_host[pi.plan_idx];
@@ -400,31 +418,40 @@ int run_layer(del_ctx *c, const PassInfo &pi, int l, bool write_exit) {
         GemmArgs a = gemm_base(c, pi.plan_idx, l);
         a.K = D.nh * D.hd;
         a.n_items = D.d / 16;
-        a.X = c->B.ATT;
+        a.X = c->B.ATT; a.XL = c->B.ATTL;
         a.W0 = c->wo[l - 1];
         a.gain_a = c->ffn_norm[l - 1];
-        TAG(CLS_OPROJ, 2.0 * D.d * D.nh * D.hd);
-        LAUNCH(launch_rowgemm(EPI_OPROJ, a, pi.m, c->n_sms, c->st, P));
+        for (a.row0 = 0; a.row0 < pi.m; a.row0 += DEL_GEMM_ROWS) {
+            if (a.row0) a.tile_ctr = next_counter(c);
+            TAG(CLS_OPROJ, 2.0 * D.d * D.nh * D.hd);
+            LAUNCH(launch_rowgemm(EPI_OPROJ, a, pi.m, c->n_sms, c->st, P));
+        }
     }
     {
         GemmArgs a = gemm_base(c, pi.plan_idx, l);
         a.K = D.d;
         a.n_items = D.F / 8;
-        a.X = c->B.XM;
+        a.X = c->B.XM; a.XL = c->B.XML;
         a.W0 = c->w_gate[l - 1]; a.W1 = c->w_up[l - 1];
-        TAG(CLS_GATEUP, 4.0 * D.F * D.d);
-        LAUNCH(launch_rowgemm(EPI_GATEUP, a, pi.m, c->n_sms, c->st, P));
+        for (a.row0 = 0; a.row0 < pi.m; a.row0 += DEL_GEMM_ROWS) {
+            if (a.row0) a.tile_ctr = next_counter(c);
+            TAG(CLS_GATEUP, 4.0 * D.F * D.d);
+            LAUNCH(launch_rowgemm(EPI_GATEUP, a, pi.m, c->n_sms, c->st, P));
+        }
     }
     {
         GemmArgs a = gemm_base(c, pi.plan_idx, l);
         a.K = D.F;
         a.n_items = D.d / 16;
-        a.X = c->B.ACT;
+        a.X = c->B.ACT; a.XL = c->B.ACTL;
         a.W0 = c->w_down[l - 1];
         a.gain_a = l < D.L ? c->attn_norm[l] : nullptr;
         a.gain_b = write_exit ? c->final_norm : nullptr;
-        TAG(CLS_DOWN, 2.0 * D.d * D.F);
-        LAUNCH(launch_rowgemm(EPI_DOWN, a, pi.m, c->n_sms, c->st, P));
+        for (a.row0 = 0; a.row0 < pi.m; a.row0 += DEL_GEMM_ROWS) {
+            if (a.row0) a.tile_ctr = next_counter(c);
+            TAG(CLS_DOWN, 2.0 * D.d * D.F);
+            LAUNCH(launch_rowgemm(EPI_DOWN, a, pi.m, c->n_sms, c->st, P));
+        }
     }
     return DEL_OK;
 }
@@ -510,7 +537,7 @@ int launch_draft_step(del_ctx *c, const DraftStep &st, const std::vector<int> &E
     TAG(CLS_LMHEAD, 2.0 * c->D.V * c->D.d);
     LAUNCH(launch_rowgemm(EPI_LMHEAD, a, full.m, c->n_sms, c->st, P));
     CtlArgs ca = ctl_base(c, full.plan_idx);
-    ca.n_part = rowgemm_lmhead_grid(a.n_items, full.m, c->n_sms);
+    ca.n_part = rowgemm_lmhead_grid(a.n_items, full.m, c->n_sms, a.ctas_per_sm);
     if (stamp != 0 && c->post_conf != nullptr) {
         ca.post_conf = c->post_conf;
         ca.post_stamp = c->post_stamp;
@@ -648,14 +675,14 @@ int prefill_bulk(del_ctx *c, int sq, int n_pos, int win0) {
             a.layer = l;
             a.K = D.d;
             a.n_ntiles = prefill_tc_ntiles(PF_QKV, D);
-            LAUNCH(launch_prefill_gemm(PF_QKV, c->pf_xs.b, c->pf_wq[l - 1].b, c->pf_wk[l - 1].b, c->pf_wv[l - 1].b, a, c->n_sms, c->st, P));
+            LAUNCH(launch_prefill_gemm(PF_QKV, c->pf_xs.b, c->pf_xsl.b, c->pf_wq[l - 1].b, c->pf_wk[l - 1].b, c->pf_wv[l - 1].b, a, c->n_sms, c->st, P));
             if (l == D.L && !has_window) break;       // of the last layer only the keys and values are needed
             if (!(c->flags & FLAG_DECODE_ATTN_PREFILL)) {
                 // one flash-style pass over the chunk's rows and all keys up to each row's position
                 PfAttnArgs pa;
                 memset(&pa, 0, sizeof(pa));
                 pa.D = D;
-                pa.Q = a.Q; pa.ATT = a.ATT;
+                pa.Q = a.Q; pa.QL = a.QL; pa.ATT = a.ATT; pa.ATTL = a.ATTL;
                 pa.KP = c->B.KP; pa.VP = c->B.VP; pa.PT = c->B.PT;
                 pa.M = a.M; pa.layer = l; pa.seq = sq; pa.pos0 = p0;
                 LAUNCH(launch_prefill_attention(pa, c->st, P));
@@ -666,7 +693,9 @@ int prefill_bulk(del_ctx *c, int sq, int n_pos, int win0) {
                 at.D = D;
                 at.B = c->B;
                 at.B.Q = a.Q + (size_t)r0 * D.nh * D.hd;
+                at.B.QL = a.QL + (size_t)r0 * D.nh * D.hd;
                 at.B.ATT = a.ATT + (size_t)r0 * D.nh * D.hd;
+                at.B.ATTL = a.ATTL + (size_t)r0 * D.nh * D.hd;
                 const int nr = std::min(DEL_ROWS_MAX, a.M - r0);
                 at.plan.m = nr;
                 at.plan.n_seg = 1;
@@ -681,14 +710,14 @@ int prefill_bulk(del_ctx *c, int sq, int n_pos, int win0) {
             a.K = D.nh * D.hd;
             a.n_ntiles = prefill_tc_ntiles(PF_OPROJ, D);
             a.gain = c->ffn_norm[l - 1];
-            LAUNCH(launch_prefill_gemm(PF_OPROJ, c->pf_att.b, c->pf_wo[l - 1].b, nullptr, nullptr, a, c->n_sms, c->st, P));
+            LAUNCH(launch_prefill_gemm(PF_OPROJ, c->pf_att.b, c->pf_attl.b, c->pf_wo[l - 1].b, nullptr, nullptr, a, c->n_sms, c->st, P));
             a.K = D.d;
             a.n_ntiles = prefill_tc_ntiles(PF_GATEUP, D);
-            LAUNCH(launch_prefill_gemm(PF_GATEUP, c->pf_xm.b, c->pf_wg[l - 1].b, c->pf_wu[l - 1].b, nullptr, a, c->n_sms, c->st, P));
+            LAUNCH(launch_prefill_gemm(PF_GATEUP, c->pf_xm.b, c->pf_xml.b, c->pf_wg[l - 1].b, c->pf_wu[l - 1].b, nullptr, a, c->n_sms, c->st, P));
             a.K = D.F;
             a.n_ntiles = prefill_tc_ntiles(PF_DOWN, D);
             a.gain = l < D.L ? c->attn_norm[l] : nullptr;      // the next layer's attention norm
-            LAUNCH(launch_prefill_gemm(PF_DOWN, c->pf_act.b, c->pf_wd[l - 1].b, nullptr, nullptr, a, c->n_sms, c->st, P));
+            LAUNCH(launch_prefill_gemm(PF_DOWN, c->pf_act.b, c->pf_actl.b, c->pf_wd[l - 1].b, nullptr, nullptr, a, c->n_sms, c->st, P));
         }
     }
     return DEL_OK;
@@ -879,7 +908,7 @@ int enqueue_update(del_ctx *c, const std::vector<Job> &jobs, int mode, int W, bo
         a.row_scale = c->B.RS + (size_t)k * DEL_ROWS_MAX;
         TAG(CLS_LMSTACK, 2.0 * c->D.V * c->D.d);
         LAUNCH(launch_rowgemm(EPI_LMHEAD, a, m, c->n_sms, c->st, P));
-        const int n_part = rowgemm_lmhead_grid(a.n_items, m, c->n_sms);
+        const int n_part = rowgemm_lmhead_grid(a.n_items, m, c->n_sms, a.ctas_per_sm);
         LAUNCH(launch_shadow_reduce(ca, up, c->B.LPV, c->B.LPI, c->B.LPS, n_part, DEL_ROWS_MAX, 1, k * DEL_ROWS_MAX, m,
                                     c->st, P));
     }
@@ -1024,7 +1053,11 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
         bool ok = lmhead_tc_make_map(c->pf_xs.b, c->pf.XS, PF_ROWS, d, 128) == 0 &&
                   lmhead_tc_make_map(c->pf_att.b, c->pf.ATT, PF_ROWS, qd, 128) == 0 &&
                   lmhead_tc_make_map(c->pf_xm.b, c->pf.XM, PF_ROWS, d, 128) == 0 &&
-                  lmhead_tc_make_map(c->pf_act.b, c->pf.ACT, PF_ROWS, F, 128) == 0;
+                  lmhead_tc_make_map(c->pf_act.b, c->pf.ACT, PF_ROWS, F, 128) == 0 &&
+                  lmhead_tc_make_map(c->pf_xsl.b, c->pf.XSL, PF_ROWS, d, 128) == 0 &&
+                  lmhead_tc_make_map(c->pf_attl.b, c->pf.ATTL, PF_ROWS, qd, 128) == 0 &&
+                  lmhead_tc_make_map(c->pf_xml.b, c->pf.XML, PF_ROWS, d, 128) == 0 &&
+                  lmhead_tc_make_map(c->pf_actl.b, c->pf.ACTL, PF_ROWS, F, 128) == 0;
         auto maps = [&](std::vector<del_ctx::TMap> &dst, const std::vector<const bf16 *> &w, uint64_t rows, uint64_t cols, uint32_t box) {
             dst.resize(L);
             for (int l = 0; l < L && ok; ++l) ok = lmhead_tc_make_map(dst[l].b, w[l], rows, cols, box) == 0;
@@ -1069,6 +1102,7 @@ int del_release(del_ctx *c, int sq) {
 
 int del_prefill(del_ctx *c, int sq, const int32_t *prompt, int n_prompt, int max_new_tokens, del_round_out *first_out) {
     if (!seq_ok(c, sq) || !prompt || n_prompt < 1 || max_new_tokens < 1) return DEL_EINVAL;
+    c->in_round = false;
     for (int i = 0; i < n_prompt; ++i)
         if (prompt[i] < 0 || prompt[i] >= c->D.V) return DEL_EINVAL;
     if (n_prompt + max_new_tokens + c->sh.g_max + 1 > c->D.max_seq) return DEL_ENOSPC;
@@ -1142,6 +1176,7 @@ int del_draft(del_ctx *c, int sq, int E, int gamma) {
     SeqHost &s = c->seq[sq];
     if (E < 1 || E >= c->D.L || gamma < 0 || gamma > c->sh.g_max) return DEL_EINVAL;
     if (!s.active || s.remaining < 1 || s.phase != 0) return DEL_ESTATE;
+    c->in_round = true;
     const int g = clip_gamma(s, gamma);
     int rc = ensure_pages(c, sq, s.T + g + 1);
     if (rc) return rc;
@@ -1158,6 +1193,7 @@ int del_verify(del_ctx *c, int sq) {
     if (!seq_ok(c, sq)) return DEL_EINVAL;
     SeqHost &s = c->seq[sq];
     if (!s.active || s.phase != 1) return DEL_ESTATE;
+    c->in_round = true;
     int rc = enqueue_verify(c, {Job{sq, s.cur_E, s.cur_g, s.cur_stopped}});
     if (rc) return rc;
     s.phase = 2;
@@ -1216,6 +1252,7 @@ int del_select(del_ctx *c, int sq, int32_t *E, int32_t *gamma) {
 
 int del_round(del_ctx *c, del_round_out *out) {
     if (!c || !out) return DEL_EINVAL;
+    c->in_round = true;
     std::vector<Job> jobs;
     bool any_exit = false;
     for (int sq = 0; sq < c->D.B; ++sq) {
@@ -1495,6 +1532,15 @@ int del_get_kv(del_ctx *c, int sq, int layer, int pos, float *k_out, float *v_ou
     return DEL_OK;
 }
 
+int del_debug_inject_error(del_ctx *c, int code) {
+    if (!c || code == 0) return DEL_EINVAL;
+    int32_t *src = reinterpret_cast<int32_t *>(c->stage_host) + 4096;     // pinned: the copy is stream-ordered
+    *src = code;
+    CK(cudaMemcpyAsync(c->B.ERR, src, sizeof(int32_t), cudaMemcpyHostToDevice, c->st));
+    CK(cudaStreamSynchronize(c->st));
+    return DEL_OK;
+}
+
 int del_committed_len(del_ctx *c, int sq) {
     if (!seq_ok(c, sq)) return DEL_EINVAL;
     return c->seq[sq].active ? c->seq[sq].T : DEL_ESTATE;
@@ -1524,7 +1570,6 @@ int del_set_flags(del_ctx *c, int flags) {
     if (!c) return DEL_EINVAL;
     const int old = c->flags;
     c->flags = flags;
-    rowgemm_set_ctas_per_sm((flags & FLAG_ONECTA) ? 1 : 2);
     return old;
 }
 

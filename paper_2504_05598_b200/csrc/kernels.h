@@ -3,6 +3,22 @@
 
 #include "common.cuh"
 
+// cudaFuncSetAttribute acts on the current device only: a kernel's dynamic shared-memory limit is raised once per
+// device (a process may drive contexts on several GPUs).  `done` is the caller's static per-kernel record.
+#define DEL_MAX_DEVICES 64
+struct SmemAttrOnce {
+    bool done[DEL_MAX_DEVICES] = {};
+    template <typename K> cudaError_t set(K kern, int bytes) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < DEL_MAX_DEVICES && done[dev]) return cudaSuccess;
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e == cudaSuccess && dev >= 0 && dev < DEL_MAX_DEVICES) done[dev] = true;
+        return e;
+    }
+};
+
 enum { EPI_QKV = 0, EPI_OPROJ = 1, EPI_GATEUP = 2, EPI_DOWN = 3, EPI_LMHEAD = 4 };
 
 struct GemmArgs {
@@ -13,8 +29,11 @@ struct GemmArgs {
     int32_t K;                 // in-features
     int32_t n_items;           // work items: tile pairs (QKV, GATEUP) or 16-row tiles
     const bf16 *X;             // activations (see rowgemm.cu for the indexing per epilogue)
+    const bf16 *XL;            // their low parts (layer GEMMs; the LM head takes single bf16 rows)
+    int32_t row0;              // layer GEMMs: first row of the pass this launch handles (a launch takes up to 32 rows)
     const bf16 *W0, *W1, *W2;
     const bf16 *gain_a, *gain_b;
+    int32_t ctas_per_sm;       // weight-streaming CTAs per SM for passes of up to 8 rows: 1 or 2 (0: 2)
     int32_t *tile_ctr;         // per-launch zeroed counter for dynamic tile claims (nullptr: static round-robin)
     int32_t x_by_row;          // LMHEAD: activations are X[c] (stacked rows) instead of XE[seq][slot]
     const float *row_scale;    // LMHEAD with x_by_row: log2(e) / rms per row (nullptr: taken from B.SSE)
@@ -23,8 +42,8 @@ struct GemmArgs {
 };
 
 cudaError_t launch_rowgemm(int epi, const GemmArgs &a, int m, int n_sms, cudaStream_t st, bool pdl);
-int rowgemm_lmhead_grid(int n_items, int m, int n_sms);
-void rowgemm_set_ctas_per_sm(int n);
+// CTAs an LM-head launch of m rows uses (= number of arg-max partials it leaves per row)
+int rowgemm_lmhead_grid(int n_items, int m, int n_sms, int ctas_per_sm);
 
 struct AttnArgs {
     Dims D;
@@ -33,6 +52,11 @@ struct AttnArgs {
     int32_t layer;
     int32_t n_splits;          // key-range splits per (segment, kv head)
     int32_t max_rows;          // largest segment (rows), decides the number of query tiles
+    // Per segment: cache positions below this one were written before the host last synchronised with the stream
+    // (positions committed in earlier rounds), so the kernel may read them before it waits for its producer.
+    // Everything later may come from a launch that is still running (the wait of a launch covers its whole chain
+    // of predecessors, but nothing bounds how far ahead of that wait a dependent launch may start).  0: nothing.
+    int32_t early_pos[DEL_SEQ_MAX];
 };
 cudaError_t launch_attention(const AttnArgs &a, int n_seg, cudaStream_t st, bool pdl);
 int attention_splits(int pages, int n_units, int tiles_par, int n_sms);
@@ -138,12 +162,12 @@ struct PfArgs {
     int32_t n_ssp;             // partial sums of squares per row (= output tiles of a d-wide GEMM)
     int32_t layer, seq, pos0;  // 1-based layer; the rows are positions pos0 .. pos0 + M - 1 of sequence seq
     float *H;                  // [PF_ROWS][d] residual stream, updated in place
-    bf16 *XS;                  // [PF_ROWS][d] bf16(h * attention-norm gain): input of QKV, written by DOWN
+    bf16 *XS, *XSL;            // [PF_ROWS][d] h * attention-norm gain (high / low part): input of QKV, written by DOWN
     float *SSP;                // [PF_ROWS][n_ssp] sums of squares of h per output tile of DOWN (QKV's 1/rms)
-    bf16 *Q, *ATT;             // [PF_ROWS][nh * hd]
-    bf16 *XM;                  // [PF_ROWS][d] bf16(h_mid * ffn-norm gain), written by OPROJ
+    bf16 *Q, *QL, *ATT, *ATTL; // [PF_ROWS][nh * hd] queries, attention output (each as high / low part)
+    bf16 *XM, *XML;            // [PF_ROWS][d] h_mid * ffn-norm gain (high / low part), written by OPROJ
     float *SSPM;               // [PF_ROWS][n_ssp]
-    bf16 *ACT;                 // [PF_ROWS][F]
+    bf16 *ACT, *ACTL;          // [PF_ROWS][F] (high / low part)
     const bf16 *gain;          // OPROJ: ffn-norm gain; DOWN: the next layer's attention-norm gain
     bf16 *KP, *VP;             // paged cache
     const int32_t *PT;
@@ -163,13 +187,13 @@ int prefill_tc_nssp(const Dims &D);            // partial sums of squares per ro
 // against the paged cache of `layer` (which already holds the chunk's own keys and values) -> ATT.
 struct PfAttnArgs {
     Dims D;
-    const bf16 *Q;             // [M][nh * hd]
-    bf16 *ATT;                 // [M][nh * hd]
+    const bf16 *Q, *QL;        // [M][nh * hd] queries, high and low part
+    bf16 *ATT, *ATTL;          // [M][nh * hd] output, high and low part
     const bf16 *KP, *VP;
     const int32_t *PT;
     int32_t M, layer, seq, pos0;
 };
 cudaError_t launch_prefill_attention(const PfAttnArgs &a, cudaStream_t st, bool pdl);
-cudaError_t launch_prefill_gemm(int epi, const void *map_a, const void *map_b0, const void *map_b1, const void *map_b2,
-                                const PfArgs &p, int n_sms, cudaStream_t st, bool pdl);
+cudaError_t launch_prefill_gemm(int epi, const void *map_a, const void *map_a_lo, const void *map_b0, const void *map_b1,
+                                const void *map_b2, const PfArgs &p, int n_sms, cudaStream_t st, bool pdl);
 cudaError_t launch_prefill_embed(const PfArgs &p, const bf16 *tok_emb, const int32_t *prompt, const bf16 *gain0, cudaStream_t st);

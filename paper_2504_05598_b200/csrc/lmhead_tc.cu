@@ -244,11 +244,10 @@ cudaError_t launch_lmhead_tc(const void *map_x, const void *map_w, float *part_v
     p.n_tiles = p.n_mtiles * p.n_vtiles;
     p.err = err;
     const size_t smem = (size_t)STAGES * STAGE_BYTES + 1024;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(lmhead_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static SmemAttrOnce attr;
+    {
+        cudaError_t e = attr.set(lmhead_tc_kernel, (int)((int)smem));
         if (e != cudaSuccess) return e;
-        attr_done = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.n_tiles < n_sms ? p.n_tiles : n_sms);

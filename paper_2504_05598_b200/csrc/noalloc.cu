@@ -78,7 +78,7 @@ extern "C" int del_head_argmax_static(const void *x, const void *lm_head, int ro
     unsigned char *scratch = g_scratch_ptr[dev];
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const int n_items = vocab / 16;
-    const int n_part = rowgemm_lmhead_grid(n_items, rows, n_sms);
+    const int n_part = rowgemm_lmhead_grid(n_items, rows, n_sms, 2);
     if (n_part > MAX_CTAS) return DEL_EINVAL;                            // beyond the static scratch
 
     GemmArgs a;
@@ -90,6 +90,7 @@ extern "C" int del_head_argmax_static(const void *x, const void *lm_head, int ro
     a.X = reinterpret_cast<const bf16 *>(x);
     a.W0 = reinterpret_cast<const bf16 *>(lm_head);
     a.x_by_row = 1;
+    a.ctas_per_sm = 2;
     a.B.LPV = reinterpret_cast<float *>(scratch);
     a.B.LPI = reinterpret_cast<int32_t *>(scratch + PART_BYTES);
 

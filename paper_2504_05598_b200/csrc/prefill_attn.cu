@@ -176,20 +176,27 @@ __global__ void __launch_bounds__(PA_THREADS) prefill_attention_kernel(const __g
     const float i0 = 1.f / l0, i1 = 1.f / l1;
 #pragma unroll
     for (int j = 0; j < HD / 8; ++j) {
-        if (r0 < a.M)
-            *reinterpret_cast<uint32_t *>(a.ATT + (size_t)r0 * qdim + head * HD + 8 * j + 2 * t) = pack_bf16(O[j][0] * i0, O[j][1] * i0);
-        if (r1 < a.M)
-            *reinterpret_cast<uint32_t *>(a.ATT + (size_t)r1 * qdim + head * HD + 8 * j + 2 * t) = pack_bf16(O[j][2] * i1, O[j][3] * i1);
+        // stored as high + low bf16 parts: the O-projection takes its input as such a pair
+        uint32_t hi, lo;
+        if (r0 < a.M) {
+            split_bf16x2(O[j][0] * i0, O[j][1] * i0, hi, lo);
+            *reinterpret_cast<uint32_t *>(a.ATT + (size_t)r0 * qdim + head * HD + 8 * j + 2 * t) = hi;
+            *reinterpret_cast<uint32_t *>(a.ATTL + (size_t)r0 * qdim + head * HD + 8 * j + 2 * t) = lo;
+        }
+        if (r1 < a.M) {
+            split_bf16x2(O[j][2] * i1, O[j][3] * i1, hi, lo);
+            *reinterpret_cast<uint32_t *>(a.ATT + (size_t)r1 * qdim + head * HD + 8 * j + 2 * t) = hi;
+            *reinterpret_cast<uint32_t *>(a.ATTL + (size_t)r1 * qdim + head * HD + 8 * j + 2 * t) = lo;
+        }
     }
 }
 
 template <int HD>
 cudaError_t launch_hd(const PfAttnArgs &a, cudaStream_t st, bool pdl) {
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_attention_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<HD>::SMEM_BYTES);
+    static SmemAttrOnce attr;
+    {
+        cudaError_t e = attr.set(prefill_attention_kernel<HD>, (int)(Lay<HD>::SMEM_BYTES));
         if (e != cudaSuccess) return e;
-        attr_done = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((a.M + BQ - 1) / BQ, a.D.nh);

@@ -12,9 +12,13 @@
 // the acceptance statistics: the hidden state of those rows after every layer (and their embedding) is
 // copied into the hidden stack, where the stacked LM head finds it.
 //
+// The activations enter every GEMM as a pair of bf16 values (high + low part, see common.cuh): each k-block is
+// two MMAs on the same weight tile, one per part, into the same accumulator, so that the prompt's keys, values
+// and hidden states carry the same accuracy as those the decode kernels make.
+//
 // CTA tile 128 rows x 256 output features (128 for the two d-wide projections, whose 256-wide tiles would
 // fill less than half of the SMs), K blocks of 64 (one 128-byte swizzle span), same roles as
-// the stacked LM head: warp 0 issues TMA loads into a 4-stage shared-memory ring, warp 1 issues
+// the stacked LM head: warp 0 issues TMA loads into a 3-stage shared-memory ring, warp 1 issues
 // tcgen05.mma into one of two 256-column accumulators in tensor memory, warps 2-5 read their own row
 // with tcgen05.ld and run the epilogue while the next tile's MMAs proceed.  Ragged shapes (rows, N, K)
 // rely on TMA zero fill plus store masks.  Every mbarrier wait is bounded.
@@ -27,8 +31,9 @@ namespace {
 
 using namespace tc;
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
-constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 3;
+// a stage: high parts of the activation tile, their low parts, the weight tile
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2, STAGE_BYTES = 2 * A_BYTES + B_BYTES;
 constexpr int PF_THREADS = 192;
 // O-proj and down (N = d_model) use a narrower tile, p.bn_narrow, chosen per model shape (prefill_tc_narrow)
 template <int EPI> __device__ __forceinline__ int tile_n(const PfArgs &p) {
@@ -36,7 +41,7 @@ template <int EPI> __device__ __forceinline__ int tile_n(const PfArgs &p) {
 }
 
 struct PfMaps {
-    CUtensorMap a;             // activations [PF_ROWS, K], box 64 x 128
+    CUtensorMap a, a_lo;       // activations [PF_ROWS, K], high and low parts, box 64 x 128
     CUtensorMap b0, b1, b2;    // weights [N, K]: QKV Wq / Wk / Wv (box 64 x 256); GATEUP gate / up (box 64 x 128); else b0
 };
 
@@ -56,6 +61,19 @@ __device__ __forceinline__ void store_bf16x32(bf16 *dst, const float (&v)[32]) {
         w.z = pack_bf16(v[8 * q + 4], v[8 * q + 5]);
         w.w = pack_bf16(v[8 * q + 6], v[8 * q + 7]);
         *reinterpret_cast<uint4 *>(dst + 8 * q) = w;
+    }
+}
+// the same values as high parts to `hi` and low parts to `lo`
+__device__ __forceinline__ void store_split_x32(bf16 *hi, bf16 *lo, const float (&v)[32]) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint4 wh, wl;
+        split_bf16x2(v[8 * q + 0], v[8 * q + 1], wh.x, wl.x);
+        split_bf16x2(v[8 * q + 2], v[8 * q + 3], wh.y, wl.y);
+        split_bf16x2(v[8 * q + 4], v[8 * q + 5], wh.z, wl.z);
+        split_bf16x2(v[8 * q + 6], v[8 * q + 7], wh.w, wl.w);
+        *reinterpret_cast<uint4 *>(hi + 8 * q) = wh;
+        *reinterpret_cast<uint4 *>(lo + 8 * q) = wl;
     }
 }
 
@@ -92,11 +110,15 @@ __device__ __forceinline__ void epilogue(const PfArgs &p, uint32_t taddr, int ro
                         lo[e] = a * c - b * s;
                         hi[e] = b * c + a * s;
                     }
-                    bf16 *dst;
-                    if (which == 0) dst = p.Q + (size_t)row * (D.nh * hd) + n + jj;
-                    else dst = p.KP + ((((size_t)pg * D.L + (p.layer - 1)) * D.nkv + n / hd) * 16 + sl) * hd + jj;
-                    store_bf16x32(dst, lo);
-                    store_bf16x32(dst + half, hi);
+                    if (which == 0) {
+                        const size_t qo = (size_t)row * (D.nh * hd) + n + jj;
+                        store_split_x32(p.Q + qo, p.QL + qo, lo);
+                        store_split_x32(p.Q + qo + half, p.QL + qo + half, hi);
+                    } else {
+                        bf16 *dst = p.KP + ((((size_t)pg * D.L + (p.layer - 1)) * D.nkv + n / hd) * 16 + sl) * hd + jj;
+                        store_bf16x32(dst, lo);
+                        store_bf16x32(dst + half, hi);
+                    }
                 }
             }
         } else {
@@ -131,16 +153,16 @@ __device__ __forceinline__ void epilogue(const PfArgs &p, uint32_t taddr, int ro
                 const float g = rs * __uint_as_float(r0[e]), u = rs * __uint_as_float(r1[e]);
                 act[e] = g / (1.f + __expf(-g)) * u;
             }
-            bf16 *dst = p.ACT + (size_t)row * D.F + f0;
+            bf16 *dst = p.ACT + (size_t)row * D.F + f0, *dlo = p.ACTL + (size_t)row * D.F + f0;
             if (f0 + 32 <= D.F) {
-                store_bf16x32(dst, act);
+                store_split_x32(dst, dlo, act);
             } else {
-                for (int e = 0; e < 32 && f0 + e < D.F; ++e) dst[e] = __float2bfloat16_rn(act[e]);
+                for (int e = 0; e < 32 && f0 + e < D.F; ++e) split_bf16(act[e], dst[e], dlo[e]);
             }
         }
     } else {   // PF_OPROJ, PF_DOWN: residual update in place, next norm input, sums of squares of the new h
         float ss = 0.f;
-        bf16 *xo = EPI == PF_OPROJ ? p.XM : p.XS;
+        bf16 *xo = EPI == PF_OPROJ ? p.XM : p.XS, *xl = EPI == PF_OPROJ ? p.XML : p.XSL;
         for (int c0 = 0; c0 < p.bn_narrow; c0 += 32) {
             __syncwarp();
             tmem_ld32(taddr + (uint32_t)c0, r0);
@@ -170,7 +192,7 @@ __device__ __forceinline__ void epilogue(const PfArgs &p, uint32_t taddr, int ro
                 ss += h[e] * h[e];
                 x[e] = p.gain ? h[e] * bf16_to_f(p.gain[n + e]) : 0.f;
             }
-            if (p.gain) store_bf16x32(xo + (size_t)row * D.d + n, x);
+            if (p.gain) store_split_x32(xo + (size_t)row * D.d + n, xl + (size_t)row * D.d + n, x);
             // one partial sum of squares per 128 columns, whatever the tile width: results do not depend on it
             if ((c0 & 127) == 96 || n + 32 >= D.d) {
                 (EPI == PF_OPROJ ? p.SSPM : p.SSP)[(size_t)row * p.n_ssp + (n >> 7)] = ss;
@@ -223,9 +245,11 @@ __global__ void __launch_bounds__(PF_THREADS, 1) prefill_gemm_kernel(const __gri
                 for (int kb = 0; kb < n_kb; ++kb, ++it) {
                     const int s = it % STAGES;
                     if (!mbar_wait(&empty_bar[s], ((it / STAGES) & 1) ^ 1)) { s_err = 1; break; }
-                    mbar_expect_tx(&full_bar[s], A_BYTES + tile_n<EPI>(p) * BK * 2);
+                    mbar_expect_tx(&full_bar[s], 2 * A_BYTES + tile_n<EPI>(p) * BK * 2);
                     unsigned char *sa = tiles + (size_t)s * STAGE_BYTES;
                     tma_load_2d(sa, &maps.a, kb * BK, mt * BM, &full_bar[s]);
+                    tma_load_2d(sa + A_BYTES, &maps.a_lo, kb * BK, mt * BM, &full_bar[s]);
+                    sa += A_BYTES;               // the weight tile follows the two activation tiles
                     if (EPI == PF_QKV) {
                         if (nt < n_qt) tma_load_2d(sa + A_BYTES, &maps.b0, kb * BK, nt * BN, &full_bar[s]);
                         else if (nt < n_qt + n_kt) tma_load_2d(sa + A_BYTES, &maps.b1, kb * BK, (nt - n_qt) * BN, &full_bar[s]);
@@ -257,10 +281,12 @@ __global__ void __launch_bounds__(PF_THREADS, 1) prefill_gemm_kernel(const __gri
                     if (!mbar_wait(&full_bar[s], (it / STAGES) & 1)) { s_err = 3; ok = false; break; }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t sa = smem_u32(tiles + (size_t)s * STAGE_BYTES);
-                    const uint64_t da = umma_desc(sa), db = umma_desc(sa + A_BYTES);
+                    const uint64_t da = umma_desc(sa), dl = umma_desc(sa + A_BYTES), db = umma_desc(sa + 2 * A_BYTES);
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
+                    for (int k = 0; k < BK / 16; ++k) {
                         umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+                        umma_bf16(d_tmem, dl + 2 * k, db + 2 * k, idesc, 1u);
+                    }
                     umma_commit(&empty_bar[s]);      // the stage may be refilled once these MMAs have read it
                 }
                 if (!ok) break;
@@ -303,7 +329,7 @@ __global__ void __launch_bounds__(256) prefill_embed_kernel(const PfArgs p, cons
         const float h = bf16_to_f(e[o]);
         p.H[(size_t)row * d + o] = h;
         if (sp) sp[o] = h;
-        p.XS[(size_t)row * d + o] = __float2bfloat16_rn(h * bf16_to_f(gain0[o]));
+        split_bf16(h * bf16_to_f(gain0[o]), p.XS[(size_t)row * d + o], p.XSL[(size_t)row * d + o]);
         ss += h * h;
     }
     ss = warp_sum(ss);
@@ -321,11 +347,10 @@ template <int EPI>
 cudaError_t launch_epi(const PfMaps &maps, const PfArgs &p, int n_sms, cudaStream_t st, bool pdl) {
     const size_t smem = (size_t)STAGES * STAGE_BYTES + 1024;
     auto kern = prefill_gemm_kernel<EPI>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static SmemAttrOnce attr;
+    {
+        cudaError_t e = attr.set(kern, (int)((int)smem));
         if (e != cudaSuccess) return e;
-        attr_done = true;
     }
     const int n_tiles = ((p.M + BM - 1) / BM) * p.n_ntiles;
     cudaLaunchConfig_t cfg = {};
@@ -371,10 +396,11 @@ int prefill_tc_narrow(const Dims &D) {
 
 // map_a / map_b*: 128-byte CUtensorMap blobs made by lmhead_tc_make_map (boxes of 256 rows for Wq / Wk / Wv, of
 // 128 rows for the activations and for W_gate / W_up / W_o / W_down)
-cudaError_t launch_prefill_gemm(int epi, const void *map_a, const void *map_b0, const void *map_b1, const void *map_b2,
-                                const PfArgs &p, int n_sms, cudaStream_t st, bool pdl) {
+cudaError_t launch_prefill_gemm(int epi, const void *map_a, const void *map_a_lo, const void *map_b0, const void *map_b1,
+                                const void *map_b2, const PfArgs &p, int n_sms, cudaStream_t st, bool pdl) {
     PfMaps maps;
     maps.a = *reinterpret_cast<const CUtensorMap *>(map_a);
+    maps.a_lo = *reinterpret_cast<const CUtensorMap *>(map_a_lo);
     maps.b0 = *reinterpret_cast<const CUtensorMap *>(map_b0);
     maps.b1 = *reinterpret_cast<const CUtensorMap *>(map_b1 ? map_b1 : map_b0);
     maps.b2 = *reinterpret_cast<const CUtensorMap *>(map_b2 ? map_b2 : map_b0);

@@ -15,6 +15,13 @@
 // Partial sums of the 8 warps are added in a fixed order through shared memory: results do not depend
 // on the grid size or on how many rows share the pass.
 //
+// Activation precision.  The layer GEMMs take every activation as a pair of bf16 values (high + low part, 16
+// bits of mantissa; the weights are exact bf16 anyway), so that the product carries fp32-like accuracy.  The
+// low parts cost no extra tensor-core instruction for up to four rows: the eight columns of an MMA's n-tile
+// hold the high parts of rows 0..3 and the low parts of the same rows, and the two column halves are added
+// after the cross-warp reduction.  In general a launch of NT n-tiles serves 4 * NT rows (at most 32; a pass
+// of more rows is two launches).  The LM head takes single bf16 rows (8 * NT of them).
+//
 // Epilogues (one per use in the decoder layer):
 //   QKV    scale by the row's 1/rms, rotary embedding on q and k, q -> Q buffer, k and v -> paged cache
 //   OPROJ  + residual -> HM, XM = bf16(HM * ffn gain), partial sums of squares
@@ -24,11 +31,6 @@
 // RMSNorm is split: the producer stores bf16(h * gain) and per-tile sums of h^2, the consumer scales
 // its accumulators by rsqrt(mean(h^2) + eps) (the scale is a per-row scalar, so it commutes with W).
 #include "kernels.h"
-
-// optional per-CTA time stamps for tuning builds (a harness defines the macro); off in the library
-#ifndef DEL_TRACE_STAMP
-#define DEL_TRACE_STAMP(i)
-#endif
 
 namespace {
 
@@ -70,8 +72,10 @@ __device__ __forceinline__ void tile_rows(const GemmArgs &a, int item, const bf1
 }
 
 template <int NT, int U, int EPI>
-__global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_kernel(const __grid_constant__ GemmArgs a) {
-    constexpr int NC = NT * 8;                      // activation-row columns handled
+__global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 4 ? 2 : 1)) rowgemm_kernel(const __grid_constant__ GemmArgs a) {
+    constexpr int NC = NT * 8;                      // MMA columns
+    constexpr bool HL = EPI != EPI_LMHEAD;          // columns [0, NR): high parts of NR rows, [NR, NC): their low parts
+    constexpr int NR = HL ? NC / 2 : NC;            // activation rows handled
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float4 *red = reinterpret_cast<float4 *>(smem_raw);                       // [8 warps][NT][32]
     float *res = reinterpret_cast<float *>(smem_raw + sizeof(float4) * 8 * NT * 32);  // [NC][16]
@@ -118,7 +122,6 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     };
 
     // the first burst of weights goes out before the producer kernel has finished
-    DEL_TRACE_STAMP(0);
     // Tiles: two static turns per CTA (b, b + grid), further tiles claimed from a per-launch counter so that
     // fast CTAs take more and all CTAs finish together.  Results do not depend on who computes a tile.
     const int grid = (int)gridDim.x;
@@ -133,21 +136,23 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     claim();
     pdl_launch();
     pdl_wait();
-    DEL_TRACE_STAMP(1);
 
     const PassPlan *plan = &a.plan;
+    const int row0 = HL ? a.row0 : 0;               // rows row0 .. row0 + NR - 1 of the pass
     const int m = plan->m;
     // activation row pointers of this thread's columns
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
-        const int c = nt * 8 + g;
+        const int col = nt * 8 + g;
+        const bool low = HL && col >= NR;
+        const int c = row0 + (low ? col - NR : col);
         xrow[nt] = nullptr;
         if (c < m) {
             size_t r;
             if (EPI == EPI_QKV) r = stack_row(a.D, a.layer - 1, plan->rows[c].seq, plan->rows[c].slot);
             else if (EPI == EPI_LMHEAD) r = a.x_by_row ? (size_t)c : (size_t)plan->rows[c].seq * a.D.S + plan->rows[c].slot;
             else r = c;
-            xrow[nt] = a.X + r * (size_t)K;
+            xrow[nt] = (low ? a.XL : a.X) + r * (size_t)K;
         }
     }
     load_x(0, true);
@@ -161,8 +166,8 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
         return a.B.SS + stack_row(a.D, a.layer - 1, plan->rows[c].seq, plan->rows[c].slot) * a.D.n_sst;
     };
     if (EPI == EPI_QKV || EPI == EPI_GATEUP) {
-        const bool v0 = warp < m;
-        const float *ss = v0 ? ss_ptr(warp) : a.B.SSM;
+        const bool v0 = warp < NR && row0 + warp < m;
+        const float *ss = v0 ? ss_ptr(row0 + warp) : a.B.SSM;
 #pragma unroll
         for (int q = 0; q < SSN; ++q) {
             const int i = lane + 32 * q;
@@ -202,29 +207,33 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
         __syncthreads();
         const int item = cur_item;
         const int i = tid & 15;
-        for (int c = tid >> 4; c < NC; c += DEL_GEMM_THREADS / 16) {
+        for (int cl = tid >> 4; cl < NR; cl += DEL_GEMM_THREADS / 16) {
+            const int c = row0 + cl;                // row of the pass; cl: its column in this launch
             const bool valid = c < m;
             const RowDesc rd = valid ? plan->rows[c] : RowDesc{0, 0, 0, 0};
-            const float ra = res[c * 16 + i];
+            // product with the high parts + product with the low parts
+            const float ra = HL ? res[cl * 16 + i] + res[(cl + NR) * 16 + i] : res[cl * 16 + i];
+            // rows 8..15 of the tile at the same column (rotary partner / up row), read by threads i < 8 only
+            const float rb = HL ? res[cl * 16 + (i | 8)] + res[(cl + NR) * 16 + (i | 8)] : 0.f;
             if (EPI == EPI_QKV) {
                 if (!valid) continue;
-                const float r = rscale[c];
+                const float r = rscale[cl];
                 const int hd = a.D.hd, half = hd >> 1, h8 = hd >> 4;
                 const int nq = a.D.nh * h8, nk = a.D.nkv * h8;
                 const int pg = a.B.PT[rd.seq * a.D.pages_per_seq + (rd.pos >> 4)];
                 const int sl = rd.pos & 15;
                 if (item < nq + nk) {
                     if (i >= 8) continue;                         // rows 0..7 and their partners 8..15: one thread per pair
-                    const float va = r * ra, vb = r * res[c * 16 + 8 + i];
+                    const float va = r * ra, vb = r * rb;
                     const bool isq = item < nq;
                     const int it = isq ? item : item - nq;
                     const int head = it / h8, j = (it - head * h8) * 8 + i;
                     const float cs = a.B.rope_cos[(size_t)rd.pos * half + j], sn = a.B.rope_sin[(size_t)rd.pos * half + j];
                     const float oa = va * cs - vb * sn, ob = vb * cs + va * sn;
                     if (isq) {
-                        bf16 *q = a.B.Q + (size_t)c * (a.D.nh * hd) + head * hd + j;
-                        q[0] = __float2bfloat16_rn(oa);
-                        q[half] = __float2bfloat16_rn(ob);
+                        const size_t qo = (size_t)c * (a.D.nh * hd) + head * hd + j;
+                        split_bf16(oa, a.B.Q[qo], a.B.QL[qo]);
+                        split_bf16(ob, a.B.Q[qo + half], a.B.QL[qo + half]);
                     } else {
                         bf16 *kp = a.B.KP + ((((size_t)pg * a.D.L + (a.layer - 1)) * a.D.nkv + head) * 16 + sl) * hd + j;
                         kp[0] = __float2bfloat16_rn(oa);
@@ -237,11 +246,11 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
                 }
             } else if (EPI == EPI_GATEUP) {
                 if (!valid) continue;
-                const float r = rscale[c];
+                const float r = rscale[cl];
                 if (i >= 8) continue;                             // rows 0..7 gate, rows 8..15 the matching up rows
-                const float gate = r * ra, up = r * res[c * 16 + 8 + i];
+                const float gate = r * ra, up = r * rb;
                 const float act = gate / (1.f + __expf(-gate)) * up;
-                a.B.ACT[(size_t)c * a.D.F + 8 * item + i] = __float2bfloat16_rn(act);
+                split_bf16(act, a.B.ACT[(size_t)c * a.D.F + 8 * item + i], a.B.ACTL[(size_t)c * a.D.F + 8 * item + i]);
             } else if (EPI == EPI_OPROJ || EPI == EPI_DOWN) {
                 const int o = 16 * item + i;
                 float h = 0.f;
@@ -249,12 +258,12 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
                     if (EPI == EPI_OPROJ) {
                         h = ldg_cg_f32(a.B.H + stack_row(a.D, a.layer - 1, rd.seq, rd.slot) * a.D.d + o) + ra;
                         a.B.HM[(size_t)c * a.D.d + o] = h;
-                        a.B.XM[(size_t)c * a.D.d + o] = __float2bfloat16_rn(h * bf16_to_f(a.gain_a[o]));
+                        split_bf16(h * bf16_to_f(a.gain_a[o]), a.B.XM[(size_t)c * a.D.d + o], a.B.XML[(size_t)c * a.D.d + o]);
                     } else {
                         h = ldg_cg_f32(a.B.HM + (size_t)c * a.D.d + o) + ra;
                         const size_t sr = stack_row(a.D, a.layer, rd.seq, rd.slot);
                         a.B.H[sr * a.D.d + o] = h;
-                        if (a.gain_a) a.B.XS[sr * a.D.d + o] = __float2bfloat16_rn(h * bf16_to_f(a.gain_a[o]));
+                        if (a.gain_a) split_bf16(h * bf16_to_f(a.gain_a[o]), a.B.XS[sr * a.D.d + o], a.B.XSL[sr * a.D.d + o]);
                         if (a.gain_b)
                             a.B.XE[((size_t)rd.seq * a.D.S + rd.slot) * a.D.d + o] = __float2bfloat16_rn(h * bf16_to_f(a.gain_b[o]));
                     }
@@ -318,11 +327,11 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     };
 
     mma_burst();
-    DEL_TRACE_STAMP(2);
     if (EPI == EPI_QKV || EPI == EPI_GATEUP) {
-        for (int c = warp; c < NC; c += DEL_GEMM_WARPS) {
+        for (int cl = warp; cl < NR; cl += DEL_GEMM_WARPS) {
+            const int c = row0 + cl;
             float s = 0.f;
-            if (c == warp) {
+            if (cl == warp) {
 #pragma unroll
                 for (int q = 0; q < SSN; ++q) s += ssv[q];
                 if (c < m)
@@ -332,7 +341,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
                 for (int i = lane; i < a.D.n_sst; i += 32) s += ldg_cg_f32(ss + i);
             }
             s = warp_sum(s);
-            if (lane == 0) rscale[c] = rsqrtf(s / (float)a.D.d + a.D.eps);
+            if (lane == 0) rscale[cl] = rsqrtf(s / (float)a.D.d + a.D.eps);
         }
     }
     if (EPI == EPI_LMHEAD) {
@@ -381,7 +390,6 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
         u0 = U;
     }
 
-    DEL_TRACE_STAMP(3);
     if (EPI == EPI_LMHEAD) {
         __syncthreads();
         for (int c = tid; c < m; c += DEL_GEMM_THREADS) {
@@ -392,7 +400,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 2 ? 2 : 1)) rowgemm_k
     }
 }
 
-template <int NT> constexpr int depth_for() { return NT == 1 ? 8 : (NT == 2 ? 4 : 2); }
+template <int NT> constexpr int depth_for() { return NT == 1 ? 8 : (NT <= 4 ? 4 : 3); }
 
 template <int NT, int EPI>
 cudaError_t launch_nt(const GemmArgs &a, int grid, cudaStream_t st, bool pdl) {
@@ -400,11 +408,10 @@ cudaError_t launch_nt(const GemmArgs &a, int grid, cudaStream_t st, bool pdl) {
     constexpr int NC = NT * 8;
     const size_t smem = small_smem_bytes(NT);
     auto kern = rowgemm_kernel<NT, D, EPI>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    static SmemAttrOnce attr;
+    {
+        cudaError_t e = attr.set(kern, (int)((int)smem));
         if (e != cudaSuccess) return e;
-        attr_done = true;
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -419,20 +426,21 @@ cudaError_t launch_nt(const GemmArgs &a, int grid, cudaStream_t st, bool pdl) {
     return cudaLaunchKernelEx(&cfg, kern, a);
 }
 
-int g_cta_per_sm = 2;
-
+// m: rows this launch handles (layer GEMMs: two columns per row)
 template <int EPI>
 cudaError_t launch_epi(const GemmArgs &a, int m, int n_sms, cudaStream_t st, bool pdl) {
-    const int nt = (m + 7) / 8;
-    if (nt <= 1) return launch_nt<1, EPI>(a, min(a.n_items, g_cta_per_sm * n_sms), st, pdl);
-    if (nt <= 2) return launch_nt<2, EPI>(a, min(a.n_items, g_cta_per_sm * n_sms), st, pdl);
-    if (nt <= 4) return launch_nt<4, EPI>(a, min(a.n_items, n_sms), st, pdl);
+    const int nt = EPI == EPI_LMHEAD ? (m + 7) / 8 : (m + 3) / 4;
+    const int per_sm = a.ctas_per_sm == 1 ? 1 : 2;
+    if (nt <= 1) return launch_nt<1, EPI>(a, min(a.n_items, per_sm * n_sms), st, pdl);
+    if (nt <= 2) return launch_nt<2, EPI>(a, min(a.n_items, per_sm * n_sms), st, pdl);
+    if (nt <= 4) return launch_nt<4, EPI>(a, min(a.n_items, per_sm * n_sms), st, pdl);
     return launch_nt<8, EPI>(a, min(a.n_items, n_sms), st, pdl);
 }
 
 }  // namespace
 
 cudaError_t launch_rowgemm(int epi, const GemmArgs &a, int m, int n_sms, cudaStream_t st, bool pdl) {
+    if (epi != EPI_LMHEAD) m = min(m - a.row0, DEL_GEMM_ROWS);
     switch (epi) {
         case EPI_QKV: return launch_epi<EPI_QKV>(a, m, n_sms, st, pdl);
         case EPI_OPROJ: return launch_epi<EPI_OPROJ>(a, m, n_sms, st, pdl);
@@ -443,10 +451,8 @@ cudaError_t launch_rowgemm(int epi, const GemmArgs &a, int m, int n_sms, cudaStr
     return cudaErrorInvalidValue;
 }
 
-void rowgemm_set_ctas_per_sm(int n) { g_cta_per_sm = n < 1 ? 1 : (n > 2 ? 2 : n); }
-
-int rowgemm_lmhead_grid(int n_items, int m, int n_sms) {
+int rowgemm_lmhead_grid(int n_items, int m, int n_sms, int ctas_per_sm) {
     const int nt = (m + 7) / 8;
-    const int cap = nt <= 2 ? g_cta_per_sm * n_sms : n_sms;
+    const int cap = nt <= 4 ? (ctas_per_sm == 1 ? 1 : 2) * n_sms : n_sms;
     return n_items < cap ? n_items : cap;
 }

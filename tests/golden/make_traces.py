@@ -5,6 +5,8 @@ Calls only ``synth`` (seeded inputs) and ``oracle`` (the CPU oracle); nothing fr
     python tests/golden/make_traces.py tiny
     python tests/golden/make_traces.py llama2_7b [--gen-len N] [--seqs K]
     python tests/golden/make_traces.py llama2_7b --exit-mode --gen-len 128     (-> trace_llama2_7b_exit.json)
+    python tests/golden/make_traces.py llama3_8b_b4 --resume-dir DIR   (hours of CPU: every finished sequence is
+                                                                        kept in DIR and reused by a restarted run)
 
 Output: tests/golden/trace_<config>.json.  Per sequence: the prompt recipe's identifiers, the token
 emitted by the prefill, the initial window's shadow tokens / margins / statistics, and for every round
@@ -85,6 +87,7 @@ def main():
     ap.add_argument("--seqs", type=int, default=None)
     ap.add_argument("--out", default=None)
     ap.add_argument("--exit-mode", action="store_true")
+    ap.add_argument("--resume-dir", default=None)
     a = ap.parse_args()
     cfg = synth.CONFIGS[a.config]
     gen_len = a.gen_len or cfg.gen_len
@@ -93,11 +96,25 @@ def main():
     weights = synth.make_weights(cfg)
     print(f"weights: {weights.nbytes() / 1e9:.2f} GB in {time.time() - t0:.1f}s; threads {oracle.num_threads()}",
           flush=True)
+    def one(s):
+        if not a.resume_dir:
+            return trace_sequence(cfg, weights, s, gen_len, a.exit_mode)
+        os.makedirs(a.resume_dir, exist_ok=True)
+        part = os.path.join(a.resume_dir, f"{cfg.name}{'_exit' if a.exit_mode else ''}_g{gen_len}_seq{s}.json")
+        if os.path.exists(part):
+            with open(part) as f:
+                return json.load(f)
+        rec = trace_sequence(cfg, weights, s, gen_len, a.exit_mode)
+        with open(part + ".tmp", "w") as f:
+            json.dump(rec, f, separators=(",", ":"))
+        os.replace(part + ".tmp", part)
+        return rec
+
     doc = {"config": cfg.name, "seed": cfg.seed, "prompt_len": cfg.prompt_len, "gen_len": gen_len,
            "e_range": [cfg.e_min, cfg.e_max], "g_range": [cfg.g_min, cfg.g_max], "omega": cfg.omega,
            "oracle_threads": oracle.num_threads(),
            "exit_mode": bool(a.exit_mode),
-           "sequences": [trace_sequence(cfg, weights, s, gen_len, a.exit_mode) for s in range(n_seq)]}
+           "sequences": [one(s) for s in range(n_seq)]}
     out = a.out or os.path.join(os.path.dirname(os.path.abspath(__file__)),
                                 f"trace_{cfg.name}{'_exit' if a.exit_mode else ''}.json")
     with open(out, "w") as f:

@@ -64,6 +64,18 @@ def forward_all(cfg, w: synth.Weights, tokens, n_layers=None):
     return out
 
 
+def kv_rows(cfg, w: synth.Weights, h_in, layer: int):
+    """Keys (rotated) and values (not rotated) that 1-based `layer` caches for every position, from the hidden
+    states entering it: two [T, n_kv_heads * hd] arrays."""
+    lw = w.layers[layer - 1]
+    T = h_in.shape[0]
+    a = rmsnorm(h_in, _f64(lw["attn_norm"]), cfg.rms_eps)
+    k = (a @ _f64(lw["wk"]).T).reshape(T, cfg.n_kv_heads, cfg.head_dim)
+    v = a @ _f64(lw["wv"]).T
+    k = rope_complex(k, np.arange(T, dtype=np.float64), cfg.head_dim, cfg.rope_theta)
+    return k.reshape(T, -1), v
+
+
 def exit_logits(cfg, w: synth.Weights, h):
     """Shared final RMSNorm + LM head on hidden rows [.., d] -> logits [.., V]."""
     a = rmsnorm(h, _f64(w.final_norm), cfg.rms_eps)

@@ -80,6 +80,7 @@ class Report:
     conf_max_rel: float = 0.0
     decisions: int = 0
     decision_flips: int = 0
+    max_flip_margin: float = 0.0            # largest oracle margin among the arg-max results that differ
     failures: List[str] = field(default_factory=list)
 
     def ok(self) -> bool:
@@ -178,6 +179,7 @@ def compare_init(ctx, seq, ref: SeqRef, total_tokens: int, rep: Report, policy=N
         for j in range(ncol):
             rep.compared += 1
             if sh[l, j] != ref.init_shadow[l, j]:
+                rep.max_flip_margin = max(rep.max_flip_margin, float(ref.init_margin[l, j]))
                 if ref.init_margin[l, j] > MARGIN:
                     rep.failures.append(f"init shadow l={l + 1} j={j}: gpu {sh[l, j]} oracle {ref.init_shadow[l, j]} "
                                         f"margin {ref.init_margin[l, j]:.3f}")
@@ -258,6 +260,7 @@ def compare_round(ctx, seq, out, r: RoundRef, rep: Report, check_choice=True, la
     last_row = r.g
     for i in range(r.g):
         if drafts[i] != r.drafts[i]:
+            rep.max_flip_margin = max(rep.max_flip_margin, float(r.margin[r.E - 1, i]))
             if r.margin[r.E - 1, i] > MARGIN:
                 rep.failures.append(f"round {rep.rounds}: draft {i} gpu {drafts[i]} oracle {r.drafts[i]} margin "
                                     f"{r.margin[r.E - 1, i]:.3f}")
@@ -268,6 +271,7 @@ def compare_round(ctx, seq, out, r: RoundRef, rep: Report, check_choice=True, la
         for i in range(last_row + 1):
             rep.compared += 1
             if sh[l, i] != r.shadow[l, i]:
+                rep.max_flip_margin = max(rep.max_flip_margin, float(r.margin[l, i]))
                 if r.margin[l, i] > MARGIN:
                     rep.failures.append(f"round {rep.rounds}: shadow l={l + 1} i={i} gpu {sh[l, i]} oracle {r.shadow[l, i]} "
                                         f"margin {r.margin[l, i]:.3f}")

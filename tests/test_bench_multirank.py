@@ -70,3 +70,18 @@ def test_reference_arm_other_ranks_exit_without_work():
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
                         "--warmup", "1"], env=env, capture_output=True, text=True, timeout=120)
     assert r.returncode == 0 and r.stdout.strip() == ""
+
+
+def test_reference_arm_runs_the_named_workload():
+    """The oracle arm prefills the configuration's whole prompt and prints the same `config` object as the GPU arm."""
+    sys.path.insert(0, ROOT)
+    import bench
+    import synth
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "tiny", "--steps", "3",
+                        "--warmup", "1"], capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-500:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    cfg = synth.CONFIGS["tiny"]
+    assert line["impl"] == "reference" and line["config"] == bench.bench_config(cfg, 1)
+    assert f"the {cfg.prompt_len}-token prompt" in line["cpu_baseline"]["sample"]
+    assert line["value"] > 0 and line["cpu_baseline"]["kind"] == "oracle"

@@ -7,7 +7,7 @@ import pytest
 
 import synth
 from cases import TINY, TINY_GQA, TINY_GQA_LONG, TINY_LONG, TINY_LONG2, TINY_LONG3, TINY_SHORT
-from parity import MARGIN, ref_from_golden, ref_from_oracle, run_batch, run_sequence
+from parity import MARGIN, Report, _resync, compare_init, compare_round, ref_from_golden, ref_from_oracle, run_batch, run_sequence
 
 pytestmark = pytest.mark.gpu
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
@@ -230,6 +230,39 @@ def test_error_codes(small):
     assert ctx.round()[0].n_emitted >= 1
 
 
+def test_expired_device_wait_is_reported_cleared_and_survivable(small):
+    """The path a bounded device-side wait takes when it gives up: a non-zero error word -> DEL_ETIMEOUT from the next
+    call that reads results, the word cleared, the context usable.  The word is written from the host (test hook), so
+    no kernel waits and nothing on the GPU misbehaves."""
+    import paper_2504_05598_b200 as dl
+    cfg, w, ctx = small
+    lib, h = ctx.lib, ctx._h
+    prompt = synth.make_prompt(cfg)
+    ref = ref_from_oracle(cfg, w, prompt)
+    assert lib.del_debug_inject_error(h, 0) == dl.EINVAL
+    # through del_round (results come back by the mailbox, whose status word carries the error)
+    ctx.prefill(0, prompt, cfg.gen_len)
+    ctx.round()
+    ctx.debug_inject_error(3)
+    outs = (dl.RoundOut * ctx.shape.max_batch)()
+    assert lib.del_round(h, outs) == dl.ETIMEOUT
+    assert b"wait" in lib.del_strerror(dl.ETIMEOUT)
+    # through the step calls (results come back by copy)
+    ctx.prefill(0, prompt, cfg.gen_len)
+    ctx.draft(0, cfg.e_min, 1)
+    ctx.verify(0)
+    ctx.debug_inject_error(4)
+    assert lib.del_layer_accept(h, 0, None) == dl.ETIMEOUT
+    # and through a prefill
+    ctx.debug_inject_error(1)
+    p = np.ascontiguousarray(prompt, dtype=np.int32)
+    assert lib.del_prefill(h, 0, p.ctypes.data, len(p), cfg.gen_len, None) == dl.ETIMEOUT
+    # the word was cleared each time: a fresh run of the sequence matches the oracle from start to end
+    rep = run_sequence(ctx, 0, ref, cfg.gen_len)
+    assert rep.ok(), rep.failures[:5]
+    assert rep.rounds == len(ref.rounds)
+
+
 def test_kv_pages_run_out_and_come_back():
     """Two sequences share a page pool that holds one and a half of them: the second prefill is refused with
     DEL_ENOSPC, the first sequence keeps decoding correctly, and after its release the second one fits."""
@@ -271,37 +304,38 @@ def test_generation_stops_at_budget(small):
 
 
 def test_batch_of_independent_sequences():
-    """Three sequences with their own prompts, (E, gamma) and statistics share the layer passes."""
+    """Three sequences with their own prompts, (E, gamma), statistics and generation lengths share the layer passes;
+    a sequence that has emitted all its tokens drops out of the later rounds."""
+    import paper_2504_05598_b200 as dl
     cfg = synth.small_variant(TINY_GQA, batch=3)
     w = synth.make_weights(cfg)
     ctx = make_ctx(cfg, w)
-    refs = [ref_from_oracle(cfg, w, synth.make_prompt(cfg, s), gen_len=20 + 7 * s) for s in range(3)]
+    totals = [20 + 7 * s for s in range(3)]
+    refs = [ref_from_oracle(cfg, w, synth.make_prompt(cfg, s), gen_len=totals[s]) for s in range(3)]
+    reps = [Report() for _ in refs]
     for s in range(3):
-        out = ctx.prefill(s, refs[s].prompt, 20 + 7 * s)
-        assert out.tokens[0] == refs[s].first_token
-    got = [[r.first_token] for r in refs]
-    k = [0, 0, 0]
-    import paper_2504_05598_b200 as dl
+        compare_init(ctx, s, refs[s], totals[s], reps[s])
+    k, done = [0, 0, 0], [1, 1, 1]
     while True:
         rc, outs = ctx.try_round()
         if rc != dl.OK:
+            assert rc == dl.ESTATE                      # no live sequence is left
             break
         for s in range(3):
-            if outs[s].n_emitted == 0:
+            if k[s] >= len(refs[s].rounds):
+                assert outs[s].n_emitted == 0           # finished: takes no part in the round
                 continue
             r = refs[s].rounds[k[s]]
-            clean = (r.margin > MARGIN).all()
-            if clean:
-                assert (outs[s].E, outs[s].g, outs[s].n_accept) == (r.E, r.g, r.n), (s, k[s])
-                assert outs[s].emitted() == list(r.emitted)
-                assert (outs[s].next_E, outs[s].next_gamma) == (r.next_E, r.next_gamma)
+            need = compare_round(ctx, s, outs[s], r, reps[s])
+            done[s] += r.n + 1
             k[s] += 1
-            got[s] += outs[s].emitted()
+            if need and k[s] < len(refs[s].rounds):
+                reps[s].resyncs += 1
+                _resync(ctx, s, refs[s], done[s], r.Sc, r.Sn, r.next_E, r.next_gamma, totals[s], r.Stcs, r.Sfcs)
     for s in range(3):
-        assert len(got[s]) == 20 + 7 * s
-        low = any((r.margin <= MARGIN).any() for r in refs[s].rounds) or (refs[s].init_margin <= MARGIN).any()
-        if not low:
-            assert got[s] == refs[s].tokens
+        print(f"seq {s}: rounds {reps[s].rounds} compared {reps[s].compared} flips {reps[s].flips}")
+        assert reps[s].ok(), (s, reps[s].failures[:5])
+        assert k[s] == len(refs[s].rounds) and done[s] == totals[s]
 
 
 @pytest.mark.parametrize("name,max_rounds", [("llama2_7b", None), ("llama32_1b", None), ("llama2_13b", None)])
@@ -317,7 +351,10 @@ def test_full_size_config_against_stored_trace(name, max_rounds):
     ctx = make_ctx(cfg, w)
     ref = ref_from_golden(doc, 0, synth.make_prompt(cfg, 0))
     rep = run_sequence(ctx, 0, ref, doc["gen_len"], max_rounds=max_rounds)
-    print(f"{name}: rounds {rep.rounds} compared {rep.compared} flips {rep.flips} resyncs {rep.resyncs}")
+    print(f"{name}: rounds {rep.rounds} compared {rep.compared} flips {rep.flips} resyncs {rep.resyncs} "
+          f"largest differing margin {rep.max_flip_margin:.3f}")
+    # the bar is 0.05 (a failure above it); what actually differs sits well inside
+    assert rep.max_flip_margin <= 0.03
     assert rep.ok(), rep.failures[:8]
     assert rep.flips <= rep.compared // 20
 
@@ -525,35 +562,42 @@ def test_interleaved_sequence_lifetimes_with_few_pages():
     ctx.close()
 
 
-def test_logit_error_at_full_width():
-    """The 7B layer shape (d = 4096, F = 11008, V = 32000) with six layers and a 100-token prompt, oracle run live:
-    how far the library's bf16 activations put it from the oracle's fp32 ones.  Hidden states: relative rms error
-    per layer; exit-head logits over the whole vocabulary: rms and max-abs error per layer.  Measured 3.5e-3 ->
-    7.5e-3 (hidden), 0.005 -> 0.010 (logit rms), 0.021 -> 0.042 (logit max over 32000 tokens) from layer 1 to 6;
-    the bounds below are those levels with a margin, so that a loss of precision anywhere in the path shows."""
+@pytest.mark.parametrize("n_layers,layers", [(6, (1, 2, 3, 4, 5, 6)), (32, (8, 16, 24, 32))])
+def test_logit_error_at_full_width(n_layers, layers):
+    """The 7B layer shape (d = 4096, F = 11008, V = 32000), six layers and the full 32, a 100-token prompt, oracle run
+    live: exit-head logits over the whole vocabulary must stay within max-abs 3e-2 of the oracle's at every layer
+    compared, through the tensor-core prefill and through the decode kernels.  (Every GEMM input is a bf16 high + low
+    pair; with single bf16 inputs the largest difference was 0.042 at layer 6.)"""
     import oracle
+    import paper_2504_05598_b200 as dl
     base = synth.CONFIGS["llama2_7b"]
-    cfg = synth.small_variant(base, name="llama2_7b_L6", n_layers=6, e_min=1, e_max=5, g_max=5, prompt_len=100, gen_len=20, seed=11)
+    cfg = synth.small_variant(base, name=f"llama2_7b_L{n_layers}", n_layers=n_layers, e_min=1, e_max=n_layers - 1, g_max=5,
+                              prompt_len=100, gen_len=20, seed=11)
     w = synth.make_weights(cfg)
     prompt = synth.make_prompt(cfg)
-    ctx = make_ctx(cfg, w)
     o = oracle.OracleSeq(cfg, w)
     o.prefill(prompt)
-    ctx.prefill(0, prompt, cfg.gen_len)
     j = cfg.init_window - 1
-    worst = 0.0
-    for l in range(1, cfg.n_layers + 1):
-        ho, hl = o.hidden(l, j), ctx.get_hidden(0, l, j)
-        h_rel = float(np.sqrt(((hl - ho) ** 2).mean()) / np.sqrt((ho ** 2).mean()))
-        _, _, lo = o.exit_head(ho, want_logits=True)
-        ll = ctx.debug_logits(0, l, j)
-        rms, mx = float(np.sqrt(((ll - lo) ** 2).mean())), float(np.abs(ll - lo).max())
-        print(f"layer {l}: hidden rel rms {h_rel:.2e}, logits rms {rms:.4f} max {mx:.4f} (logit std {lo.std():.2f})")
-        assert h_rel <= 4.5e-3 * np.sqrt(l) and rms <= 6.5e-3 * np.sqrt(l) and mx <= 0.028 * np.sqrt(l), (l, h_rel, rms, mx)
-        worst = max(worst, mx)
-    assert worst <= 0.06
+    want = {}
+    for l in layers:
+        ho = o.hidden(l, j)
+        want[l] = (ho, o.exit_head(ho, want_logits=True)[2])
     o.close()
-    ctx.close()
+    dev = dl.upload_weights(w)
+    for path, flags in (("tensor-core prefill", dl.FLAG_PDL | dl.FLAG_TC), ("decode kernels", dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_NO_BULK_PREFILL)):
+        ctx = dl.DelContext(dl.make_shape(cfg), dev)
+        ctx.set_flags(flags)
+        ctx.prefill(0, prompt, cfg.gen_len)
+        for l in layers:
+            ho, lo = want[l]
+            hl = ctx.get_hidden(0, l, j)
+            h_rel = float(np.sqrt(((hl - ho) ** 2).mean()) / np.sqrt((ho ** 2).mean()))
+            ll = ctx.debug_logits(0, l, j)
+            rms, mx = float(np.sqrt(((ll - lo) ** 2).mean())), float(np.abs(ll - lo).max())
+            print(f"{path}, layer {l}: hidden rel rms {h_rel:.2e}, logits rms {rms:.4f} max {mx:.4f} (logit std {lo.std():.2f})")
+            assert mx <= 3e-2, (path, l, mx)
+            assert h_rel <= 6e-3 and rms <= 8e-3, (path, l, h_rel, rms)
+        ctx.close()
 
 
 def test_fs_baseline_policy_against_oracle(small):

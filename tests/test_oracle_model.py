@@ -6,7 +6,7 @@ import pytest
 import oracle
 import synth
 from cases import TINY, TINY_GQA, TINY_SHORT
-from np_model import exit_logits, forward_all
+from np_model import exit_logits, forward_all, kv_rows, rmsnorm
 
 CASES = [TINY, TINY_GQA, TINY_SHORT]
 
@@ -29,6 +29,15 @@ def test_cached_forward_equals_full_recompute(case):
             want = ref[l][len(prompt) - W + j]
             assert np.allclose(got, want, rtol=2e-5, atol=2e-5 * np.abs(want).max()), (l, j)
     # keys/values in the cache, first and last position of layer 1 and L: K is rotated, V is not
+    for l in (1, cfg.n_layers):
+        k_ref, v_ref = kv_rows(cfg, w, ref[l - 1], l)
+        for pos in (0, len(prompt) - 1):
+            assert np.allclose(o.k_row(l, pos), k_ref[pos], rtol=2e-5, atol=2e-5 * np.abs(k_ref).max()), (l, pos)
+            assert np.allclose(o.v_row(l, pos), v_ref[pos], rtol=2e-5, atol=2e-5 * np.abs(v_ref).max()), (l, pos)
+        # the rotation is real: at the last position the cached key differs from the unrotated projection
+        a = rmsnorm(ref[l - 1][-1], synth.bf16_to_f32(w.layers[l - 1]["attn_norm"]).astype(np.float64), cfg.rms_eps)
+        k_plain = a @ synth.bf16_to_f32(w.layers[l - 1]["wk"]).astype(np.float64).T
+        assert np.abs(o.k_row(l, len(prompt) - 1) - k_plain).max() > 1e-2 * np.abs(k_plain).max()
     lg = exit_logits(cfg, w, ref[-1][-1])
     assert int(np.argmax(lg)) == tok
     _, mg, logits = o.exit_head(o.hidden(cfg.n_layers, W - 1), want_logits=True)
@@ -175,3 +184,23 @@ def test_resume_from_stats_reproduces_the_trace(case):
         r = b.round(cfg.gen_len - len(emitted) - len(tail))
         tail += r.emitted
     assert emitted + tail == out
+
+
+def test_stored_tiny_trace_is_what_the_oracle_writes_today():
+    """tests/golden/trace_tiny.json was written by make_traces.py from the oracle; the oracle as it stands must write
+    the same trace (tokens, shadow tokens, margins, counts, statistics, choices): the stored full-size traces, which
+    take hours to regenerate, come from the same code path."""
+    import importlib.util
+    import json
+    import os
+    golden = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_traces", os.path.join(golden, "make_traces.py"))
+    mt = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mt)
+    doc = json.load(open(os.path.join(golden, "trace_tiny.json")))
+    cfg = synth.CONFIGS["tiny"]
+    assert doc["seed"] == cfg.seed and doc["prompt_len"] == cfg.prompt_len
+    rec = mt.trace_sequence(cfg, synth.make_weights(cfg), 0, doc["gen_len"])
+    want = doc["sequences"][0]
+    rec.pop("oracle_seconds"), want.pop("oracle_seconds")
+    assert json.loads(json.dumps(rec)) == want
