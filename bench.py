@@ -245,6 +245,20 @@ def run_ours(a):
     dev_ms, wall, tokens, bytes_total = aggregate_replicas(dev_ms, wall, tokens, bytes_total, world, dev)
     value = tokens / (dev_ms / 1000.0)
 
+    if a.timed_only:
+        # the timed region alone (the run a profiler's launch list is taken from): no other legs, short line
+        if rank == 0:
+            peak, _ = measured_peaks()
+            print(json.dumps({"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": W,
+                              "ms_per_step": dev_ms / K, "config": bench_config(cfg, world), "gpu_launches": launches,
+                              "round": {"hbm_gbs": (bytes_total / world / 1e9) / (dev_ms / 1e3),
+                                        "frac_of_measured_peak": (bytes_total / world / 1e9) / (dev_ms / 1e3) / peak},
+                              "note": "--timed-only: prefill, warm-up rounds and the timed rounds only"}), flush=True)
+        ctx.close()
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
     # ---- vanilla (gamma = 0) rounds on the same kernels, for the speculative speed-up on this model
     for s in range(cfg.batch):
         ctx.set_policy(s, 1, 0)
@@ -470,8 +484,13 @@ def run_profile_case(a):
     import paper_2504_05598_b200 as dl
     base = synth.CONFIGS[a.config]
     L = a.layers
+    kw = {}
+    if a.heads:          # slim layers (few heads, narrow FFN) under the configuration's model width and LM head: many
+        kw.update(n_heads=a.heads, n_kv_heads=a.heads)      # layers (= many stacked LM-head rows) in little memory
+    if a.ffn:
+        kw.update(d_ffn=a.ffn)
     cfg = synth.small_variant(base, n_layers=L, e_min=min(base.e_min, L - 1), e_max=min(base.e_max, L - 1),
-                              prompt_len=a.prompt, gen_len=a.rounds * (base.g_max + 1) + 8)
+                              prompt_len=a.prompt, gen_len=a.rounds * (base.g_max + 1) + 8, **kw)
     w = synth.make_weights(cfg)
     ctx = dl.DelContext(dl.make_shape(cfg), dl.upload_weights(w))
     for s in range(cfg.batch):
@@ -519,6 +538,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=20.0)
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-fixed", action="store_true", help="skip the fixed-policy block")
+    ap.add_argument("--timed-only", action="store_true", help="prefill, warm-up and the timed rounds only (for a launch list)")
     # --profile-case: the small case of the ncu captures (no JSON bench line)
     ap.add_argument("--profile-case", action="store_true")
     ap.add_argument("--layers", type=int, default=4)
@@ -526,6 +546,8 @@ def main():
     ap.add_argument("--prompt", type=int, default=512)
     ap.add_argument("--policy", default="", help="E,G: fixed setting instead of the dynamic one")
     ap.add_argument("--sampling", default="", help="T,top_p: speculative sampling instead of greedy verification")
+    ap.add_argument("--heads", type=int, default=0, help="profile case: query = kv heads per layer (0: the configuration's)")
+    ap.add_argument("--ffn", type=int, default=0, help="profile case: FFN width (0: the configuration's)")
     ap.add_argument("--no-timing", action="store_true")
     ap.add_argument("--no-pdl", action="store_true")
     ap.add_argument("--one-cta", action="store_true")

@@ -77,7 +77,7 @@ struct Buffers {
     bf16 *XSL;                   // low part of XS
     float *SS;                   // [L+1][B][S][n_sst] partial sums of squares of h
     bf16 *XE;                    // [B][S][d]         h * gain of the final norm at the exit layer
-    bf16 *Q, *QL;                // [ROWS][nh*hd]     queries after the rotary embedding, high and low part
+    bf16 *Q;                     // [ROWS][nh*hd]     queries after the rotary embedding
     bf16 *ATT, *ATTL;            // [ROWS][nh*hd]     attention output, high and low part
     float *HM;                   // [ROWS][d]         residual after attention
     bf16 *XM, *XML;              // [ROWS][d]         HM * gain of the ffn norm, high and low part

@@ -16,7 +16,7 @@ namespace {
 constexpr int PLAN_RING = 192;
 constexpr int CTR_RING = 4096;
 constexpr int FLAG_PDL = 1, FLAG_GRAPH = 2, FLAG_TC = 4, FLAG_TIMING = 8, FLAG_ONECTA = 16, FLAG_NO_BULK_PREFILL = 32,
-              FLAG_DECODE_ATTN_PREFILL = 64, FLAG_TRIM_ROWS = 128;
+              FLAG_DECODE_ATTN_PREFILL = 64, FLAG_TRIM_ROWS = 128, FLAG_MMA_SYNC_PREFILL_ATTN = 256;
 enum { CLS_QKV = 0, CLS_ATTN, CLS_OPROJ, CLS_GATEUP, CLS_DOWN, CLS_LMHEAD, CLS_LMSTACK, CLS_OTHER, CLS_N };
 
 struct SeqHost {
@@ -75,6 +75,8 @@ struct del_ctx {
     PfArgs pf;                                            // buffer pointers (the per-launch fields are filled in later)
     TMap pf_xs, pf_att, pf_xm, pf_act;                    // activation buffers, high parts ...
     TMap pf_xsl, pf_attl, pf_xml, pf_actl;                // ... and low parts
+    TMap pf_q, pf_ql, kv_k, kv_v;                         // tcgen05 prefill attention: query buffers, paged cache
+    bool pfa_ok = false;
     std::vector<TMap> pf_wq, pf_wk, pf_wv, pf_wo, pf_wg, pf_wu, pf_wd;
     bool pf_ok = false;
     // mailbox of the draft loop's confidence check: pinned host memory that the finalise kernel writes directly
@@ -121,7 +123,6 @@ size_t carve_all(const del_shape &s, void *base, Dims &D, Buffers &B, int &R_max
     B.SS = c.take<float>(base, L1 * BS * D.n_sst);
     B.XE = c.take<bf16>(base, BS * D.d);
     B.Q = c.take<bf16>(base, DEL_ROWS_MAX * qd);
-    B.QL = c.take<bf16>(base, DEL_ROWS_MAX * qd);
     B.ATT = c.take<bf16>(base, DEL_ROWS_MAX * qd);
     B.ATTL = c.take<bf16>(base, DEL_ROWS_MAX * qd);
     B.HM = c.take<float>(base, (size_t)DEL_ROWS_MAX * D.d);
@@ -685,7 +686,10 @@ int prefill_bulk(del_ctx *c, int sq, int n_pos, int win0) {
                 pa.Q = a.Q; pa.QL = a.QL; pa.ATT = a.ATT; pa.ATTL = a.ATTL;
                 pa.KP = c->B.KP; pa.VP = c->B.VP; pa.PT = c->B.PT;
                 pa.M = a.M; pa.layer = l; pa.seq = sq; pa.pos0 = p0;
-                LAUNCH(launch_prefill_attention(pa, c->st, P));
+                if (c->pfa_ok && !(c->flags & FLAG_MMA_SYNC_PREFILL_ATTN))
+                    LAUNCH(launch_prefill_attention_tc(c->pf_q.b, c->pf_ql.b, c->kv_k.b, c->kv_v.b, pa, c->B.ERR, c->st, P));
+                else
+                    LAUNCH(launch_prefill_attention(pa, c->st, P));
             } else
             for (int r0 = 0; r0 < a.M; r0 += DEL_ROWS_MAX) {
                 AttnArgs at;
@@ -693,7 +697,6 @@ int prefill_bulk(del_ctx *c, int sq, int n_pos, int win0) {
                 at.D = D;
                 at.B = c->B;
                 at.B.Q = a.Q + (size_t)r0 * D.nh * D.hd;
-                at.B.QL = a.QL + (size_t)r0 * D.nh * D.hd;
                 at.B.ATT = a.ATT + (size_t)r0 * D.nh * D.hd;
                 at.B.ATTL = a.ATTL + (size_t)r0 * D.nh * D.hd;
                 const int nr = std::min(DEL_ROWS_MAX, a.M - r0);
@@ -1072,6 +1075,10 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
         maps(c->pf_wd, c->w_down, d, F, bn_narrow);
         c->pf.bn_narrow = (int32_t)bn_narrow;
         c->pf_ok = ok;
+        c->pfa_ok = ok && prefill_attention_tc_supported(c->D) &&
+                    lmhead_tc_make_map(c->pf_q.b, c->pf.Q, PF_ROWS, qd, 128) == 0 &&
+                    lmhead_tc_make_map(c->pf_ql.b, c->pf.QL, PF_ROWS, qd, 128) == 0 &&
+                    prefill_attention_tc_make_maps(c->kv_k.b, c->kv_v.b, c->B.KP, c->B.VP, c->D, shape->n_pages) == 0;
         c->pf.D = c->D;
         c->pf.KP = c->B.KP; c->pf.VP = c->B.VP; c->pf.PT = c->B.PT;
         c->pf.rope_cos = c->B.rope_cos; c->pf.rope_sin = c->B.rope_sin;

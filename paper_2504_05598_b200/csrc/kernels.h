@@ -194,6 +194,12 @@ struct PfAttnArgs {
     int32_t M, layer, seq, pos0;
 };
 cudaError_t launch_prefill_attention(const PfAttnArgs &a, cudaStream_t st, bool pdl);
+// The same on tcgen05 / TMEM / TMA (prefill_attn_tc.cu), for head dimension 128.  map_qh / map_ql: the chunk's query
+// buffers (lmhead_tc_make_map, boxes of 128 rows); map_k / map_v: 5-d maps of the paged cache.
+bool prefill_attention_tc_supported(const Dims &D);
+int prefill_attention_tc_make_maps(void *map_k, void *map_v, const void *k_pages, const void *v_pages, const Dims &D, int n_pages);
+cudaError_t launch_prefill_attention_tc(const void *map_qh, const void *map_ql, const void *map_k, const void *map_v,
+                                        const PfAttnArgs &a, int32_t *err, cudaStream_t st, bool pdl);
 cudaError_t launch_prefill_gemm(int epi, const void *map_a, const void *map_a_lo, const void *map_b0, const void *map_b1,
                                 const void *map_b2, const PfArgs &p, int n_sms, cudaStream_t st, bool pdl);
 cudaError_t launch_prefill_embed(const PfArgs &p, const bf16 *tok_emb, const int32_t *prompt, const bf16 *gain0, cudaStream_t st);

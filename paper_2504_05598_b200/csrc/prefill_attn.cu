@@ -72,17 +72,21 @@ __global__ void __launch_bounds__(PA_THREADS) prefill_attention_kernel(const __g
 
     // this warp's query rows as A fragments: rows g and g + 8 of its 16
     constexpr int KS = HD / 16;
-    uint32_t qf[KS][4];
+    // (queries and probabilities enter their products as bf16 high + low pairs: two MMAs each)
+    uint32_t qf[KS][4], ql[KS][4];
     const int r0 = q0 + warp * 16 + g, r1 = r0 + 8;
     {
-        const bf16 *q0p = a.Q + (size_t)r0 * qdim + head * HD + 2 * t;
-        const bf16 *q1p = a.Q + (size_t)r1 * qdim + head * HD + 2 * t;
+        const size_t o0 = (size_t)r0 * qdim + head * HD + 2 * t, o1 = (size_t)r1 * qdim + head * HD + 2 * t;
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
-            qf[ks][0] = r0 < a.M ? *reinterpret_cast<const uint32_t *>(q0p + 16 * ks) : 0u;
-            qf[ks][1] = r1 < a.M ? *reinterpret_cast<const uint32_t *>(q1p + 16 * ks) : 0u;
-            qf[ks][2] = r0 < a.M ? *reinterpret_cast<const uint32_t *>(q0p + 16 * ks + 8) : 0u;
-            qf[ks][3] = r1 < a.M ? *reinterpret_cast<const uint32_t *>(q1p + 16 * ks + 8) : 0u;
+            qf[ks][0] = r0 < a.M ? *reinterpret_cast<const uint32_t *>(a.Q + o0 + 16 * ks) : 0u;
+            qf[ks][1] = r1 < a.M ? *reinterpret_cast<const uint32_t *>(a.Q + o1 + 16 * ks) : 0u;
+            qf[ks][2] = r0 < a.M ? *reinterpret_cast<const uint32_t *>(a.Q + o0 + 16 * ks + 8) : 0u;
+            qf[ks][3] = r1 < a.M ? *reinterpret_cast<const uint32_t *>(a.Q + o1 + 16 * ks + 8) : 0u;
+            ql[ks][0] = r0 < a.M ? *reinterpret_cast<const uint32_t *>(a.QL + o0 + 16 * ks) : 0u;
+            ql[ks][1] = r1 < a.M ? *reinterpret_cast<const uint32_t *>(a.QL + o1 + 16 * ks) : 0u;
+            ql[ks][2] = r0 < a.M ? *reinterpret_cast<const uint32_t *>(a.QL + o0 + 16 * ks + 8) : 0u;
+            ql[ks][3] = r1 < a.M ? *reinterpret_cast<const uint32_t *>(a.QL + o1 + 16 * ks + 8) : 0u;
         }
     }
     const int qp0 = a.pos0 + r0, qp1 = a.pos0 + r1;              // positions of the two rows
@@ -118,6 +122,8 @@ __global__ void __launch_bounds__(PA_THREADS) prefill_attention_kernel(const __g
                     ldsm4(b, ks_ + (8 * (j + (mi >> 1)) + mr) * L::KROW + 16 * ks + 8 * (mi & 1));
                     mma_bf16_16816(S[j], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b[0], b[1]);
                     mma_bf16_16816(S[j + 1], qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3], b[2], b[3]);
+                    mma_bf16_16816(S[j], ql[ks][0], ql[ks][1], ql[ks][2], ql[ks][3], b[0], b[1]);
+                    mma_bf16_16816(S[j + 1], ql[ks][0], ql[ks][1], ql[ks][2], ql[ks][3], b[2], b[3]);
                 }
             // scale, causal mask (only blocks that reach past a row's position need it), running maximum
             const bool diag = kb * BKEY + BKEY - 1 > a.pos0 + q0 + warp * 16;
@@ -142,15 +148,15 @@ __global__ void __launch_bounds__(PA_THREADS) prefill_attention_kernel(const __g
             const float al0 = exp2f(m0 - base0), al1 = exp2f(m1 - base1);
             m0 = n0; m1 = n1;
             float ps0 = 0.f, ps1 = 0.f;
-            uint32_t pf[BKEY / 8][2];                              // probabilities as bf16 pairs: rows g, g + 8
+            uint32_t pf[BKEY / 8][2], pl[BKEY / 8][2];             // probabilities as bf16 pairs (high, low): rows g, g + 8
 #pragma unroll
             for (int j = 0; j < BKEY / 8; ++j) {
                 const float p00 = exp2f(S[j][0] - base0), p01 = exp2f(S[j][1] - base0);
                 const float p10 = exp2f(S[j][2] - base1), p11 = exp2f(S[j][3] - base1);
                 ps0 += p00 + p01;
                 ps1 += p10 + p11;
-                pf[j][0] = pack_bf16(p00, p01);
-                pf[j][1] = pack_bf16(p10, p11);
+                split_bf16x2(p00, p01, pf[j][0], pl[j][0]);
+                split_bf16x2(p10, p11, pf[j][1], pl[j][1]);
             }
             l0 = l0 * al0 + ps0;
             l1 = l1 * al1 + ps1;
@@ -165,6 +171,8 @@ __global__ void __launch_bounds__(PA_THREADS) prefill_attention_kernel(const __g
                     ldsm4(b, vs_ + (kk * HD + 8 * (jd + (mi >> 1)) + mr) * L::VROW + 8 * (mi & 1));
                     mma_bf16_16816(O[jd], pf[2 * kk][0], pf[2 * kk][1], pf[2 * kk + 1][0], pf[2 * kk + 1][1], b[0], b[1]);
                     mma_bf16_16816(O[jd + 1], pf[2 * kk][0], pf[2 * kk][1], pf[2 * kk + 1][0], pf[2 * kk + 1][1], b[2], b[3]);
+                    mma_bf16_16816(O[jd], pl[2 * kk][0], pl[2 * kk][1], pl[2 * kk + 1][0], pl[2 * kk + 1][1], b[0], b[1]);
+                    mma_bf16_16816(O[jd + 1], pl[2 * kk][0], pl[2 * kk][1], pl[2 * kk + 1][0], pl[2 * kk + 1][1], b[2], b[3]);
                 }
         }
         __syncthreads();                                           // the stage is free for the block after next

@@ -231,9 +231,9 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 4 ? 2 : 1)) rowgemm_k
                     const float cs = a.B.rope_cos[(size_t)rd.pos * half + j], sn = a.B.rope_sin[(size_t)rd.pos * half + j];
                     const float oa = va * cs - vb * sn, ob = vb * cs + va * sn;
                     if (isq) {
-                        const size_t qo = (size_t)c * (a.D.nh * hd) + head * hd + j;
-                        split_bf16(oa, a.B.Q[qo], a.B.QL[qo]);
-                        split_bf16(ob, a.B.Q[qo + half], a.B.QL[qo + half]);
+                        bf16 *q = a.B.Q + (size_t)c * (a.D.nh * hd) + head * hd + j;
+                        q[0] = __float2bfloat16_rn(oa);
+                        q[half] = __float2bfloat16_rn(ob);
                     } else {
                         bf16 *kp = a.B.KP + ((((size_t)pg * a.D.L + (a.layer - 1)) * a.D.nkv + head) * 16 + sl) * hd + j;
                         kp[0] = __float2bfloat16_rn(oa);

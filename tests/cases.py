@@ -14,3 +14,9 @@ TINY_GQA_LONG = synth.small_variant(TINY_GQA, name="tiny_gqa_long", prompt_len=2
 TINY_LONG2 = synth.small_variant(TINY, name="tiny_long2", prompt_len=600, gen_len=16, emb_scale=10.0, seed=12)
 TINY_LONG3 = synth.small_variant(TINY_GQA, name="tiny_gqa_long3", prompt_len=530, gen_len=16, seed=79)
 TINY_SHORT = synth.small_variant(TINY, name="tiny_short", prompt_len=7, gen_len=21, emb_scale=10.0, seed=5)
+# head dimension 128 (the shape the tcgen05 prefill attention serves): a ragged last query tile; and two prefill passes
+# with grouped-query attention
+TINY_HD128 = synth.small_variant(TINY, name="tiny_hd128", n_heads=2, n_kv_heads=2, head_dim=128, prompt_len=300, gen_len=24,
+                                 emb_scale=10.0, seed=21)
+TINY_HD128_GQA = synth.small_variant(TINY_GQA, name="tiny_hd128_gqa", n_heads=4, n_kv_heads=2, head_dim=128, prompt_len=600,
+                                     gen_len=16, seed=22)

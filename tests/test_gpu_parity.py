@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 
 import synth
-from cases import TINY, TINY_GQA, TINY_GQA_LONG, TINY_LONG, TINY_LONG2, TINY_LONG3, TINY_SHORT
+from cases import TINY, TINY_GQA, TINY_GQA_LONG, TINY_HD128, TINY_HD128_GQA, TINY_LONG, TINY_LONG2, TINY_LONG3, TINY_SHORT
 from parity import MARGIN, Report, _resync, compare_init, compare_round, ref_from_golden, ref_from_oracle, run_batch, run_sequence
 
 pytestmark = pytest.mark.gpu
@@ -57,7 +57,7 @@ def test_prefill_hidden_kv_and_logits(small):
             assert int(np.argmax(got)) == int(np.argmax(ref))
 
 
-@pytest.mark.parametrize("cfg", [TINY_LONG, TINY_GQA_LONG, TINY_LONG2, TINY_LONG3], ids=lambda c: c.name)
+@pytest.mark.parametrize("cfg", [TINY_LONG, TINY_GQA_LONG, TINY_LONG2, TINY_LONG3, TINY_HD128, TINY_HD128_GQA], ids=lambda c: c.name)
 def test_tensor_core_prefill_against_oracle(cfg):
     """Prompts longer than the initialisation window: their bulk is prefilled by the tcgen05 GEMMs (only the KV
     cache comes out of it).  Cached K/V of bulk positions in every layer, the window's hidden states (which
@@ -71,8 +71,10 @@ def test_tensor_core_prefill_against_oracle(cfg):
     o.prefill(prompt)
     P, W = len(prompt), min(cfg.init_window, len(prompt))
     ref = ref_from_oracle(cfg, w, prompt)
-    for flags in (dl.FLAG_PDL | dl.FLAG_TC, dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_DECODE_ATTN_PREFILL,
-                  dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_NO_BULK_PREFILL):
+    # attention of the bulk prefill: tcgen05 (head dimension 128) or mma.sync flash-style; the mma.sync one where the
+    # other is the default; the decode attention kernel in passes of 64 rows; everything through the decode kernels
+    for flags in (dl.FLAG_PDL | dl.FLAG_TC, dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_MMA_SYNC_PREFILL_ATTN,
+                  dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_DECODE_ATTN_PREFILL, dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_NO_BULK_PREFILL):
         ctx.set_flags(flags)
         launches0 = ctx.launch_count()
         ctx.prefill(0, prompt, cfg.gen_len)
