@@ -502,7 +502,7 @@ def run_profile_case(a):
             E, G = (int(v) for v in a.policy.split(","))
             ctx.set_policy(s, E, G)
     flags = (0 if a.no_pdl else dl.FLAG_PDL) | (dl.FLAG_ONECTA if a.one_cta else 0) | (0 if a.no_tc else dl.FLAG_TC) | \
-        (dl.FLAG_TRIM_ROWS if a.trim else 0)
+        (dl.FLAG_TRIM_ROWS if a.trim else 0) | a.extra_flags
     ctx.set_flags(flags)
     ctx.round()
     ctx.round()
@@ -553,6 +553,7 @@ def main():
     ap.add_argument("--one-cta", action="store_true")
     ap.add_argument("--no-tc", action="store_true")
     ap.add_argument("--trim", action="store_true", help="stacked LM head over the candidate layers only")
+    ap.add_argument("--extra-flags", type=int, default=0, help="profile case: further del_set_flags bits")
     a = ap.parse_args()
     if a.profile_case:
         run_profile_case(a)

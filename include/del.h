@@ -288,7 +288,8 @@ int del_get_traffic(const del_ctx *ctx, int64_t *h2d_bytes, int64_t *d2h_bytes);
  * passes of 64 rows instead of the flash-style prefill attention, bit 7: the stacked LM head runs only over the
  * layers the selection can pick (e_min..e_max) and the last one; shadow tokens, counts and statistics of the other
  * layers are then not maintained, bit 8: the mma.sync flash-style prefill attention also where the tcgen05 one
- * (head dimension 128) would run).  Returns the previous flags. */
+ * (head dimension 128) would run, bit 9: the decode attention kernel does not request the O-projection's weights into
+ * L2).  Returns the previous flags. */
 int del_set_flags(del_ctx *ctx, int flags);
 
 /* With flag bit 3 set, per kernel class (0 QKV, 1 attention, 2 O-proj, 3 gate/up, 4 down, 5 draft LM

@@ -22,7 +22,7 @@ MAX_ROWS = 64
 
 OK, EINVAL, ENOSPC, ESTATE, ETIMEOUT, ECUDA = 0, -1, -2, -3, -4, -5
 FLAG_PDL, FLAG_GRAPH, FLAG_TC, FLAG_TIMING, FLAG_ONECTA, FLAG_NO_BULK_PREFILL, FLAG_DECODE_ATTN_PREFILL, FLAG_TRIM_ROWS = 1, 2, 4, 8, 16, 32, 64, 128
-FLAG_MMA_SYNC_PREFILL_ATTN = 256
+FLAG_MMA_SYNC_PREFILL_ATTN, FLAG_NO_WEIGHT_PREFETCH = 256, 512
 KERNEL_CLASSES = ["qkv_rope", "attention", "o_proj", "gate_up", "down", "lm_head_draft", "lm_head_stacked", "other"]
 
 EXPORTS = ["del_workspace_bytes", "del_init", "del_prefill", "del_draft", "del_verify", "del_layer_accept",

@@ -22,7 +22,7 @@ __global__ void __launch_bounds__(NW * 32) attention_kernel(const __grid_constan
     __shared__ int s_last;
     pdl_launch();                  // (the wait for the producer kernel sits inside partial / partial_staged)
 
-    const AttnView v{a.D, a.B, a.layer, a.early_pos[blockIdx.z]};
+    const AttnView v{a.D, a.B, a.layer, a.early_pos[blockIdx.z], &a.pf};
     const Segment seg = a.plan.seg[blockIdx.z];
     const int kvh = blockIdx.y, split = blockIdx.x, n_splits = a.n_splits;
     const int n_pages = (seg.pos0 + seg.nrows + 15) >> 4;

@@ -29,6 +29,7 @@ struct AttnView {
     const Buffers &B;
     int32_t layer;
     int32_t early_pos;         // of this CTA's segment, see AttnArgs
+    const AttnPrefetch *pf;    // weights to request into L2 for the following launches
 };
 
 namespace attn {
@@ -42,6 +43,23 @@ __device__ __forceinline__ void split_row(int rr, int ms, int &hq, int &i) {
 }
 
 constexpr float LOG2E = 1.4426950408889634f;
+
+// Every CTA of the launch requests its share of the regions in pieces of 32 KB, one piece per lane of its last warp
+// (called once the warps' own early cache reads have been issued, before the wait for the producer kernel).
+__device__ __forceinline__ void prefetch_weights(const AttnPrefetch &pf) {
+    constexpr uint32_t PIECE = 32768;
+    if ((threadIdx.x >> 5) != 7) return;
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t n_cta = gridDim.x * gridDim.y * gridDim.z;
+    const uint32_t cta = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+    for (int r = 0; r < pf.n; ++r) {
+        const uint32_t n_piece = (pf.bytes[r] + PIECE - 1) / PIECE;
+        for (uint32_t i = cta + n_cta * lane; i < n_piece; i += n_cta * 32) {
+            const uint32_t off = i * PIECE, len = min(PIECE, pf.bytes[r] - off) & ~15u;
+            if (len) l2_prefetch_bulk(reinterpret_cast<const unsigned char *>(pf.ptr[r]) + off, len);
+        }
+    }
+}
 constexpr int NW = 8;                 // warps per CTA
 constexpr int PG = 4;                 // page ids fetched ahead per warp
 constexpr int MAX_SLOTS = 16;
@@ -281,7 +299,14 @@ __device__ __forceinline__ void partial(const AttnView &a, float *sm, const Segm
         }
 #pragma unroll
         for (int j = 0; j < NJ; ++j) vf0[j] = ldg_act8(vpage + (8 * j + g) * 16 + 4 * t);
+        // the warp's further committed pages: into L2 for now (one page per lane, two bulk requests per page)
+        for (int p2 = p_first + n_kl * (1 + lane); p2 < p_end && p2 < (a.early_pos >> 4); p2 += n_kl * 32) {
+            const size_t off = (size_t)pt[p2] * page_stride + head_off;
+            l2_prefetch_bulk(a.B.KP + off, 16 * HD * 2);
+            l2_prefetch_bulk(a.B.VP + off, 16 * HD * 2);
+        }
     }
+    prefetch_weights(*a.pf);
     pdl_wait();
 
     for (int it = 0; it < n_iter; ++it) {
@@ -363,6 +388,7 @@ __device__ __forceinline__ void partial_staged(const AttnView &a, unsigned char 
     const int n_pages = max(p_end - p_begin, 0), n_chunks = (n_pages + CH - 1) / CH;
     const int n_iter = (n_mt + P - 1) / P;          // groups of P concurrent query tiles; each group stages the pages again
 
+    prefetch_weights(*a.pf);
     pdl_wait();
     // every thread copies the same pieces of every page: 2*HD 16-byte pieces of keys, 2*HD of values
     auto issue = [&](int c) {

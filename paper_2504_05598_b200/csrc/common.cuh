@@ -115,6 +115,13 @@ struct Buffers {
     const float *rope_cos, *rope_sin;
 };
 
+// Regions of global memory that a kernel requests into L2 for its successors: up to 3, 16-byte aligned; n = 0: none.
+struct AttnPrefetch {
+    const void *ptr[3];
+    uint32_t bytes[3];
+    int32_t n, pad;
+};
+
 __device__ __forceinline__ size_t stack_row(const Dims &D, int layer, int seq, int slot) {
     return ((size_t)layer * D.B + seq) * D.S + slot;
 }
@@ -153,6 +160,10 @@ __device__ __forceinline__ uint4 ldg_act16_pred(const void *p, bool pred) {
                  "@q ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];\n\t}"
                  : "=&r"(v.x), "=&r"(v.y), "=&r"(v.z), "=&r"(v.w) : "l"(p), "r"((uint32_t)pred));
     return v;
+}
+// request `bytes` (a multiple of 16, 16-byte aligned start) of global memory into L2; nothing waits for it
+__device__ __forceinline__ void l2_prefetch_bulk(const void *p, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
 }
 // 16-byte asynchronous global -> shared copy (zero fill when `pred` is false)
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src, bool pred) {

@@ -57,6 +57,10 @@ struct AttnArgs {
     // Everything later may come from a launch that is still running (the wait of a launch covers its whole chain
     // of predecessors, but nothing bounds how far ahead of that wait a dependent launch may start).  0: nothing.
     int32_t early_pos[DEL_SEQ_MAX];
+    // Weights that the launches after this one stream (the O-projection's, the head of gate / up): requested into L2
+    // by this kernel's CTAs once their own cache reads are on their way, so that HBM works while attention, which is
+    // bound by latency, runs.
+    AttnPrefetch pf;
 };
 cudaError_t launch_attention(const AttnArgs &a, int n_seg, cudaStream_t st, bool pdl);
 int attention_splits(int pages, int n_units, int tiles_par, int n_sms);

@@ -265,6 +265,31 @@ def test_expired_device_wait_is_reported_cleared_and_survivable(small):
     assert rep.rounds == len(ref.rounds)
 
 
+def test_early_reads_and_l2_requests_change_no_result(small):
+    """The decode attention reads committed cache pages and asks for the O-projection's weights before it waits for the
+    QKV launch: scheduling only.  With the weight requests switched off, and through the step calls (whose launches
+    meet other timing), the stream and the last hidden states are bit-identical."""
+    import paper_2504_05598_b200 as dl
+    cfg, w, ctx = small
+    prompt = synth.make_prompt(cfg)
+
+    def run(flags):
+        old = ctx.set_flags(flags)
+        try:
+            toks = [ctx.prefill(0, prompt, cfg.gen_len).tokens[0]]
+            while len(toks) < cfg.gen_len:
+                toks += ctx.round()[0].emitted()
+            return toks, ctx.get_hidden(0, cfg.n_layers, 0).copy()
+        finally:
+            ctx.set_flags(old)
+
+    a = run(dl.FLAG_PDL | dl.FLAG_TC)
+    b = run(dl.FLAG_PDL | dl.FLAG_TC | dl.FLAG_NO_WEIGHT_PREFETCH)
+    c = run(dl.FLAG_TC | dl.FLAG_NO_WEIGHT_PREFETCH)                  # no programmatic dependent launch either
+    assert a[0] == b[0] == c[0] and len(a[0]) == cfg.gen_len
+    assert np.array_equal(a[1], b[1]) and np.array_equal(a[1], c[1])
+
+
 def test_kv_pages_run_out_and_come_back():
     """Two sequences share a page pool that holds one and a half of them: the second prefill is refused with
     DEL_ENOSPC, the first sequence keeps decoding correctly, and after its release the second one fits."""
