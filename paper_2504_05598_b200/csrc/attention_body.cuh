@@ -299,8 +299,9 @@ __device__ __forceinline__ void partial(const AttnView &a, float *sm, const Segm
         }
 #pragma unroll
         for (int j = 0; j < NJ; ++j) vf0[j] = ldg_act8(vpage + (8 * j + g) * 16 + 4 * t);
-        // the warp's further committed pages: into L2 for now (one page per lane, two bulk requests per page)
-        for (int p2 = p_first + n_kl * (1 + lane); p2 < p_end && p2 < (a.early_pos >> 4); p2 += n_kl * 32) {
+        // when weights are requested below: the warp's further committed pages first, into L2 (one page per lane, two
+        // bulk requests per page), so that none of attention's own reads queues behind the weights
+        for (int p2 = p_first + n_kl * (1 + lane); a.pf->n > 0 && p2 < p_end && p2 < (a.early_pos >> 4); p2 += n_kl * 32) {
             const size_t off = (size_t)pt[p2] * page_stride + head_off;
             l2_prefetch_bulk(a.B.KP + off, 16 * HD * 2);
             l2_prefetch_bulk(a.B.VP + off, 16 * HD * 2);
