@@ -699,6 +699,7 @@ def test_full_size_batch_of_four_against_stored_trace():
     doc = json.load(open(path))
     cfg = synth.CONFIGS[name]
     assert doc["seed"] == cfg.seed and len(doc["sequences"]) == cfg.batch
+    assert doc["gen_len"] == cfg.gen_len == 512                  # the whole generation of every sequence, not a prefix
     w = synth.make_weights(cfg)
     ctx = make_ctx(cfg, w)
     refs = [ref_from_golden(doc, s, synth.make_prompt(cfg, s)) for s in range(cfg.batch)]
@@ -706,4 +707,4 @@ def test_full_size_batch_of_four_against_stored_trace():
     for s, rep in enumerate(reps):
         print(f"{name} seq {s}: rounds {rep.rounds} compared {rep.compared} flips {rep.flips} resyncs {rep.resyncs}")
         assert rep.ok(), (s, rep.failures[:8])
-        assert rep.rounds == len(refs[s].rounds)
+        assert rep.rounds == len(refs[s].rounds) >= 300
