@@ -183,8 +183,8 @@ int del_set_policy_fs(del_ctx *ctx, int seq, int E, int gamma0);
  * g_max tokens (del_round) or the given gamma (del_draft) and ends it at the first token whose
  * confidence (top-1 softmax probability of the exit head, fp32) is below the threshold of layer E from
  * Eq. 3; that token is not appended, and its pass through layers 1..E is reused by the verify phase.
- * The host checks the confidence after every draft step (the kernel posts it in pinned host memory and the
- * host polls), so a round then has one host round trip per drafted token instead of one per round.  mode 0 (default) drafts exactly gamma tokens.  The
+ * The kernel that finalises a drafted token takes the decision and posts it in pinned host memory; the host polls for
+ * it before it enqueues the next draft step, so a round then has one host round trip per drafted token instead of one per round.  mode 0 (default) drafts exactly gamma tokens.  The
  * confidence statistics and thresholds are maintained in both modes. */
 int del_set_exit_mode(del_ctx *ctx, int seq, int mode);
 

@@ -140,6 +140,7 @@ __global__ void __launch_bounds__(CTL_THREADS) draft_finalize_embed_kernel(const
         a.B.DCONF[rd.seq * (a.D.S + 1) + rd.slot + 1] = conf;
         if (a.post_conf != nullptr) {
             a.post_conf[rd.seq] = conf;
+            a.post_stop[rd.seq] = (a.exit_tau[rd.seq] > 0.0 && (double)conf < a.exit_tau[rd.seq]) ? 1u : 0u;
             __threadfence_system();              // the confidence is in host memory before the stamp that announces it
             a.post_stamp[rd.seq] = a.stamp;
         }

@@ -82,6 +82,7 @@ struct del_ctx {
     // mailbox of the draft loop's confidence check: pinned host memory that the finalise kernel writes directly
     volatile float *post_conf = nullptr;
     volatile uint32_t *post_stamp = nullptr;
+    volatile uint32_t *post_stop = nullptr;               // the draft loop's break, decided by the finalise kernel
     volatile int32_t *post_out = nullptr;                 // round results posted by the update kernel
     volatile uint32_t *post_done = nullptr;
     uint32_t post_seq = 0;
@@ -553,6 +554,8 @@ int launch_draft_step(del_ctx *c, const DraftStep &st, const std::vector<int> &E
     if (stamp != 0 && c->post_conf != nullptr) {
         ca.post_conf = c->post_conf;
         ca.post_stamp = c->post_stamp;
+        ca.post_stop = c->post_stop;
+        for (int sq = 0; sq < c->D.B; ++sq) ca.exit_tau[sq] = c->seq[sq].exit_mode ? c->seq[sq].cur_tau : 0.0;
         ca.stamp = stamp;
     }
     LAUNCH(launch_draft_finalize_embed(ca, full.m, true, c->st, P));
@@ -613,6 +616,7 @@ int draft_with_exit(del_ctx *c, std::vector<Job> &jobs) {
     }
     const std::vector<int> Es = exit_layers(jobs);
     float *conf_host = reinterpret_cast<float *>(c->stage_host) + 2048;
+    std::vector<char> stop_dev(jobs.size(), 0);
     for (int i = 0; i < gmax; ++i) {
         std::vector<Job> act;
         std::vector<size_t> who;
@@ -643,7 +647,8 @@ int draft_with_exit(del_ctx *c, std::vector<Job> &jobs) {
                 }
                 if (!posted) break;
                 conf_host[k] = c->post_conf[sq];
-                c->d2h_bytes += sizeof(float) + sizeof(uint32_t);
+                stop_dev[k] = c->post_stop[sq] != 0;
+                c->d2h_bytes += sizeof(float) + 2 * sizeof(uint32_t);
             }
         }
         if (!posted) {
@@ -659,7 +664,10 @@ int draft_with_exit(del_ctx *c, std::vector<Job> &jobs) {
         }
         for (size_t k : who) {
             const SeqHost &s = c->seq[jobs[k].seq];
-            if (s.exit_mode && (double)conf_host[k] < s.cur_tau) jobs[k].stopped = 1;   // Algorithm 1: break, token dropped
+            // Algorithm 1: break, token dropped.  The finalise kernel has taken the decision (same comparison: the fp32
+            // confidence widened against the fp64 threshold); the copy fall-back repeats it here.
+            const bool stop = posted ? stop_dev[k] : (s.exit_mode && (double)conf_host[k] < s.cur_tau);
+            if (stop) jobs[k].stopped = 1;
             else jobs[k].g = i + 1;
         }
     }
@@ -1031,7 +1039,7 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
     if (e == cudaSuccess) {
         // mailbox for the draft loop's confidence check (device-writable pinned memory); optional
         void *mb = nullptr;
-        const size_t mb_bytes = 3 * DEL_SEQ_MAX * sizeof(uint32_t) + DEL_SEQ_MAX * sizeof(del_round_out);
+        const size_t mb_bytes = 4 * DEL_SEQ_MAX * sizeof(uint32_t) + DEL_SEQ_MAX * sizeof(del_round_out);
         if (cudaHostAlloc(&mb, mb_bytes, cudaHostAllocMapped) == cudaSuccess) {
             memset(mb, 0, mb_bytes);
             void *dp = nullptr;
@@ -1039,7 +1047,8 @@ int del_init(del_ctx **out, const del_shape *shape, const del_weights *w, const 
                 c->post_conf = reinterpret_cast<volatile float *>(mb);
                 c->post_stamp = reinterpret_cast<volatile uint32_t *>(mb) + DEL_SEQ_MAX;
                 c->post_done = reinterpret_cast<volatile uint32_t *>(mb) + 2 * DEL_SEQ_MAX;
-                c->post_out = reinterpret_cast<volatile int32_t *>(reinterpret_cast<uint32_t *>(mb) + 3 * DEL_SEQ_MAX);
+                c->post_stop = reinterpret_cast<volatile uint32_t *>(mb) + 3 * DEL_SEQ_MAX;
+                c->post_out = reinterpret_cast<volatile int32_t *>(reinterpret_cast<uint32_t *>(mb) + 4 * DEL_SEQ_MAX);
             } else {
                 cudaFreeHost(mb);
             }

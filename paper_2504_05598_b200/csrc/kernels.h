@@ -84,6 +84,10 @@ struct CtlArgs {
     // host memory that the device can write, so that the host sees it without a copy and a stream synchronisation
     volatile float *post_conf;          // [DEL_SEQ_MAX] device-visible host memory, or nullptr
     volatile uint32_t *post_stamp;      // [DEL_SEQ_MAX]
+    // the break of Algorithm 1's draft loop is decided here: per sequence the threshold of its exit layer (0: the
+    // sequence does not use draft-exiting), and where the decision (1: confidence below the threshold) is posted
+    volatile uint32_t *post_stop;       // [DEL_SEQ_MAX]
+    double exit_tau[DEL_SEQ_MAX];
     uint32_t stamp;
     // end of a round: the update kernel also posts every sequence's result (with the device error word as its
     // status) and a stamp there
