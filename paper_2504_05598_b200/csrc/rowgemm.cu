@@ -36,8 +36,8 @@ namespace {
 
 
 // bytes of the reduction buffer, result tile, row scales and arg-max state (16-byte multiple)
-__host__ __device__ constexpr size_t small_smem_bytes(int nt) {
-    return (sizeof(float4) * 8 * nt * 32 + sizeof(float) * (nt * 8 * 16 + 4 * nt * 8) + 15) & ~(size_t)15;
+__host__ __device__ constexpr size_t small_smem_bytes(int nt, int nw) {
+    return (sizeof(float4) * nw * nt * 32 + sizeof(float) * (nt * 8 * 16 + 4 * nt * 8) + 15) & ~(size_t)15;
 }
 
 // The 16 weight rows of a tile are two groups of 8 (MMA rows g and g+8), which need not be adjacent:
@@ -71,14 +71,17 @@ __device__ __forceinline__ void tile_rows(const GemmArgs &a, int item, const bf1
     hi = lo + (size_t)8 * a.K;
 }
 
-template <int NT, int U, int EPI>
-__global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 4 ? 2 : 1)) rowgemm_kernel(const __grid_constant__ GemmArgs a) {
+// NW warps split K: 8 (two CTAs per SM for up to 32 columns), or 16 in one CTA per SM for launches with no more
+// tiles than SMs and a long K, where a second CTA per SM would find no tile and the tile's bursts run in a row
+template <int NT, int U, int EPI, int NW>
+__global__ void __launch_bounds__(NW * 32, (NW == 8 && NT <= 4 ? 2 : 1)) rowgemm_kernel(const __grid_constant__ GemmArgs a) {
+    constexpr int NTHREADS = NW * 32;
     constexpr int NC = NT * 8;                      // MMA columns
     constexpr bool HL = EPI != EPI_LMHEAD;          // columns [0, NR): high parts of NR rows, [NR, NC): their low parts
     constexpr int NR = HL ? NC / 2 : NC;            // activation rows handled
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float4 *red = reinterpret_cast<float4 *>(smem_raw);                       // [8 warps][NT][32]
-    float *res = reinterpret_cast<float *>(smem_raw + sizeof(float4) * 8 * NT * 32);  // [NC][16]
+    float4 *red = reinterpret_cast<float4 *>(smem_raw);                       // [NW warps][NT][32]
+    float *res = reinterpret_cast<float *>(smem_raw + sizeof(float4) * NW * NT * 32);  // [NC][16]
     float *rscale = res + NC * 16;                                      // [NC]
     float *best_v = rscale + NC;                                              // [NC]
     int *best_i = reinterpret_cast<int *>(best_v + NC);                       // [NC]
@@ -87,7 +90,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 4 ? 2 : 1)) rowgemm_k
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g = lane >> 2, t = lane & 3;
     const int K = a.K;
     const int n_ksteps = (K + 31) >> 5;
-    const int nkw = (n_ksteps + 7) >> 3;            // k-steps per warp and tile (the last ones may be empty)
+    const int nkw = (n_ksteps + NW - 1) / NW;       // k-steps per warp and tile (the last ones may be empty)
     __shared__ int s_claim[2];                      // tile claimed for the turn after next (double-buffered)
 
     uint4 wa[U], wb[U];
@@ -105,7 +108,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 4 ? 2 : 1)) rowgemm_k
     auto load_w = [&](int u0, bool live) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int k0 = (warp + 8 * (u0 + u)) << 5;
+            const int k0 = (warp + NW * (u0 + u)) << 5;
             const bool ok = live && (u0 + u < nkw) && (k0 + 8 * t < K);
             wa[u] = ldg_stream16_pred(base + k0, ok);
             wb[u] = ldg_stream16_pred(base_hi + k0, ok);
@@ -114,7 +117,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 4 ? 2 : 1)) rowgemm_k
     auto load_x = [&](int u0, bool live) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int k0 = ((warp + 8 * (u0 + u)) << 5) + 8 * t;
+            const int k0 = ((warp + NW * (u0 + u)) << 5) + 8 * t;
             const bool ok = live && (u0 + u < nkw) && (k0 < K);
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) xv[u][nt] = ldg_act16_pred(xrow[nt] + k0, ok && xrow[nt] != nullptr);
@@ -175,7 +178,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 4 ? 2 : 1)) rowgemm_k
         }
     }
     if (EPI == EPI_LMHEAD) {
-        for (int c = tid; c < NC; c += DEL_GEMM_THREADS) { best_v[c] = -INFINITY; best_i[c] = 0x7fffffff; best_s[c] = 0.f; }
+        for (int c = tid; c < NC; c += NTHREADS) { best_v[c] = -INFINITY; best_i[c] = 0x7fffffff; best_s[c] = 0.f; }
     }
     // no barrier here: rscale / best_* are first read in an epilogue, after the two barriers of tile_end
 
@@ -193,10 +196,10 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 4 ? 2 : 1)) rowgemm_k
             acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
         }
         __syncthreads();
-        for (int e = tid; e < NT * 32; e += DEL_GEMM_THREADS) {
+        for (int e = tid; e < NT * 32; e += NTHREADS) {
             float4 s = red[e];
 #pragma unroll
-            for (int w = 1; w < DEL_GEMM_WARPS; ++w) {
+            for (int w = 1; w < NW; ++w) {
                 const float4 v = red[w * NT * 32 + e];
                 s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
             }
@@ -207,7 +210,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 4 ? 2 : 1)) rowgemm_k
         __syncthreads();
         const int item = cur_item;
         const int i = tid & 15;
-        for (int cl = tid >> 4; cl < NR; cl += DEL_GEMM_THREADS / 16) {
+        for (int cl = tid >> 4; cl < NR; cl += NTHREADS / 16) {
             const int c = row0 + cl;                // row of the pass; cl: its column in this launch
             const bool valid = c < m;
             const RowDesc rd = valid ? plan->rows[c] : RowDesc{0, 0, 0, 0};
@@ -328,7 +331,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 4 ? 2 : 1)) rowgemm_k
 
     mma_burst();
     if (EPI == EPI_QKV || EPI == EPI_GATEUP) {
-        for (int cl = warp; cl < NR; cl += DEL_GEMM_WARPS) {
+        for (int cl = warp; cl < NR; cl += NW) {
             const int c = row0 + cl;
             float s = 0.f;
             if (cl == warp) {
@@ -345,7 +348,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 4 ? 2 : 1)) rowgemm_k
         }
     }
     if (EPI == EPI_LMHEAD) {
-        for (int c = warp; c < NC; c += DEL_GEMM_WARPS) {
+        for (int c = warp; c < NC; c += NW) {
             float k = 0.f;
             if (c < m) {
                 if (a.row_scale) {
@@ -392,7 +395,7 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 4 ? 2 : 1)) rowgemm_k
 
     if (EPI == EPI_LMHEAD) {
         __syncthreads();
-        for (int c = tid; c < m; c += DEL_GEMM_THREADS) {
+        for (int c = tid; c < m; c += NTHREADS) {
             a.B.LPV[(size_t)blockIdx.x * DEL_ROWS_MAX + c] = best_v[c];
             a.B.LPI[(size_t)blockIdx.x * DEL_ROWS_MAX + c] = best_i[c];
             if (a.B.LPS) a.B.LPS[(size_t)blockIdx.x * DEL_ROWS_MAX + c] = best_s[c];
@@ -402,12 +405,12 @@ __global__ void __launch_bounds__(DEL_GEMM_THREADS, (NT <= 4 ? 2 : 1)) rowgemm_k
 
 template <int NT> constexpr int depth_for() { return NT == 1 ? 8 : (NT <= 4 ? 4 : 3); }
 
-template <int NT, int EPI>
+template <int NT, int EPI, int NW = DEL_GEMM_WARPS>
 cudaError_t launch_nt(const GemmArgs &a, int grid, cudaStream_t st, bool pdl) {
     constexpr int D = depth_for<NT>();
     constexpr int NC = NT * 8;
-    const size_t smem = small_smem_bytes(NT);
-    auto kern = rowgemm_kernel<NT, D, EPI>;
+    const size_t smem = small_smem_bytes(NT, NW);
+    auto kern = rowgemm_kernel<NT, D, EPI, NW>;
     static SmemAttrOnce attr;
     {
         cudaError_t e = attr.set(kern, (int)((int)smem));
@@ -415,7 +418,7 @@ cudaError_t launch_nt(const GemmArgs &a, int grid, cudaStream_t st, bool pdl) {
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(DEL_GEMM_THREADS);
+    cfg.blockDim = dim3(NW * 32);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute at[1];
@@ -431,7 +434,13 @@ template <int EPI>
 cudaError_t launch_epi(const GemmArgs &a, int m, int n_sms, cudaStream_t st, bool pdl) {
     const int nt = EPI == EPI_LMHEAD ? (m + 7) / 8 : (m + 3) / 4;
     const int per_sm = a.ctas_per_sm == 1 ? 1 : 2;
-    if (nt <= 1) return launch_nt<1, EPI>(a, min(a.n_items, per_sm * n_sms), st, pdl);
+    if (nt <= 1) {
+        // no more tiles than SMs and at least two bursts per warp even with 16 warps: one CTA of 16 warps per tile
+        if constexpr (EPI == EPI_OPROJ || EPI == EPI_DOWN) {
+            if (a.n_items <= n_sms && a.K >= 2 * 16 * 32 * depth_for<1>()) return launch_nt<1, EPI, 16>(a, a.n_items, st, pdl);
+        }
+        return launch_nt<1, EPI>(a, min(a.n_items, per_sm * n_sms), st, pdl);
+    }
     if (nt <= 2) return launch_nt<2, EPI>(a, min(a.n_items, per_sm * n_sms), st, pdl);
     if (nt <= 4) return launch_nt<4, EPI>(a, min(a.n_items, per_sm * n_sms), st, pdl);
     return launch_nt<8, EPI>(a, min(a.n_items, n_sms), st, pdl);
