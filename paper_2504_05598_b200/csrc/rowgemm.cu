@@ -188,6 +188,46 @@ __global__ void __launch_bounds__(NW * 32, (NW == 8 && NT <= 4 ? 2 : 1)) rowgemm
 
     int turn = 0;
 
+    // The residual element that this thread's epilogue adds (O-projection: the hidden stack; down: the stream after
+    // attention) is requested when the tile starts, so that the epilogue of a CTA's last tile does not begin with a
+    // round trip to L2.  One element per thread; the 8- and 16-column variants only (the wider ones have no register
+    // to spare).
+    constexpr bool RES_PRE = (EPI == EPI_OPROJ || EPI == EPI_DOWN) && NT <= 2;
+    float h_pre = 0.f;
+    bf16 ga_pre = __float2bfloat16_rn(0.f), gb_pre = __float2bfloat16_rn(0.f);      // the norm gains of that output feature
+    // QKV: the rotation's cos / sin of this thread's pair and the cache page of its row
+    constexpr bool ROPE_PRE = EPI == EPI_QKV && NT <= 2;
+    float cs_pre = 0.f, sn_pre = 0.f;
+    int pg_pre = 0;
+    if (ROPE_PRE) {
+        const int cl = tid >> 4, c = row0 + cl;
+        if (cl < NR && c < m) pg_pre = a.B.PT[plan->rows[c].seq * a.D.pages_per_seq + (plan->rows[c].pos >> 4)];
+    }
+    auto prefetch_residual = [&](int item) {
+        if (RES_PRE) {
+            const int cl = tid >> 4, c = row0 + cl;
+            if (cl < NR && c < m) {
+                const int o = 16 * item + (tid & 15);
+                if (EPI == EPI_OPROJ) h_pre = ldg_cg_f32(a.B.H + stack_row(a.D, a.layer - 1, plan->rows[c].seq, plan->rows[c].slot) * a.D.d + o);
+                else h_pre = ldg_cg_f32(a.B.HM + (size_t)c * a.D.d + o);
+                if (a.gain_a) ga_pre = a.gain_a[o];
+                if (EPI == EPI_DOWN && a.gain_b) gb_pre = a.gain_b[o];
+            }
+        }
+        if (ROPE_PRE) {
+            const int cl = tid >> 4, c = row0 + cl, i = tid & 15;
+            const int hd = a.D.hd, half = hd >> 1, h8 = hd >> 4;
+            const int nq = a.D.nh * h8, nk = a.D.nkv * h8;
+            if (cl < NR && c < m && i < 8 && item < nq + nk) {
+                const int it = item < nq ? item : item - nq;
+                const int j = (it - (it / h8) * h8) * 8 + i;
+                cs_pre = a.B.rope_cos[(size_t)plan->rows[c].pos * half + j];
+                sn_pre = a.B.rope_sin[(size_t)plan->rows[c].pos * half + j];
+            }
+        }
+    };
+    prefetch_residual(cur_item);
+
     auto tile_end = [&]() {
         // fixed-order sum of the 8 warps' partials
 #pragma unroll
@@ -223,7 +263,7 @@ __global__ void __launch_bounds__(NW * 32, (NW == 8 && NT <= 4 ? 2 : 1)) rowgemm
                 const float r = rscale[cl];
                 const int hd = a.D.hd, half = hd >> 1, h8 = hd >> 4;
                 const int nq = a.D.nh * h8, nk = a.D.nkv * h8;
-                const int pg = a.B.PT[rd.seq * a.D.pages_per_seq + (rd.pos >> 4)];
+                const int pg = ROPE_PRE ? pg_pre : a.B.PT[rd.seq * a.D.pages_per_seq + (rd.pos >> 4)];
                 const int sl = rd.pos & 15;
                 if (item < nq + nk) {
                     if (i >= 8) continue;                         // rows 0..7 and their partners 8..15: one thread per pair
@@ -231,7 +271,8 @@ __global__ void __launch_bounds__(NW * 32, (NW == 8 && NT <= 4 ? 2 : 1)) rowgemm
                     const bool isq = item < nq;
                     const int it = isq ? item : item - nq;
                     const int head = it / h8, j = (it - head * h8) * 8 + i;
-                    const float cs = a.B.rope_cos[(size_t)rd.pos * half + j], sn = a.B.rope_sin[(size_t)rd.pos * half + j];
+                    const float cs = ROPE_PRE ? cs_pre : a.B.rope_cos[(size_t)rd.pos * half + j];
+                    const float sn = ROPE_PRE ? sn_pre : a.B.rope_sin[(size_t)rd.pos * half + j];
                     const float oa = va * cs - vb * sn, ob = vb * cs + va * sn;
                     if (isq) {
                         bf16 *q = a.B.Q + (size_t)c * (a.D.nh * hd) + head * hd + j;
@@ -259,16 +300,16 @@ __global__ void __launch_bounds__(NW * 32, (NW == 8 && NT <= 4 ? 2 : 1)) rowgemm
                 float h = 0.f;
                 if (valid) {
                     if (EPI == EPI_OPROJ) {
-                        h = ldg_cg_f32(a.B.H + stack_row(a.D, a.layer - 1, rd.seq, rd.slot) * a.D.d + o) + ra;
+                        h = (RES_PRE ? h_pre : ldg_cg_f32(a.B.H + stack_row(a.D, a.layer - 1, rd.seq, rd.slot) * a.D.d + o)) + ra;
                         a.B.HM[(size_t)c * a.D.d + o] = h;
-                        split_bf16(h * bf16_to_f(a.gain_a[o]), a.B.XM[(size_t)c * a.D.d + o], a.B.XML[(size_t)c * a.D.d + o]);
+                        split_bf16(h * bf16_to_f(RES_PRE ? ga_pre : a.gain_a[o]), a.B.XM[(size_t)c * a.D.d + o], a.B.XML[(size_t)c * a.D.d + o]);
                     } else {
-                        h = ldg_cg_f32(a.B.HM + (size_t)c * a.D.d + o) + ra;
+                        h = (RES_PRE ? h_pre : ldg_cg_f32(a.B.HM + (size_t)c * a.D.d + o)) + ra;
                         const size_t sr = stack_row(a.D, a.layer, rd.seq, rd.slot);
                         a.B.H[sr * a.D.d + o] = h;
-                        if (a.gain_a) split_bf16(h * bf16_to_f(a.gain_a[o]), a.B.XS[sr * a.D.d + o], a.B.XSL[sr * a.D.d + o]);
+                        if (a.gain_a) split_bf16(h * bf16_to_f(RES_PRE ? ga_pre : a.gain_a[o]), a.B.XS[sr * a.D.d + o], a.B.XSL[sr * a.D.d + o]);
                         if (a.gain_b)
-                            a.B.XE[((size_t)rd.seq * a.D.S + rd.slot) * a.D.d + o] = __float2bfloat16_rn(h * bf16_to_f(a.gain_b[o]));
+                            a.B.XE[((size_t)rd.seq * a.D.S + rd.slot) * a.D.d + o] = __float2bfloat16_rn(h * bf16_to_f(RES_PRE ? gb_pre : a.gain_b[o]));
                     }
                 }
                 float ss = h * h;
@@ -389,6 +430,7 @@ __global__ void __launch_bounds__(NW * 32, (NW == 8 && NT <= 4 ? 2 : 1)) rowgemm
         nxt_item = (after >= 0 && after < a.n_items) ? after : -1;
         ++turn;
         claim();
+        prefetch_residual(cur_item);
         mma_burst();
         u0 = U;
     }
