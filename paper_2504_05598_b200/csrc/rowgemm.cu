@@ -190,13 +190,13 @@ __global__ void __launch_bounds__(NW * 32, (NW == 8 && NT <= 4 ? 2 : 1)) rowgemm
 
     // The residual element that this thread's epilogue adds (O-projection: the hidden stack; down: the stream after
     // attention) is requested when the tile starts, so that the epilogue of a CTA's last tile does not begin with a
-    // round trip to L2.  One element per thread; the 8- and 16-column variants only (the wider ones have no register
-    // to spare).
-    constexpr bool RES_PRE = (EPI == EPI_OPROJ || EPI == EPI_DOWN) && NT <= 2;
+    // round trip to L2.  One element per thread; the 8-column variant only (the 16-column one does not gain, the wider
+    // ones have no register to spare).
+    constexpr bool RES_PRE = (EPI == EPI_OPROJ || EPI == EPI_DOWN) && NT == 1;
     float h_pre = 0.f;
     bf16 ga_pre = __float2bfloat16_rn(0.f), gb_pre = __float2bfloat16_rn(0.f);      // the norm gains of that output feature
     // QKV: the rotation's cos / sin of this thread's pair and the cache page of its row
-    constexpr bool ROPE_PRE = EPI == EPI_QKV && NT <= 2;
+    constexpr bool ROPE_PRE = EPI == EPI_QKV && NT == 1;
     float cs_pre = 0.f, sn_pre = 0.f;
     int pg_pre = 0;
     if (ROPE_PRE) {
