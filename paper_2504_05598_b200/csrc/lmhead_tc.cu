@@ -3,7 +3,7 @@
 // W_lm is streamed from HBM once for all R = L * (gamma + 1) rows of the round.
 //
 // CTA tile: 128 rows x 256 vocabulary entries, K blocks of 64 (one 128-byte swizzle span).  Roles:
-//   warp 0     one lane issues the TMA loads (cp.async.bulk.tensor, no multicast) of the Xn tile
+//   warp 0     one lane issues the TMA loads (cp.async.bulk.tensor, every CTA loads its own tiles) of the Xn tile
 //              [128 x 64] and the W_lm tile [256 x 64] into a 4-stage shared-memory ring;
 //   warp 1     allocates tensor memory; one lane issues tcgen05.mma (M 128, N 256, K 16, bf16 inputs,
 //              fp32 accumulators in TMEM) and commits each stage back to the producer;

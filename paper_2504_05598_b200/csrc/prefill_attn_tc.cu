@@ -3,8 +3,8 @@
 // One CTA = 128 query rows of one query head.  Keys and values come from the paged cache in blocks of 64
 // keys (four pages): the key pages [16 tokens][128 dims] and the value pages, which the cache stores transposed
 // ([128 dims][16 tokens]), are exactly the K-major operand tiles tcgen05.mma wants, so TMA copies them as they lie
-// (cp.async.bulk.tensor over 5-d maps of the cache, 128-byte swizzle for keys, 32-byte swizzle for values, no
-// multicast) and nothing is transposed.  Per key block:
+// (cp.async.bulk.tensor over 5-d maps of the cache, 128-byte swizzle for keys, 32-byte swizzle for values, every
+// CTA loading its own tiles) and nothing is transposed.  Per key block:
 //   S = Q K^T        16 MMAs (M 128, N 64, K 16) into one of two 64-column accumulators in tensor memory;
 //   softmax          four warps, one thread per query row: tcgen05.ld of the row's 64 scores, scale, causal mask,
 //                    p = 2^(s - m) against a lazily raised reference maximum m (the running output in tensor

@@ -1,5 +1,5 @@
 // tcgen05 / TMA / mbarrier building blocks shared by the tensor-core kernels (stacked LM head, prefill
-// GEMMs): one elected thread issues TMA loads (cp.async.bulk.tensor, no multicast) and tcgen05.mma, the
+// GEMMs): one elected thread issues TMA loads (cp.async.bulk.tensor, every CTA loads its own tiles) and tcgen05.mma, the
 // accumulators live in tensor memory and are read back with tcgen05.ld.  Every mbarrier wait is bounded.
 #pragma once
 
