@@ -478,7 +478,7 @@ cudaError_t launch_epi(const GemmArgs &a, int m, int n_sms, cudaStream_t st, boo
     const int per_sm = a.ctas_per_sm == 1 ? 1 : 2;
     if (nt <= 1) {
         // no more tiles than SMs and at least two bursts per warp even with 16 warps: one CTA of 16 warps per tile
-        if constexpr (EPI == EPI_OPROJ || EPI == EPI_DOWN) {
+        if constexpr (EPI == EPI_DOWN) {
             if (a.n_items <= n_sms && a.K >= 2 * 16 * 32 * depth_for<1>()) return launch_nt<1, EPI, 16>(a, a.n_items, st, pdl);
         }
         return launch_nt<1, EPI>(a, min(a.n_items, per_sm * n_sms), st, pdl);
