@@ -34,18 +34,18 @@ __global__ void __launch_bounds__(NW * 32) attention_kernel(const __grid_constan
     else attn::partial<HD>(v, sm, seg, kvh, p_begin, p_end, 0, 0x7fffffff, split, n_splits);
 
     if (n_splits > 1) {
-        __threadfence();
+        // The CTA's partial states are published by one release-acquire ticket: the barrier orders every thread's
+        // stores before thread 0's release, and the last CTA's acquire, followed by its barrier, orders all splits'
+        // stores before the merge's loads (which go to L2, not to L1).
         __syncthreads();
         if (threadIdx.x == 0) {
-            const int ticket = atomicAdd(a.B.ACNT + blockIdx.z * a.D.nkv + kvh, 1);
+            int ticket;
+            asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(ticket) : "l"(a.B.ACNT + blockIdx.z * a.D.nkv + kvh) : "memory");
             s_last = (ticket == n_splits - 1);
             if (s_last) a.B.ACNT[blockIdx.z * a.D.nkv + kvh] = 0;     // ready for the next launch
         }
         __syncthreads();
-        if (s_last) {
-            __threadfence();
-            attn::merge_slots<HD>(v, seg, kvh, n_splits);
-        }
+        if (s_last) attn::merge_slots<HD>(v, seg, kvh, n_splits);
     }
 }
 
